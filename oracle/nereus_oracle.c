@@ -1,0 +1,362 @@
+/*
+ * TEST INFRASTRUCTURE -- NOT PART OF THE PRODUCT.
+ *
+ * Plain, slow, single-threaded CPU oracle for the EMU reshard: the layout
+ * change that carries one model-stage's parameter shards theta = {theta_i},
+ * i = 1..tp*pp (EMU definition, Section 5) from a source (TP, PP) layout to a
+ * target (TP, PP) layout.  Split and Merge "change placement and sharding
+ * without changing logical state" (Section 6.2, "Preserving training
+ * semantics"), and Split is a position-wise AllGather followed by a local
+ * layout change (Section 6.2, "DAG Execution and Safety" and
+ * "Resharding--transport interplay").  So the result has a plain definition
+ * and this file is that definition written out, per logical tensor:
+ *
+ *     1. GATHER  the full logical tensor [rows][cols] from the source shards,
+ *     2. CAST    element by element when the target dtype differs (fp32->bf16,
+ *                round to nearest even),
+ *     3. SLICE   it by the target plan's rule into the target shards.
+ *
+ * The paper fixes none of the tensor-level layout (fused QKV, fused gate/up,
+ * vocabulary rows, row-parallel columns, packing of a shard buffer, the cast):
+ * those are this build's layout contract.  They are "parity unpinned" by the
+ * paper; what pins them is stated next to each function and in the tests
+ * (identity, round trip, np.split/np.concatenate special cases, a brute-force
+ * per-element owner function, checksum conservation, published parameter
+ * counts, torch's fp32->bf16 conversion over all 2^32 inputs).
+ *
+ * Only tests, the smoke check and the benchmark's cpu_baseline / reference
+ * arm may build, load or call this file.  It shares no code with the CUDA
+ * path and includes none of its headers.
+ *
+ * Layout contract (restated here on purpose, independently of the product):
+ *   model      L layers, hidden H, nq query heads, nkv KV heads, hd = H / nq,
+ *              FFN F, vocabulary V, element size es (2 = bf16, 4 = fp32),
+ *              optional value head [1, H] in place of the LM head [V, H].
+ *   plan       (tp, pp): pipeline stage p owns layers [p*L/pp, (p+1)*L/pp),
+ *              the embedding lives on stage 0, final norm + head on stage
+ *              pp-1; shard index = p * tp + r  (TP rank fastest).
+ *   TP rank r of t holds
+ *     embed, LM head [V, H]   rows    [r*V/t, (r+1)*V/t)
+ *     wq [nq*hd, H]           rows of q heads  [r*nq/t, (r+1)*nq/t)
+ *     wk, wv [nkv*hd, H]      rows of kv heads [r*nkv/t, (r+1)*nkv/t)
+ *     wo [H, nq*hd]           columns [r*nq*hd/t, (r+1)*nq*hd/t)
+ *     wgate, wup [F, H]       rows    [r*F/t, (r+1)*F/t)
+ *     wdown [H, F]            columns [r*F/t, (r+1)*F/t)
+ *     ln1, ln2, ln_f [H], value head [1, H]   whole tensor (replicated)
+ *   shard buffer packing, every stored tensor starting on a 256-byte boundary:
+ *     [embed], then per local layer: ln1, {wq;wk;wv} fused, wo, ln2,
+ *     {wgate;wup} fused, wdown, then [ln_f, head].
+ *     Inside the fused QKV block the rank's Q rows come first, then its K
+ *     rows, then its V rows; inside gate/up the rank's gate rows, then its up
+ *     rows.  The buffer length is the end of the last tensor rounded up to
+ *     256 bytes.  Padding bytes are never read and never written.
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#include <stddef.h>
+
+enum { ORACLE_OK = 0, ORACLE_ERR_ARG = -1, ORACLE_ERR_INDIVISIBLE = -2,
+       ORACLE_ERR_UNSUPPORTED = -3, ORACLE_ERR_REPLICA_MISMATCH = -4,
+       ORACLE_ERR_NOMEM = -5 };
+
+enum { ORACLE_BF16 = 1, ORACLE_FP32 = 2 };
+
+typedef struct {
+    int64_t L, H, nq, nkv, F, V;
+    int dtype;        /* ORACLE_BF16 or ORACLE_FP32: dtype of a plan whose dtype field is 0 */
+    int value_head;   /* 0: LM head [V, H]; 1: value head [1, H] */
+} oracle_model;
+
+typedef struct { int tp, pp, dtype; } oracle_plan;
+
+/* kinds of logical tensor */
+enum { K_EMBED, K_LN1, K_WQ, K_WK, K_WV, K_WO, K_LN2, K_WGATE, K_WUP, K_WDOWN, K_LNF, K_HEAD };
+
+static int64_t align256(int64_t x) { return (x + 255) / 256 * 256; }
+
+static int plan_es(const oracle_model* m, oracle_plan p) {
+    int d = p.dtype ? p.dtype : m->dtype;
+    return d == ORACLE_FP32 ? 4 : 2;
+}
+
+int64_t oracle_num_logical(const oracle_model* m) { return 9 * m->L + 3; }
+
+/* logical id -> (kind, layer).  Order: embed, per layer ln1 wq wk wv wo ln2 wgate wup wdown, ln_f, head */
+static void decode_id(const oracle_model* m, int64_t id, int* kind, int64_t* layer) {
+    static const int per_layer[9] = { K_LN1, K_WQ, K_WK, K_WV, K_WO, K_LN2, K_WGATE, K_WUP, K_WDOWN };
+    if (id == 0) { *kind = K_EMBED; *layer = -1; return; }
+    if (id == 9 * m->L + 1) { *kind = K_LNF; *layer = -1; return; }
+    if (id == 9 * m->L + 2) { *kind = K_HEAD; *layer = -1; return; }
+    *layer = (id - 1) / 9;
+    *kind = per_layer[(id - 1) % 9];
+}
+
+/* Full logical shape [rows][cols] of a tensor kind. */
+static void kind_shape(const oracle_model* m, int kind, int64_t* rows, int64_t* cols) {
+    int64_t hd = m->H / m->nq;
+    switch (kind) {
+    case K_EMBED:  *rows = m->V;        *cols = m->H; break;
+    case K_HEAD:   *rows = m->value_head ? 1 : m->V; *cols = m->H; break;
+    case K_LN1: case K_LN2: case K_LNF: *rows = 1; *cols = m->H; break;
+    case K_WQ:     *rows = m->nq * hd;  *cols = m->H; break;
+    case K_WK: case K_WV: *rows = m->nkv * hd; *cols = m->H; break;
+    case K_WO:     *rows = m->H;        *cols = m->nq * hd; break;
+    case K_WGATE: case K_WUP: *rows = m->F; *cols = m->H; break;
+    case K_WDOWN:  *rows = m->H;        *cols = m->F; break;
+    default:       *rows = 0;           *cols = 0;
+    }
+}
+
+int oracle_logical_shape(const oracle_model* m, int64_t id, int64_t* rows, int64_t* cols) {
+    int kind; int64_t layer;
+    if (!m || id < 0 || id >= oracle_num_logical(m)) return ORACLE_ERR_ARG;
+    decode_id(m, id, &kind, &layer);
+    kind_shape(m, kind, rows, cols);
+    return ORACLE_OK;
+}
+
+int oracle_check_plan(const oracle_model* m, oracle_plan p) {
+    if (!m || p.tp < 1 || p.pp < 1) return ORACLE_ERR_ARG;
+    if (m->L < 1 || m->H < 1 || m->nq < 1 || m->nkv < 1 || m->F < 1 || m->V < 1) return ORACLE_ERR_ARG;
+    if (m->H % m->nq || m->nq % m->nkv) return ORACLE_ERR_INDIVISIBLE;
+    if (p.tp > m->nkv) return ORACLE_ERR_UNSUPPORTED;      /* no KV-head replication */
+    if (m->nkv % p.tp || m->nq % p.tp || m->F % p.tp || m->V % p.tp || m->L % p.pp)
+        return ORACLE_ERR_INDIVISIBLE;
+    return ORACLE_OK;
+}
+
+/* The part of a logical tensor of `kind` that TP rank r of t holds:
+ * rows [*r0, *r0 + *nr), columns [*c0, *c0 + *nc) of the full tensor. */
+static void rank_part(const oracle_model* m, int kind, int64_t r, int64_t t,
+                      int64_t* r0, int64_t* nr, int64_t* c0, int64_t* nc) {
+    int64_t rows, cols;
+    kind_shape(m, kind, &rows, &cols);
+    *r0 = 0; *nr = rows; *c0 = 0; *nc = cols;
+    switch (kind) {
+    case K_EMBED: case K_WQ: case K_WK: case K_WV: case K_WGATE: case K_WUP:
+        *nr = rows / t; *r0 = r * (rows / t); break;            /* dim-0 (column-parallel) */
+    case K_HEAD:
+        if (!m->value_head) { *nr = rows / t; *r0 = r * (rows / t); }
+        break;                                                  /* value head: replicated */
+    case K_WO: case K_WDOWN:
+        *nc = cols / t; *c0 = r * (cols / t); break;            /* dim-1 (row-parallel) */
+    default: break;                                             /* norms: replicated */
+    }
+}
+
+static int kind_replicated(const oracle_model* m, int kind) {
+    return kind == K_LN1 || kind == K_LN2 || kind == K_LNF || (kind == K_HEAD && m->value_head);
+}
+
+/* Elements of `kind` stored by one TP rank of t. */
+static int64_t rank_elems(const oracle_model* m, int kind, int64_t t) {
+    int64_t r0, nr, c0, nc;
+    rank_part(m, kind, 0, t, &r0, &nr, &c0, &nc);
+    return nr * nc;
+}
+
+/* Walk the packing order of shard (stage p, any TP rank) and return the byte
+ * offset of the first element of logical tensor (kind, layer), or -1 if the
+ * stage does not hold it.  *total gets the shard buffer length. */
+static int64_t pack_offset(const oracle_model* m, oracle_plan pl, int64_t p,
+                           int want_kind, int64_t want_layer, int64_t* total) {
+    int64_t es = plan_es(m, pl), t = pl.tp, cur = 0, found = -1;
+    int64_t lps = m->L / pl.pp;
+    if (p == 0) {
+        cur = align256(cur);
+        if (want_kind == K_EMBED) found = cur;
+        cur += rank_elems(m, K_EMBED, t) * es;
+    }
+    for (int64_t l = p * lps; l < (p + 1) * lps; ++l) {
+        int hit = (l == want_layer);
+        cur = align256(cur);                                    /* ln1 */
+        if (hit && want_kind == K_LN1) found = cur;
+        cur += rank_elems(m, K_LN1, t) * es;
+        cur = align256(cur);                                    /* fused q;k;v */
+        if (hit && want_kind == K_WQ) found = cur;
+        cur += rank_elems(m, K_WQ, t) * es;
+        if (hit && want_kind == K_WK) found = cur;
+        cur += rank_elems(m, K_WK, t) * es;
+        if (hit && want_kind == K_WV) found = cur;
+        cur += rank_elems(m, K_WV, t) * es;
+        cur = align256(cur);                                    /* wo */
+        if (hit && want_kind == K_WO) found = cur;
+        cur += rank_elems(m, K_WO, t) * es;
+        cur = align256(cur);                                    /* ln2 */
+        if (hit && want_kind == K_LN2) found = cur;
+        cur += rank_elems(m, K_LN2, t) * es;
+        cur = align256(cur);                                    /* fused gate;up */
+        if (hit && want_kind == K_WGATE) found = cur;
+        cur += rank_elems(m, K_WGATE, t) * es;
+        if (hit && want_kind == K_WUP) found = cur;
+        cur += rank_elems(m, K_WUP, t) * es;
+        cur = align256(cur);                                    /* wdown */
+        if (hit && want_kind == K_WDOWN) found = cur;
+        cur += rank_elems(m, K_WDOWN, t) * es;
+    }
+    if (p == pl.pp - 1) {
+        cur = align256(cur);
+        if (want_kind == K_LNF) found = cur;
+        cur += rank_elems(m, K_LNF, t) * es;
+        cur = align256(cur);
+        if (want_kind == K_HEAD) found = cur;
+        cur += rank_elems(m, K_HEAD, t) * es;
+    }
+    if (total) *total = align256(cur);
+    return found;
+}
+
+int oracle_num_shards(const oracle_model* m, oracle_plan pl, int64_t* n) {
+    int rc = oracle_check_plan(m, pl);
+    if (rc) return rc;
+    *n = (int64_t)pl.tp * pl.pp;
+    return ORACLE_OK;
+}
+
+int oracle_shard_bytes(const oracle_model* m, oracle_plan pl, int64_t shard, int64_t* bytes) {
+    int rc = oracle_check_plan(m, pl);
+    if (rc) return rc;
+    if (shard < 0 || shard >= (int64_t)pl.tp * pl.pp) return ORACLE_ERR_ARG;
+    pack_offset(m, pl, shard / pl.tp, -1, -1, bytes);
+    return ORACLE_OK;
+}
+
+/* Where shard `shard` of plan `pl` keeps its part of logical tensor `id`:
+ * byte offset of the part's first element in the shard buffer, and the part's
+ * position [r0, r0+nr) x [c0, c0+nc) in the full tensor.  The part is stored
+ * row-major with nc elements per row.  *held = 0 when the shard's stage does
+ * not own the tensor. */
+int oracle_locate(const oracle_model* m, oracle_plan pl, int64_t shard, int64_t id,
+                  int* held, int64_t* offset, int64_t* r0, int64_t* nr, int64_t* c0, int64_t* nc) {
+    int kind; int64_t layer, off;
+    int rc = oracle_check_plan(m, pl);
+    if (rc) return rc;
+    if (shard < 0 || shard >= (int64_t)pl.tp * pl.pp || id < 0 || id >= oracle_num_logical(m))
+        return ORACLE_ERR_ARG;
+    decode_id(m, id, &kind, &layer);
+    off = pack_offset(m, pl, shard / pl.tp, kind, layer, NULL);
+    *held = off >= 0;
+    *offset = off >= 0 ? off : 0;
+    rank_part(m, kind, shard % pl.tp, pl.tp, r0, nr, c0, nc);
+    if (!*held) { *nr = 0; *nc = 0; }
+    return ORACLE_OK;
+}
+
+/* fp32 -> bf16, round to nearest, ties to even, on the bit pattern.
+ * NaN (any payload, either sign) -> 0x7FC0; everything else
+ * (u + 0x7FFF + lsb) >> 16, so finite values beyond the bf16 range become
+ * +-Inf, signed zeros keep their sign and subnormals are rounded, not flushed.
+ * The cast belongs to this build's contract (train -> generation weight sync
+ * between the actor's two model-stages, Section 5); the paper states no
+ * precision. */
+uint16_t oracle_rne_bf16(uint32_t u) {
+    if ((u & 0x7FFFFFFFu) > 0x7F800000u) return 0x7FC0;
+    return (uint16_t)((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);
+}
+
+void oracle_rne_bf16_array(const uint32_t* in, uint16_t* out, int64_t n) {
+    for (int64_t i = 0; i < n; ++i) out[i] = oracle_rne_bf16(in[i]);
+}
+
+/* One logical tensor: gather -> cast -> slice.
+ * src_parts[i] / dst_parts[i] point at the FIRST ELEMENT of shard i's part of
+ * this tensor (host memory), or are ignored for shards that do not hold it. */
+int oracle_reshard_tensor_parts(const oracle_model* m, oracle_plan sp, oracle_plan dp, int64_t id,
+                                const void* const* src_parts, void* const* dst_parts) {
+    int rc, held, kind; int64_t layer, rows, cols, off, r0, nr, c0, nc;
+    if ((rc = oracle_check_plan(m, sp))) return rc;
+    if ((rc = oracle_check_plan(m, dp))) return rc;
+    if (id < 0 || id >= oracle_num_logical(m) || !src_parts || !dst_parts) return ORACLE_ERR_ARG;
+    int64_t ses = plan_es(m, sp), des = plan_es(m, dp);
+    if (!(ses == des || (ses == 4 && des == 2))) return ORACLE_ERR_UNSUPPORTED;
+    decode_id(m, id, &kind, &layer);
+    kind_shape(m, kind, &rows, &cols);
+
+    unsigned char* full = (unsigned char*)malloc((size_t)(rows * cols * ses));
+    if (!full) return ORACLE_ERR_NOMEM;
+
+    /* 1. GATHER */
+    int first_replica = 1;
+    for (int64_t s = 0; s < (int64_t)sp.tp * sp.pp; ++s) {
+        oracle_locate(m, sp, s, id, &held, &off, &r0, &nr, &c0, &nc);
+        if (!held) continue;
+        const unsigned char* part = (const unsigned char*)src_parts[s];
+        if (!part) { free(full); return ORACLE_ERR_ARG; }
+        if (kind_replicated(m, kind) && !first_replica) {
+            /* every TP rank of the owning stage holds the same logical state */
+            if (memcmp(full, part, (size_t)(rows * cols * ses)) != 0) {
+                free(full); return ORACLE_ERR_REPLICA_MISMATCH;
+            }
+            continue;
+        }
+        for (int64_t i = 0; i < nr; ++i)
+            for (int64_t j = 0; j < nc; ++j)
+                memcpy(full + ((r0 + i) * cols + (c0 + j)) * ses, part + (i * nc + j) * ses, (size_t)ses);
+        first_replica = 0;
+    }
+
+    /* 2. CAST */
+    unsigned char* cast = full;
+    if (des != ses) {
+        cast = (unsigned char*)malloc((size_t)(rows * cols * des));
+        if (!cast) { free(full); return ORACLE_ERR_NOMEM; }
+        for (int64_t e = 0; e < rows * cols; ++e) {
+            uint32_t u; uint16_t b;
+            memcpy(&u, full + e * 4, 4);
+            b = oracle_rne_bf16(u);
+            memcpy(cast + e * 2, &b, 2);
+        }
+    }
+
+    /* 3. SLICE */
+    for (int64_t d = 0; d < (int64_t)dp.tp * dp.pp; ++d) {
+        oracle_locate(m, dp, d, id, &held, &off, &r0, &nr, &c0, &nc);
+        if (!held) continue;
+        unsigned char* part = (unsigned char*)dst_parts[d];
+        if (!part) { if (cast != full) free(cast); free(full); return ORACLE_ERR_ARG; }
+        for (int64_t i = 0; i < nr; ++i)
+            for (int64_t j = 0; j < nc; ++j)
+                memcpy(part + (i * nc + j) * des, cast + ((r0 + i) * cols + (c0 + j)) * des, (size_t)des);
+    }
+    if (cast != full) free(cast);
+    free(full);
+    return ORACLE_OK;
+}
+
+/* Same, addressed by whole shard buffers (host memory). */
+int oracle_reshard_tensor(const oracle_model* m, oracle_plan sp, oracle_plan dp, int64_t id,
+                          const void* const* src_bufs, void* const* dst_bufs) {
+    int rc, held; int64_t off, r0, nr, c0, nc;
+    if ((rc = oracle_check_plan(m, sp))) return rc;
+    if ((rc = oracle_check_plan(m, dp))) return rc;
+    if (!src_bufs || !dst_bufs) return ORACLE_ERR_ARG;
+    int64_t ns = (int64_t)sp.tp * sp.pp, nd = (int64_t)dp.tp * dp.pp;
+    const void** sparts = (const void**)calloc((size_t)ns, sizeof(void*));
+    void** dparts = (void**)calloc((size_t)nd, sizeof(void*));
+    if (!sparts || !dparts) { free(sparts); free(dparts); return ORACLE_ERR_NOMEM; }
+    for (int64_t s = 0; s < ns; ++s) {
+        rc = oracle_locate(m, sp, s, id, &held, &off, &r0, &nr, &c0, &nc);
+        if (rc) break;
+        sparts[s] = held ? (const unsigned char*)src_bufs[s] + off : NULL;
+    }
+    for (int64_t d = 0; !rc && d < nd; ++d) {
+        rc = oracle_locate(m, dp, d, id, &held, &off, &r0, &nr, &c0, &nc);
+        if (rc) break;
+        dparts[d] = held ? (unsigned char*)dst_bufs[d] + off : NULL;
+    }
+    if (!rc) rc = oracle_reshard_tensor_parts(m, sp, dp, id, sparts, dparts);
+    free(sparts); free(dparts);
+    return rc;
+}
+
+/* The whole model-stage: every logical tensor in catalogue order. */
+int oracle_reshard(const oracle_model* m, oracle_plan sp, oracle_plan dp,
+                   const void* const* src_bufs, void* const* dst_bufs) {
+    int rc;
+    if ((rc = oracle_check_plan(m, sp))) return rc;
+    if ((rc = oracle_check_plan(m, dp))) return rc;
+    for (int64_t id = 0; id < oracle_num_logical(m); ++id)
+        if ((rc = oracle_reshard_tensor(m, sp, dp, id, src_bufs, dst_bufs))) return rc;
+    return ORACLE_OK;
+}

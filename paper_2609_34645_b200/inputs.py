@@ -1,0 +1,122 @@
+"""Seeded synthetic inputs and the workload table.  Serves the CUDA path's tests and benchmark and the
+oracle's tests alike, and therefore holds none of the reshard's arithmetic: no shard rule, no packing,
+no cast.  Whoever calls it brings the buffer sizes and the replica groups from its own side's layout
+query.
+
+Weights are drawn ~N(0, 0.02) from the stated seed, in fp32 and, for bf16 buffers, rounded by torch.  They
+stand in for the paper's trained checkpoints (Llama-3.1-8B, Qwen3-32B), which a reshard's cost and
+correctness do not depend on: it moves bits.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+
+import torch
+
+
+@dataclass(frozen=True)
+class Shape:
+    layers: int
+    hidden: int
+    heads: int
+    kv_heads: int
+    ffn: int
+    vocab: int
+
+
+TINY = Shape(2, 256, 4, 2, 688, 1024)              # head_dim 64
+LLAMA_8B = Shape(32, 4096, 32, 8, 14336, 128256)   # Llama-3-8B-shaped
+DENSE_32B = Shape(64, 5120, 40, 8, 27648, 152064)  # 32B-shaped decoder
+
+
+@dataclass(frozen=True)
+class Stage:
+    """One model-stage's transition: (tp, pp, dtype) -> (tp, pp, dtype); dtype is "bf16" or "fp32"."""
+    name: str
+    shape: Shape
+    seed: int
+    src: tuple
+    dst: tuple
+    value_head: bool = False
+
+
+@dataclass(frozen=True)
+class Workload:
+    name: str
+    stages: tuple
+    round_trip: bool = False   # run src->dst, then dst->src back, chained
+    note: str = ""
+
+
+WORKLOADS = {
+    # 1. tiny Merge, the case the oracle finishes at once
+    "tiny_tp2pp1_to_tp1pp1": Workload("tiny_tp2pp1_to_tp1pp1", (
+        Stage("tiny", TINY, 0, (2, 1, "bf16"), (1, 1, "bf16")),)),
+    # 2. 8B Split: the configuration the metric is quoted on
+    "8b_tp1pp1_to_tp4pp2": Workload("8b_tp1pp1_to_tp4pp2", (
+        Stage("8b", LLAMA_8B, 1, (1, 1, "bf16"), (4, 2, "bf16")),)),
+    # its reverse, the Merge direction of the headline
+    "8b_tp4pp2_to_tp1pp1": Workload("8b_tp4pp2_to_tp1pp1", (
+        Stage("8b", LLAMA_8B, 1, (4, 2, "bf16"), (1, 1, "bf16")),)),
+    # 3. fp32 master weights -> bf16 generation layout (train -> rollout weight sync)
+    "8b_fp32_tp2pp2_to_bf16_tp4pp1": Workload("8b_fp32_tp2pp2_to_bf16_tp4pp1", (
+        Stage("8b_master", LLAMA_8B, 2, (2, 2, "fp32"), (4, 1, "bf16")),)),
+    # 4. five PPO model-stages in one table; critic and reward carry a value head
+    "ppo5_8b": Workload("ppo5_8b", (
+        Stage("actor_generation", LLAMA_8B, 3, (4, 1, "bf16"), (2, 1, "bf16")),
+        Stage("actor_training", LLAMA_8B, 4, (2, 1, "bf16"), (4, 2, "bf16")),
+        Stage("critic", LLAMA_8B, 5, (2, 1, "bf16"), (4, 2, "bf16"), value_head=True),
+        Stage("reference", LLAMA_8B, 6, (4, 1, "bf16"), (2, 1, "bf16")),
+        Stage("reward", LLAMA_8B, 7, (4, 1, "bf16"), (2, 1, "bf16"), value_head=True),
+    ), note="generation/inference stages Merge TP4->TP2; training stages Split TP2->TP4, PP1->PP2"),
+    # 5. 32B round trip
+    "32b_tp2pp4_to_tp8pp1_and_back": Workload("32b_tp2pp4_to_tp8pp1_and_back", (
+        Stage("32b", DENSE_32B, 8, (2, 4, "bf16"), (8, 1, "bf16")),), round_trip=True),
+}
+
+# scaled-down stand-ins with the same structure, for parity tests the oracle finishes in seconds
+SMALL = Shape(4, 512, 8, 4, 1376, 2048)            # head_dim 64; several tiles and ragged tails
+MICRO = Shape(8, 64, 8, 8, 128, 128)               # head_dim 8; brute-force sized, TP up to 8, PP up to 8
+
+
+def element_size(dtype: str) -> int:
+    return {"bf16": 2, "fp32": 4}[dtype]
+
+
+def normal_bytes(nbytes: int, dtype: str, seed: int, device="cpu", std: float = 0.02,
+                 chunk_elems: int = 1 << 27) -> torch.Tensor:
+    """A uint8 buffer of ``nbytes`` whose contents are N(0, std) values of ``dtype`` from ``seed``."""
+    es = element_size(dtype)
+    assert nbytes % es == 0
+    n = nbytes // es
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    out = torch.empty(n, dtype=tdt, device=device)
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    for lo in range(0, n, chunk_elems):
+        hi = min(n, lo + chunk_elems)
+        tmp = torch.empty(hi - lo, dtype=torch.float32, device=device)
+        tmp.normal_(0.0, std, generator=g)
+        out[lo:hi] = tmp.to(tdt)
+        del tmp
+    return out.view(torch.uint8)
+
+
+def make_shards(sizes, dtype: str, seed: int, device="cpu") -> list:
+    """One buffer per shard; shard i draws from a stream derived from (seed, i)."""
+    return [normal_bytes(int(nb), dtype, seed * 1000003 + i, device) for i, nb in enumerate(sizes)]
+
+
+def tie_replicas(bufs, groups) -> None:
+    """Make replicated state identical: ``groups`` is a list of lists of (shard, byte offset, nbytes);
+    the first member's bytes are copied over the others."""
+    for grp in groups:
+        s0, o0, n0 = grp[0]
+        for s, o, n in grp[1:]:
+            assert n == n0
+            bufs[s][o:o + n] = bufs[s0][o0:o0 + n0]
+
+
+def sentinel_shards(sizes, device="cpu", value: int = 0xA5) -> list:
+    """Destination buffers pre-filled with a sentinel byte, so unwritten or over-written bytes show."""
+    return [torch.full((int(nb),), value, dtype=torch.uint8, device=device) for nb in sizes]

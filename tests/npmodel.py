@@ -1,0 +1,182 @@
+"""Test-side, third formulation of the layout contract, used only to pin the oracle.
+
+It is written differently from the oracle on purpose: logical tensors are numpy arrays, a TP shard is what
+``np.split`` along the parallel axis returns (the textbook definition of column- and row-parallel
+sharding), fused blocks are ``np.concatenate`` of the rank's pieces, and a shard buffer is those blocks laid
+end to end on 256-byte boundaries.  ``owner`` is the same contract once more as a per-element function.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+KINDS = ["ln1", "wq", "wk", "wv", "wo", "ln2", "wgate", "wup", "wdown"]
+
+
+def np_dtype(es):
+    return np.uint16 if es == 2 else np.uint32
+
+
+def logical_names(L):
+    names = ["embed"]
+    for l in range(L):
+        names += [f"{k}.{l}" for k in KINDS]
+    return names + ["ln_f", "head"]
+
+
+def logical_shapes(sh, value_head=False):
+    hd = sh.hidden // sh.heads
+    per = {"ln1": (1, sh.hidden), "ln2": (1, sh.hidden),
+           "wq": (sh.heads * hd, sh.hidden), "wk": (sh.kv_heads * hd, sh.hidden),
+           "wv": (sh.kv_heads * hd, sh.hidden), "wo": (sh.hidden, sh.heads * hd),
+           "wgate": (sh.ffn, sh.hidden), "wup": (sh.ffn, sh.hidden), "wdown": (sh.hidden, sh.ffn)}
+    out = {"embed": (sh.vocab, sh.hidden)}
+    for l in range(sh.layers):
+        for k in KINDS:
+            out[f"{k}.{l}"] = per[k]
+    out["ln_f"] = (1, sh.hidden)
+    out["head"] = (1, sh.hidden) if value_head else (sh.vocab, sh.hidden)
+    return out
+
+
+def random_logical(sh, es, seed, value_head=False):
+    rng = np.random.default_rng(seed)
+    dt = np_dtype(es)
+    return {n: rng.integers(0, np.iinfo(dt).max, size=s, dtype=dt, endpoint=True)
+            for n, s in logical_shapes(sh, value_head).items()}
+
+
+def position_coded(sh, es, salt, value_head=False):
+    """Element (tensor t, row i, col j) holds a hash of (t, i, j, salt), truncated to the element width."""
+    out = {}
+    for t, (n, (r, c)) in enumerate(logical_shapes(sh, value_head).items()):
+        i = np.arange(r, dtype=np.uint64)[:, None]
+        j = np.arange(c, dtype=np.uint64)[None, :]
+        with np.errstate(over="ignore"):
+          h = (np.uint64(t + 1) * np.uint64(0x9E3779B97F4A7C15) + i * np.uint64(0xC2B2AE3D27D4EB4F)
+               + j * np.uint64(0x165667B19E3779F9) + np.uint64(salt) * np.uint64(0x27D4EB2F165667C5))
+          h ^= h >> np.uint64(29)
+          h *= np.uint64(0xBF58476D1CE4E5B9)
+          h ^= h >> np.uint64(32)
+        out[n] = h.astype(np_dtype(es))
+    return out
+
+
+def _stored_blocks(sh, tp, pp, p, r, logical, value_head):
+    """The tensors shard (p, r) stores, in packing order, as numpy arrays (np.split formulation)."""
+    def d0(x):
+        return np.split(x, tp, axis=0)[r]
+
+    def d1(x):
+        return np.split(x, tp, axis=1)[r]
+
+    lps = sh.layers // pp
+    blocks = []
+    if p == 0:
+        blocks.append(d0(logical["embed"]))
+    for l in range(p * lps, (p + 1) * lps):
+        g = lambda k: logical[f"{k}.{l}"]
+        blocks.append(g("ln1"))
+        blocks.append(np.concatenate([d0(g("wq")), d0(g("wk")), d0(g("wv"))], axis=0))
+        blocks.append(d1(g("wo")))
+        blocks.append(g("ln2"))
+        blocks.append(np.concatenate([d0(g("wgate")), d0(g("wup"))], axis=0))
+        blocks.append(d1(g("wdown")))
+    if p == pp - 1:
+        blocks.append(logical["ln_f"])
+        blocks.append(logical["head"] if value_head else d0(logical["head"]))
+    return blocks
+
+
+def build_shards(sh, tp, pp, logical, value_head=False, pad=0xA5):
+    """Shard byte images (uint8 arrays), index = p * tp + r."""
+    out = []
+    for p in range(pp):
+        for r in range(tp):
+            chunks, cur = [], 0
+            for b in _stored_blocks(sh, tp, pp, p, r, logical, value_head):
+                start = -(-cur // 256) * 256
+                if start > cur:
+                    chunks.append(np.full(start - cur, pad, np.uint8))
+                raw = np.ascontiguousarray(b).view(np.uint8).reshape(-1)
+                chunks.append(raw)
+                cur = start + raw.size
+            end = -(-cur // 256) * 256
+            if end > cur:
+                chunks.append(np.full(end - cur, pad, np.uint8))
+            out.append(np.concatenate(chunks))
+    return out
+
+
+def owner(sh, tp, pp, es, name, i, j, value_head=False):
+    """Per-element statement of the contract: every (shard, byte offset) that holds element (i, j) of the
+    logical tensor ``name`` (several for replicated tensors)."""
+    hd = sh.hidden // sh.heads
+    H, F, V = sh.hidden, sh.ffn, sh.vocab
+    nq, nkv = sh.heads, sh.kv_heads
+    lps = sh.layers // pp
+    qr, kr, fr, vr = nq * hd // tp, nkv * hd // tp, F // tp, V // tp
+    up = lambda x: -(-x // 256) * 256
+    # byte sizes of the stored blocks of one layer, in order
+    layer_blocks = [("ln", H), ("qkv", (qr + 2 * kr) * H), ("wo", H * (nq * hd // tp)), ("ln", H),
+                    ("gu", 2 * fr * H), ("wdown", H * fr)]
+
+    def layer_base(p, l):
+        cur = 0
+        if p == 0:
+            cur = up(cur) + vr * H * es
+        for _ in range(p * lps, l):
+            for _, n in layer_blocks:
+                cur = up(cur) + n * es
+        return cur
+
+    def within_layer(idx):
+        # offset of the idx-th stored block of a layer relative to an (aligned) running cursor
+        def f(cur):
+            for k, (_, n) in enumerate(layer_blocks):
+                cur = up(cur)
+                if k == idx:
+                    return cur
+                cur += n * es
+        return f
+
+    if name == "embed":
+        r = i // vr
+        return [(0 * tp + r, up(0) + ((i % vr) * H + j) * es)]
+    if name in ("ln_f", "head"):
+        p = pp - 1
+        cur = layer_base(p, (p + 1) * lps)
+        lnf = up(cur)
+        head = up(lnf + H * es)
+        if name == "ln_f":
+            return [(p * tp + r, lnf + j * es) for r in range(tp)]
+        if value_head:
+            return [(p * tp + r, head + j * es) for r in range(tp)]
+        r = i // vr
+        return [(p * tp + r, head + ((i % vr) * H + j) * es)]
+    kind, l = name.split(".")
+    l = int(l)
+    p = l // lps
+    base = layer_base(p, l)
+    blk = {"ln1": 0, "wq": 1, "wk": 1, "wv": 1, "wo": 2, "ln2": 3, "wgate": 4, "wup": 4, "wdown": 5}[kind]
+    start = within_layer(blk)(base)
+    if kind in ("ln1", "ln2"):
+        return [(p * tp + r, start + j * es) for r in range(tp)]
+    if kind == "wq":
+        r = i // qr
+        return [(p * tp + r, start + ((i % qr) * H + j) * es)]
+    if kind in ("wk", "wv"):
+        r = i // kr
+        skip = qr + (kr if kind == "wv" else 0)
+        return [(p * tp + r, start + ((skip + i % kr) * H + j) * es)]
+    if kind in ("wgate", "wup"):
+        r = i // fr
+        skip = fr if kind == "wup" else 0
+        return [(p * tp + r, start + ((skip + i % fr) * H + j) * es)]
+    if kind == "wo":
+        w = nq * hd // tp
+        r = j // w
+        return [(p * tp + r, start + (i * w + j % w) * es)]
+    if kind == "wdown":
+        r = j // fr
+        return [(p * tp + r, start + (i * fr + j % fr) * es)]
+    raise KeyError(name)

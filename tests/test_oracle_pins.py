@@ -1,0 +1,372 @@
+"""Pins of the CPU oracle against things other than itself (no GPU).
+
+The paper prints no worked numeric example of a reshard; what it fixes is the semantic contract "Split and
+Merge change placement and sharding without changing logical state" (Section 6.2) and one layout example,
+(TP4, PP8) -> (TP4, PP2) units -> (TP8, PP2) (Section 6.1).  The pins are therefore: np.split /
+np.concatenate special cases, a brute-force per-element owner function, identity, round trips, checksum
+conservation, path independence through the paper's example, published parameter counts, and torch's
+fp32 -> bf16 conversion over every fp32 bit pattern.
+"""
+import itertools
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import npmodel
+from oracle import oracle as O
+from paper_2609_34645_b200 import inputs as I
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def model_of(sh, dtype=O.BF16, value_head=False):
+    return O.Model(sh.layers, sh.hidden, sh.heads, sh.kv_heads, sh.ffn, sh.vocab, dtype, value_head)
+
+
+def plans_for(sh, max_tp=8, max_pp=8):
+    out = []
+    for tp in (1, 2, 4, 8):
+        for pp in (1, 2, 4, 8):
+            if tp <= max_tp and pp <= max_pp and tp <= sh.kv_heads and sh.kv_heads % tp == 0 \
+                    and sh.ffn % tp == 0 and sh.vocab % tp == 0 and sh.layers % pp == 0:
+                out.append((tp, pp))
+    return out
+
+
+def payload_mask(model, plan):
+    """Boolean mask per shard: True on bytes that belong to a tensor, False on padding."""
+    masks = [np.zeros(O.shard_bytes(model, plan, s), bool) for s in range(O.num_shards(model, plan))]
+    e = O.es(model, plan)
+    for s in range(len(masks)):
+        for t in range(O.num_logical(model)):
+            p = O.locate(model, plan, s, t)
+            if p.held:
+                assert not masks[s][p.offset:p.offset + p.nr * p.nc * e].any(), "tensors overlap"
+                masks[s][p.offset:p.offset + p.nr * p.nc * e] = True
+    return masks
+
+
+# ---------------------------------------------------------------- closed forms (published sizes)
+
+@pytest.mark.parametrize("sh,vh,total", [
+    (I.LLAMA_8B, False, 8_030_261_248),    # Llama-3-8B's published parameter count
+    (I.LLAMA_8B, True, 7_504_928_768),     # LM head [128256, 4096] replaced by a [1, 4096] value head
+    (I.DENSE_32B, False, 32_763_417_600),
+    (I.TINY, False, 1_975_552),
+])
+def test_parameter_totals(sh, vh, total):
+    m = model_of(sh, value_head=vh)
+    assert O.num_logical(m) == 9 * sh.layers + 3
+    assert sum(r * c for r, c in (O.logical_shape(m, t) for t in range(O.num_logical(m)))) == total
+
+
+@pytest.mark.parametrize("sh,vh,total", [(I.LLAMA_8B, False, 8_030_261_248), (I.LLAMA_8B, True, 7_504_928_768),
+                                         (I.TINY, False, 1_975_552)])
+def test_shards_partition_the_model(sh, vh, total):
+    """Under every plan the shards' parts tile each logical tensor exactly once (replicated tensors once per
+    TP rank), and the parts fit in the shard without overlap."""
+    m = model_of(sh, value_head=vh)
+    for tp, pp in plans_for(sh, max_tp=4 if sh is I.LLAMA_8B else 8, max_pp=2 if sh is I.LLAMA_8B else 8):
+        pl = O.Plan(tp, pp)
+        n = O.num_shards(m, pl)
+        assert n == tp * pp
+        got = 0
+        for t in range(O.num_logical(m)):
+            rows, cols = O.logical_shape(m, t)
+            parts = [O.locate(m, pl, s, t) for s in range(n)]
+            held = [p for p in parts if p.held]
+            area = sum(p.nr * p.nc for p in held)
+            assert area in (rows * cols, tp * rows * cols)
+            if area == tp * rows * cols and tp > 1:
+                assert rows == 1          # only norms / value head are replicated
+            got += rows * cols
+            for s, p in enumerate(parts):
+                if p.held:
+                    assert p.offset % 256 == 0 or t != 0
+                    assert p.offset + p.nr * p.nc * 2 <= O.shard_bytes(m, pl, s)
+        assert got == total
+
+
+def test_shard_sizes_8b_split():
+    """8B bf16 TP4PP2: eight shards of about 2.008 GB, the two stages equal in size (embed vs head + ln_f)."""
+    m = model_of(I.LLAMA_8B)
+    sizes = [O.shard_bytes(m, O.Plan(4, 2), s) for s in range(8)]
+    per_layer = (25_165_824 + 16_777_216 + 117_440_512 + 58_720_256) // 4 + 2 * 4096
+    assert sizes[0] == (525_336_576 // 4 + 16 * per_layer) * 2
+    assert sizes[4] == sizes[0] + 4096 * 2
+    assert O.shard_bytes(m, O.Plan(1, 1), 0) == 8_030_261_248 * 2
+
+
+# ---------------------------------------------------------------- np.split special cases
+
+@pytest.mark.parametrize("sh", [I.TINY, I.MICRO])
+@pytest.mark.parametrize("es", [2, 4])
+@pytest.mark.parametrize("vh", [False, True])
+def test_against_np_split(sh, es, vh):
+    """TP1PP1 <-> any plan agrees with shards built by np.split / np.concatenate from numpy logical tensors
+    (sentinel padding must survive: padding is never written)."""
+    m = model_of(sh, O.BF16 if es == 2 else O.FP32, vh)
+    logical = npmodel.random_logical(sh, es, seed=11, value_head=vh)
+    full = npmodel.build_shards(sh, 1, 1, logical, vh)
+    assert full[0].size == O.shard_bytes(m, O.Plan(1, 1), 0)
+    for tp, pp in plans_for(sh):
+        want = npmodel.build_shards(sh, tp, pp, logical, vh)
+        got = O.reshard(m, O.Plan(1, 1), O.Plan(tp, pp), full, fill=0xA5)
+        assert len(got) == len(want)
+        for g, w in zip(got, want):
+            assert g.size == w.size and np.array_equal(g, w), (tp, pp)
+        back = O.reshard(m, O.Plan(tp, pp), O.Plan(1, 1), want, fill=0xA5)
+        assert np.array_equal(back[0], full[0]), (tp, pp)
+
+
+def test_any_plan_pair_against_np_split():
+    sh, es = I.MICRO, 2
+    m = model_of(sh)
+    logical = npmodel.random_logical(sh, es, seed=5)
+    images = {pl: npmodel.build_shards(sh, pl[0], pl[1], logical) for pl in plans_for(sh)}
+    for a, b in itertools.product(images, images):
+        got = O.reshard(m, O.Plan(*a), O.Plan(*b), images[a], fill=0xA5)
+        for g, w in zip(got, images[b]):
+            assert np.array_equal(g, w), (a, b)
+
+
+# ---------------------------------------------------------------- brute-force owner function
+
+@pytest.mark.parametrize("es", [2, 4])
+@pytest.mark.parametrize("vh", [False, True])
+def test_owner_brute_force(es, vh):
+    """Position-coded payload: every element of every logical tensor is looked up, one by one, through the
+    per-element owner function in the shards the oracle produced."""
+    sh = I.Shape(2, 32, 4, 2, 48, 64)
+    m = model_of(sh, O.BF16 if es == 2 else O.FP32, vh)
+    dt = npmodel.np_dtype(es)
+    for salt in (1, 2, 3):
+        logical = npmodel.position_coded(sh, es, salt, vh)
+        src = npmodel.build_shards(sh, 1, 1, logical, vh)
+        for tp, pp in [(2, 1), (1, 2), (2, 2)]:
+            dst = O.reshard(m, O.Plan(1, 1), O.Plan(tp, pp), src)
+            seen = [np.zeros(d.size, np.uint8) for d in dst]
+            for name, x in logical.items():
+                for i in range(x.shape[0]):
+                    for j in range(x.shape[1]):
+                        for shard, off in npmodel.owner(sh, tp, pp, es, name, i, j, vh):
+                            assert dst[shard][off:off + es].view(dt)[0] == x[i, j], (name, i, j, tp, pp)
+                            seen[shard][off:off + es] += 1
+            for s, mask in enumerate(payload_mask(m, O.Plan(tp, pp))):
+                assert np.array_equal(seen[s] == 1, mask)       # each payload byte owned exactly once
+
+
+def test_owner_vectorised_tiny_merge():
+    """The tiny Merge workload (TP2PP1 -> TP1PP1) checked through the owner function on sampled elements."""
+    sh, es = I.TINY, 2
+    m = model_of(sh)
+    logical = npmodel.position_coded(sh, es, 7)
+    src = npmodel.build_shards(sh, 2, 1, logical)
+    dst = O.reshard(m, O.Plan(2, 1), O.Plan(1, 1), src)
+    rng = np.random.default_rng(0)
+    for name, x in logical.items():
+        for _ in range(40):
+            i, j = int(rng.integers(x.shape[0])), int(rng.integers(x.shape[1]))
+            (shard, off), = npmodel.owner(sh, 1, 1, es, name, i, j)
+            assert dst[shard][off:off + 2].view(np.uint16)[0] == x[i, j]
+        for i, j in [(0, 0), (x.shape[0] - 1, x.shape[1] - 1)]:
+            (shard, off), = npmodel.owner(sh, 1, 1, es, name, i, j)
+            assert dst[shard][off:off + 2].view(np.uint16)[0] == x[i, j]
+
+
+# ---------------------------------------------------------------- invariants
+
+def _random_src(m, plan, seed, dtype):
+    sizes = [O.shard_bytes(m, plan, s) for s in range(O.num_shards(m, plan))]
+    bufs = I.make_shards(sizes, dtype, seed)
+    groups = []
+    for t in range(O.num_logical(m)):
+        rows, cols = O.logical_shape(m, t)
+        held = [(s, O.locate(m, plan, s, t)) for s in range(len(sizes))]
+        held = [(s, p) for s, p in held if p.held]
+        if len(held) > 1 and all(p.nr * p.nc == rows * cols for _, p in held):
+            groups.append([(s, p.offset, p.nr * p.nc * O.es(m, plan)) for s, p in held])
+    I.tie_replicas(bufs, groups)
+    return [b.numpy() for b in bufs]
+
+
+def test_identity():
+    for sh in (I.TINY, I.MICRO):
+        m = model_of(sh)
+        src = _random_src(m, O.Plan(1, 1), 0, "bf16")
+        dst = O.reshard(m, O.Plan(1, 1), O.Plan(1, 1), src, fill=0xA5)
+        mask = payload_mask(m, O.Plan(1, 1))[0]
+        assert np.array_equal(dst[0][mask], src[0][mask])
+        assert (dst[0][~mask] == 0xA5).all()
+
+
+@pytest.mark.parametrize("sh", [I.TINY, I.SMALL])
+def test_round_trip_all_plan_pairs(sh):
+    m = model_of(sh)
+    pls = plans_for(sh)
+    for a in pls:
+        src = _random_src(m, O.Plan(*a), 3, "bf16")
+        masks = payload_mask(m, O.Plan(*a))
+        for b in pls:
+            mid = O.reshard(m, O.Plan(*a), O.Plan(*b), src)
+            back = O.reshard(m, O.Plan(*b), O.Plan(*a), mid)
+            for s, k, mk in zip(src, back, masks):
+                assert np.array_equal(s[mk], k[mk]), (a, b)
+
+
+def _checksums(m, plan, bufs):
+    """Per logical tensor: (sum, xor) of element bit patterns over the shards' parts; replicated tensors
+    divided by the replica count."""
+    e = O.es(m, plan)
+    dt = npmodel.np_dtype(e)
+    out = []
+    for t in range(O.num_logical(m)):
+        rows, cols = O.logical_shape(m, t)
+        tot, x, area = 0, 0, 0
+        for s in range(len(bufs)):
+            p = O.locate(m, plan, s, t)
+            if p.held:
+                v = bufs[s][p.offset:p.offset + p.nr * p.nc * e].view(dt).astype(np.uint64)
+                tot += int(v.sum(dtype=np.uint64))
+                x ^= int(np.bitwise_xor.reduce(v)) if (area // (rows * cols)) == 0 else 0
+                area += p.nr * p.nc
+        reps = area // (rows * cols)
+        out.append(((tot // reps) % 2 ** 64, x))
+    return out
+
+
+def test_checksums_conserved():
+    sh = I.TINY
+    m = model_of(sh)
+    src = _random_src(m, O.Plan(2, 1), 0, "bf16")       # the tiny Merge workload, seed 0
+    ref = _checksums(m, O.Plan(2, 1), src)
+    for b in plans_for(sh):
+        dst = O.reshard(m, O.Plan(2, 1), O.Plan(*b), src)
+        assert _checksums(m, O.Plan(*b), dst) == ref, b
+
+
+def test_path_independence_paper_example():
+    """(TP4, PP8) -> (TP8, PP2) directly equals the route through T_sub = (TP4, PP2), the paper's example of
+    Section 6.1, and the route through the logical tensor (TP1, PP1)."""
+    sh = I.MICRO
+    m = model_of(sh)
+    a, t_sub, c = O.Plan(4, 8), O.Plan(4, 2), O.Plan(8, 2)
+    src = _random_src(m, a, 9, "bf16")
+    direct = O.reshard(m, a, c, src)
+    via_sub = O.reshard(m, t_sub, c, O.reshard(m, a, t_sub, src))
+    via_one = O.reshard(m, O.Plan(1, 1), c, O.reshard(m, a, O.Plan(1, 1), src))
+    for d, v, w in zip(direct, via_sub, via_one):
+        assert np.array_equal(d, v) and np.array_equal(d, w)
+
+
+def test_emu_example_tp1pp4_to_tp2pp4():
+    """The EMU example of Section 5.1: an actor going from (TP1, PP4) to (TP2, PP4); checked against np.split."""
+    sh = I.MICRO
+    m = model_of(sh)
+    logical = npmodel.random_logical(sh, 2, seed=21)
+    got = O.reshard(m, O.Plan(1, 4), O.Plan(2, 4), npmodel.build_shards(sh, 1, 4, logical), fill=0xA5)
+    for g, w in zip(got, npmodel.build_shards(sh, 2, 4, logical)):
+        assert np.array_equal(g, w)
+
+
+# ---------------------------------------------------------------- the cast
+
+def _golden_cases():
+    with open(os.path.join(GOLDEN, "rne_bf16_cases.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                a, b = line.split()[:2]
+                yield int(a, 16), int(b, 16)
+
+
+def test_cast_hand_cases():
+    for u, want in _golden_cases():
+        assert O.rne_bf16(u) == want, hex(u)
+
+
+def test_cast_exact_nearest_on_samples():
+    """Second formulation in exact integer arithmetic: the bf16 neighbours of a finite fp32 value are
+    hi<<16 and (hi+1)<<16 read as sign-magnitude integers; choose the nearer, ties to the even hi."""
+    rng = np.random.default_rng(1)
+    us = np.concatenate([rng.integers(0, 2 ** 32, 20000, dtype=np.uint64),
+                         np.arange(0x3F800000 - 70000, 0x3F800000 + 70000, 997, dtype=np.uint64)])
+    for u in map(int, us):
+        mag = u & 0x7FFFFFFF
+        if mag > 0x7F800000:
+            assert O.rne_bf16(u) == 0x7FC0
+            continue
+        lo = mag >> 16
+        rem = mag - (lo << 16)
+        if rem * 2 > 0x10000 or (rem * 2 == 0x10000 and lo & 1):
+            lo += 1
+        assert O.rne_bf16(u) == ((u >> 31) << 15 | lo), hex(u)
+
+
+def test_cast_matches_torch_exhaustively():
+    """Every one of the 2^32 fp32 bit patterns: equal to torch's fp32 -> bf16 conversion wherever the input is
+    not NaN; every NaN gives 0x7FC0."""
+    step = 1 << 24
+    ramp = np.arange(step, dtype=np.uint32)
+    for lo in range(0, 1 << 32, step):
+        bits = ramp + np.uint32(lo)
+        got = O.rne_bf16_array(bits)
+        ref = torch.from_numpy(bits.view(np.float32)).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+        nan = (bits & 0x7FFFFFFF) > 0x7F800000
+        assert np.array_equal(got[~nan], ref[~nan]), hex(lo)
+        assert (got[nan] == 0x7FC0).all()
+
+
+def test_cast_commutes_with_reshard():
+    sh = I.TINY
+    m32, m16 = model_of(sh, O.FP32), model_of(sh, O.BF16)
+    a, b = O.Plan(2, 2), O.Plan(1, 1)
+    src = _random_src(m32, a, 2, "fp32")
+    fused = O.reshard(m32, a, O.Plan(b.tp, b.pp, O.BF16), src)
+    # reshard in fp32, then cast the (TP1, PP1) image tensor by tensor with torch
+    mid = O.reshard(m32, a, b, src)[0]
+    want = np.zeros_like(fused[0])
+    for t in range(O.num_logical(m32)):
+        p32, p16 = O.locate(m32, b, 0, t), O.locate(m16, b, 0, t)
+        n = p32.nr * p32.nc
+        x = torch.from_numpy(mid[p32.offset:p32.offset + 4 * n].view(np.float32).copy())
+        want[p16.offset:p16.offset + 2 * n] = x.to(torch.bfloat16).view(torch.int16).numpy().view(np.uint8)
+    assert np.array_equal(fused[0], want)
+    # cast first (shard by shard), then reshard in bf16
+    a16 = []
+    for s, buf in enumerate(src):
+        out = np.zeros(O.shard_bytes(m16, a, s), np.uint8)
+        for t in range(O.num_logical(m32)):
+            p32, p16 = O.locate(m32, a, s, t), O.locate(m16, a, s, t)
+            if p32.held:
+                n = p32.nr * p32.nc
+                out[p16.offset:p16.offset + 2 * n] = O.rne_bf16_array(
+                    buf[p32.offset:p32.offset + 4 * n].view(np.uint32)).view(np.uint8)
+        a16.append(out)
+    assert np.array_equal(O.reshard(m16, a, b, a16)[0], fused[0])
+
+
+# ---------------------------------------------------------------- refusals
+
+def test_refusals():
+    m = model_of(I.TINY)
+    assert O.check_plan(m, O.Plan(4, 1)) == O.ERR_UNSUPPORTED       # tp > kv_heads
+    assert O.check_plan(m, O.Plan(1, 4)) == O.ERR_INDIVISIBLE       # 2 layers over 4 stages
+    assert O.check_plan(model_of(I.Shape(2, 256, 4, 2, 689, 1024)), O.Plan(2, 1)) == O.ERR_INDIVISIBLE
+    assert O.check_plan(m, O.Plan(0, 1)) == O.ERR_ARG
+    src = _random_src(model_of(I.TINY, O.BF16), O.Plan(1, 1), 0, "bf16")
+    with pytest.raises(O.OracleError) as e:                           # bf16 -> fp32 is not a transition
+        O.reshard(m, O.Plan(1, 1), O.Plan(1, 1, O.FP32), src, O.new_shards(model_of(I.TINY, O.FP32), O.Plan(1, 1)))
+    assert e.value.code == O.ERR_UNSUPPORTED
+
+
+def test_replica_mismatch_is_detected():
+    m = model_of(I.TINY)
+    src = _random_src(m, O.Plan(2, 1), 0, "bf16")
+    p = O.locate(m, O.Plan(2, 1), 1, 1)        # ln1 of layer 0 on TP rank 1
+    src[1][p.offset] ^= 1
+    with pytest.raises(O.OracleError) as e:
+        O.reshard(m, O.Plan(2, 1), O.Plan(1, 1), src)
+    assert e.value.code == O.ERR_REPLICA_MISMATCH

@@ -1,0 +1,438 @@
+#!/usr/bin/env python
+"""Benchmark of the EMU reshard: GB/s (bytes read + written) and ms per model-stage transition.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+A step is one pass of the whole hot path (table walk: claim, copy / cast, finish) over one workload, by
+default the 8B Split TP1PP1 -> TP4PP2 the metric is quoted on.  Inputs are seeded synthetic N(0, 0.02)
+weights, resident in HBM before the timed region; the working set (>= 32 GB) is far larger than L2, so no
+flush is needed between iterations.  With N > 1 (torchrun) every rank runs an independent replica of the
+workload on its own GPU (the path has no exchange step: replicas only), and the value is the sum over
+ranks divided by the slowest rank's time.
+
+`--impl reference` times the CPU oracle (the only "reference implementation" there is: the paper ships no
+code) on a bounded sample of the same workload, on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "reshard_throughput"
+UNIT = "GB/s"
+DEFAULT_WORKLOAD = "8b_tp1pp1_to_tp4pp2"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--cpu-layers", type=int, default=6, help="layers in the CPU-oracle sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--tile-bytes", type=int, default=0)
+    ap.add_argument("--ctas-per-sm", type=int, default=0)
+    ap.add_argument("--threads", type=int, default=0)
+    ap.add_argument("--variant", type=int, default=0)
+    return ap.parse_args()
+
+
+# ------------------------------------------------------------------------------------------------ peaks
+
+def measured_hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ------------------------------------------------------------------------------------------------ clocks
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_id: str):
+        self.gpu_id = gpu_id
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(prefix="nereus_clocks_", suffix=".csv")
+            os.close(fd)
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu_id}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()          # the exact process this object started
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.close()
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        with open(self.path) as f:
+            for line in f:
+                p = [x.strip() for x in line.split(",")]
+                if len(p) < 8:
+                    continue
+                try:
+                    sm.append(float(p[0])); mx.append(float(p[1])); power.append(float(p[2]))
+                except ValueError:
+                    continue
+                for name, v in zip(names, p[4:8]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+        try:
+            os.unlink(self.path)
+        except OSError:
+            pass
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm), "power_w_max": max(power)}
+
+
+# ------------------------------------------------------------------------------------------------ workload
+
+def build_workload(name, device, tune):
+    """Compiles the workload's transition(s) and allocates seeded sources and sentinel destinations."""
+    from paper_2609_34645_b200 import binding as B
+    from paper_2609_34645_b200 import inputs as I
+
+    wl = I.WORKLOADS[name]
+    parts, descs, srcs, dsts, keep = [], [], [], [], []
+    for st in wl.stages:
+        sh = st.shape
+        d = B.ModelDesc(sh.layers, sh.hidden, sh.heads, sh.kv_heads, sh.ffn, sh.vocab, B.DTYPES[st.src[2]],
+                        st.value_head)
+        pa, pb = B.Plan(st.src[0], st.src[1], B.DTYPES[st.src[2]]), B.Plan(st.dst[0], st.dst[1], B.DTYPES[st.dst[2]])
+        t = d.compile(pa, pb)
+        s = I.make_shards(d.shard_sizes(pa), st.src[2], st.seed, device)
+        es = I.element_size(st.src[2])
+        groups = []
+        for tid in range(d.num_tensors()):
+            g = []
+            for k in range(d.num_shards(pa)):
+                off, rows, cols, rep = d.tensor_slice(pa, k, tid)
+                if rep and rows:
+                    g.append((k, off, rows * cols * es))
+            if len(g) > 1:
+                groups.append(g)
+        I.tie_replicas(s, groups)
+        srcs += s
+        dsts += I.sentinel_shards(d.shard_sizes(pb), device)
+        parts.append(t)
+        descs.append((d, pa, pb))
+        keep.append(d)
+    if wl.round_trip:
+        assert len(parts) == 1
+        d, pa, pb = descs[0]
+        back = d.compile(pb, pa)
+        parts.append(back)
+        t = B.Transition.fuse(parts, chained=True)
+        dsts = dsts + srcs                      # the way back lands in the original source buffers
+    elif len(parts) > 1:
+        t = B.Transition.fuse(parts, chained=False)
+    else:
+        t = parts[0]
+    if any(tune.values()):
+        t.tune(**tune)
+    t.prepare()
+    return wl, t, srcs, dsts, (parts, keep, descs)
+
+
+# ------------------------------------------------------------------------------------------------ CPU oracle leg
+
+def oracle_sample(workload_name, layers, device_srcs=None):
+    """Times the oracle, as it stands, on the tensors of the first `layers` layers of the workload's first
+    stage (gather -> cast -> slice per logical tensor).  Returns (GB/s on algorithmic bytes, seconds, desc)."""
+    import numpy as np
+    import torch
+    from oracle import oracle as O
+    from paper_2609_34645_b200 import inputs as I
+
+    st = I.WORKLOADS[workload_name].stages[0]
+    sh = st.shape
+    odt = {"bf16": O.BF16, "fp32": O.FP32}
+    m = O.Model(sh.layers, sh.hidden, sh.heads, sh.kv_heads, sh.ffn, sh.vocab, odt[st.src[2]], st.value_head)
+    pa, pb = O.Plan(st.src[0], st.src[1]), O.Plan(st.dst[0], st.dst[1], odt[st.dst[2]])
+    layers = max(1, min(layers, sh.layers))
+    ses, des = I.element_size(st.src[2]), I.element_size(st.dst[2])
+    total_s, total_bytes = 0.0, 0
+    for tid in range(1, 1 + 9 * layers):
+        src_parts, dst_parts = [], []
+        for s in range(O.num_shards(m, pa)):
+            p = O.locate(m, pa, s, tid)
+            if not p.held:
+                src_parts.append(None)
+                continue
+            n = p.nr * p.nc * ses
+            if device_srcs is not None:
+                src_parts.append(device_srcs[s][p.offset:p.offset + n].cpu().numpy())
+            else:
+                src_parts.append(I.normal_bytes(n, st.src[2], st.seed * 7919 + tid).numpy())
+        # replicated tensors must agree across ranks
+        held = [x for x in src_parts if x is not None]
+        rows, cols = O.logical_shape(m, tid)
+        if len(held) > 1 and held[0].size == rows * cols * ses:
+            for x in held[1:]:
+                x[:] = held[0]
+        for d in range(O.num_shards(m, pb)):
+            p = O.locate(m, pb, d, tid)
+            dst_parts.append(np.empty(p.nr * p.nc * des, np.uint8) if p.held else None)
+            if p.held:
+                total_bytes += p.nr * p.nc * (ses + des)
+        t0 = time.perf_counter()
+        O.reshard_tensor_parts(m, pa, pb, tid, src_parts, dst_parts)
+        total_s += time.perf_counter() - t0
+    what = f"oracle on the {9 * layers} logical tensors of layers 0..{layers - 1} of stage '{st.name}' " \
+           f"({total_bytes / 1e9:.2f} GB read+written of the workload)"
+    return total_bytes / total_s / 1e9, total_s, what
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle on a bounded sample, timed on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import oracle as O
+    O.build()
+    vals, secs, what = [], [], ""
+    for k in range(args.warmup + args.steps):
+        v, s, what = oracle_sample(args.workload, 1)
+        if k >= args.warmup:
+            vals.append(v); secs.append(s)
+    value = sum(vals) / len(vals)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sum(secs) / len(secs),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic", "config": {"workload": args.workload, "sample": what},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": what},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------ ours
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device; the reshard has no CPU fallback"
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+
+    from paper_2609_34645_b200 import binding as B
+
+    tune = dict(tile_bytes=args.tile_bytes, ctas_per_sm=args.ctas_per_sm, threads=args.threads,
+                variant=args.variant)
+    wl, t, srcs, dsts, keep = build_workload(args.workload, device, tune)
+    rd, wr = t.bytes()
+    stream = torch.cuda.current_stream()
+    sp = B.Transition.pointer_array([b.data_ptr() for b in srcs])
+    dp = B.Transition.pointer_array([b.data_ptr() for b in dsts])
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        t.run(sp, dp, stream.cuda_stream)
+    torch.cuda.synchronize()
+    assert t.status() == B.DEV_OK
+
+    props = torch.cuda.get_device_properties(device)
+    gpu_id = f"GPU-{props.uuid}" if hasattr(props, "uuid") else str(local)
+    sampler = ClockSampler(gpu_id)
+    if rank == 0:
+        sampler.start()
+    launches0 = t.launches()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    barrier()
+    for a, b in ev:
+        a.record(stream)
+        t.run(sp, dp, stream.cuda_stream)
+        b.record(stream)
+    barrier()
+    per_step = [a.elapsed_time(b) for a, b in ev]                   # ms, one launch each
+    total_ms = ev[0][0].elapsed_time(ev[-1][1])
+    launches = t.launches() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    assert t.status() == B.DEV_OK
+
+    tm = torch.tensor([total_ms], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+    total_ms_max = float(tm.item())
+    ms_per_step = total_ms_max / args.steps
+    value = world * (rd + wr) / 1e9 / (ms_per_step / 1e3)
+
+    # end to end: host buffers in, host buffers out, copies inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(args, t, srcs, dsts, sp, dp, stream, rd + wr, world, device)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_hbm_peak()
+    kernel_ms = statistics.mean(per_step)
+    achieved = (rd + wr) / 1e9 / (kernel_ms / 1e3)
+    n_trans = len(wl.stages) * (2 if wl.round_trip else 1)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None,
+        "dtype": "bf16" if all(s.src[2] == "bf16" for s in wl.stages) else "fp32->bf16",
+        "data": "synthetic",
+        "config": {"workload": wl.name, "transitions_per_step": n_trans,
+                   "ms_per_transition": ms_per_step / n_trans,
+                   "bytes_read": rd, "bytes_written": wr, "l2": "inputs larger than L2, no flush",
+                   "multi_gpu": "replicas only", "tiles": t.num_tiles()[0], "levels": t.num_tiles()[1]},
+        "frac_of_nominal_8TBps": achieved / NOMINAL_HBM_GBS,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": None, "peak_kind": f"of {peak_kind}", "kernel": "nereus_walk",
+                     "kernel_ms": kernel_ms, "kernel_ms_min": min(per_step)},
+        "clocks": clocks, "gpu_launches": launches,
+    }
+    if e2e is not None:
+        line["e2e"] = e2e
+    if not args.no_cpu_baseline and world == 1:
+        try:
+            from oracle import oracle as O
+            O.build()
+            v, s, what = oracle_sample(args.workload, args.cpu_layers, srcs)
+            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": what,
+                                    "seconds": s}
+        except Exception as e:      # the baseline is a report, never a dependency of the GPU number
+            line["cpu_baseline"] = {"value": None, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                    "sample": f"failed: {e!r}"}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def host_memory_budget() -> int:
+    """Bytes of host memory this process may safely take: MemAvailable, capped by the cgroup limit."""
+    avail = 0
+    try:
+        with open("/proc/meminfo") as f:
+            for line in f:
+                if line.startswith("MemAvailable:"):
+                    avail = int(line.split()[1]) * 1024
+    except OSError:
+        pass
+    for path, cur in (("/sys/fs/cgroup/memory.max", "/sys/fs/cgroup/memory.current"),
+                      ("/sys/fs/cgroup/memory/memory.limit_in_bytes", "/sys/fs/cgroup/memory/memory.usage_in_bytes")):
+        try:
+            lim = open(path).read().strip()
+            if lim != "max":
+                used = int(open(cur).read().strip())
+                avail = min(avail, max(0, int(lim) - used)) if avail else max(0, int(lim) - used)
+        except (OSError, ValueError):
+            pass
+    return avail
+
+
+def run_e2e(args, t, srcs, dsts, sp, dp, stream, algo_bytes, world, device):
+    """Same metric through the C ABI with HOST buffers: every step copies the source shards from pinned host
+    memory to the device, runs the transition, and reads the destination shards back to pinned host memory."""
+    import torch
+    import torch.distributed as dist
+
+    need = sum(b.numel() for b in srcs) + sum(b.numel() for b in dsts)
+    budget = host_memory_budget()
+    if need > 0.5 * budget:
+        return {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
+                "note": f"skipped: {need / 1e9:.1f} GB of pinned host memory needed, {budget / 1e9:.1f} GB available"}
+    uniq_dst = list(dsts)
+    try:
+        h_src = [torch.empty(b.numel(), dtype=torch.uint8, pin_memory=True) for b in srcs]
+        h_dst = [torch.empty(b.numel(), dtype=torch.uint8, pin_memory=True) for b in uniq_dst]
+    except Exception as e:
+        return {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
+                "note": f"pinned host allocation failed: {e!r}"}
+    for h, b in zip(h_src, srcs):
+        h.copy_(b)
+    h2d = sum(b.numel() for b in srcs)
+    d2h = sum(b.numel() for b in uniq_dst)
+    steps = max(1, args.e2e_steps)
+
+    def step():
+        for h, b in zip(h_src, srcs):
+            b.copy_(h, non_blocking=True)
+        t.run(sp, dp, stream.cuda_stream)
+        for h, b in zip(h_dst, uniq_dst):
+            h.copy_(b, non_blocking=True)
+
+    step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    a.record(stream)
+    for _ in range(steps):
+        step()
+    b.record(stream)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    ms = torch.tensor([a.elapsed_time(b) / steps], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+    ms = float(ms.item())
+    return {"value": world * algo_bytes / 1e9 / (ms / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": d2h, "ms_per_step": ms, "steps": steps}
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,187 @@
+/*
+ * nereus.h -- C ABI of the B200-native EMU reshard.
+ *
+ * One model-stage's parameter shards theta = {theta_i}, i = 1..tp*pp (the EMU of Section 5 of the Nereus
+ * paper) are carried from a source (TP, PP) layout to a target (TP, PP) layout on ONE GPU, every virtual
+ * TP/PP rank's shard being a separate device buffer.  This is the local layout change that the paper's Split
+ * and Merge primitives perform next to their collectives (Section 6.2, "DAG Execution and Safety" and
+ * "Resharding--transport interplay"); it changes placement and sharding and never the logical state
+ * (Section 6.2, "Preserving training semantics").  An optional fp32 -> bf16 round-to-nearest-even cast is
+ * fused into the move for the training -> generation weight sync between the actor's two model-stages
+ * (Section 5, EMU definition).
+ *
+ * The paper fixes none of the tensor-level layout; this header does (see "Layout contract").
+ *
+ * Conventions
+ *   - Every function returns an int: NEREUS_OK (0) or a negative NEREUS_ERR_* code.  Nothing throws, aborts
+ *     or prints.  Output arguments are written only on success.
+ *   - "host" / "device" next to a pointer says where the pointed-to memory lives.
+ *   - The library never allocates, frees or keeps shard memory; the caller owns every shard buffer.  A
+ *     handle owns only its task table (host copy, plus one device copy per nereus_transition_prepare).
+ *   - Handles are not thread-safe; use one handle from one thread at a time.
+ *
+ * Layout contract
+ *   model    L layers, hidden H, nq query heads, nkv KV heads (nkv | nq), head_dim hd = H / nq, FFN F,
+ *            vocabulary V, Llama-style: untied embedding, RMSNorm weights only, no biases.
+ *   logical tensors, row-major [out, in]:
+ *            embed [V,H]; per layer ln1 [H], wq [nq*hd,H], wk [nkv*hd,H], wv [nkv*hd,H], wo [H,nq*hd],
+ *            ln2 [H], wgate [F,H], wup [F,H], wdown [H,F]; ln_f [H]; head [V,H] (or a value head [1,H]).
+ *   plan     (tp, pp, dtype).  Pipeline stage p owns layers [p*L/pp, (p+1)*L/pp); embed lives on stage 0,
+ *            ln_f and the head on stage pp-1.  Shard index = p*tp + r (TP rank r fastest).
+ *   TP rank r of t stores
+ *            embed, LM head   rows [r*V/t, (r+1)*V/t)                        (vocabulary-parallel)
+ *            qkv              one fused block [Q_r ; K_r ; V_r]: the rows of q heads [r*nq/t, (r+1)*nq/t),
+ *                             then of kv heads [r*nkv/t, (r+1)*nkv/t) of wk, then the same of wv (so a
+ *                             rank's q heads are exactly the GQA groups of its kv heads)
+ *            wo               columns [r*nq*hd/t, (r+1)*nq*hd/t), stored contiguously as [H, nq*hd/t]
+ *            gate_up          one fused block [G_r ; U_r], each F/t rows
+ *            wdown            columns [r*F/t, (r+1)*F/t), stored as [H, F/t]
+ *            ln1, ln2, ln_f, value head   the whole tensor on every TP rank of the owning stage
+ *   shard buffer packing: [embed], then per local layer ln1, qkv, wo, ln2, gate_up, wdown, then
+ *            [ln_f, head]; every stored tensor starts on a 256-byte boundary; the buffer length is the end
+ *            of the last tensor rounded up to 256 bytes.  Padding bytes are never read and never written.
+ *   stored tensor ids (argument tensor_id below): 0 = embed; 1 + 6*l + k for layer l and
+ *            k = 0 ln1, 1 qkv, 2 wo, 3 ln2, 4 gate_up, 5 wdown; 1 + 6*L = ln_f; 2 + 6*L = head.
+ *   required: tp | nkv, tp | F, tp | V, pp | L, tp <= nkv (no KV-head replication), and every contiguous piece
+ *            a transition moves must start on and span a multiple of 16 bytes on both sides (for the cast: 8
+ *            elements).
+ */
+#ifndef NEREUS_H_
+#define NEREUS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define NEREUS_OK                 0
+#define NEREUS_ERR_ARG           -1   /* null pointer, negative or zero size, index out of range          */
+#define NEREUS_ERR_INDIVISIBLE   -2   /* a divisibility or 16-byte rule of the layout contract fails       */
+#define NEREUS_ERR_UNSUPPORTED   -3   /* dtype pair other than same->same or fp32->bf16; tp > kv_heads;    */
+                                      /* more buffers than one launch can address                          */
+#define NEREUS_ERR_ALIAS         -4   /* a destination buffer overlaps a source or another destination     */
+#define NEREUS_ERR_CUDA          -5   /* a CUDA call failed; see nereus_last_cuda_error                    */
+#define NEREUS_ERR_NOMEM         -6   /* host allocation failed                                            */
+#define NEREUS_ERR_MISMATCH      -7   /* parts of a chained fuse do not connect (buffer count or sizes)    */
+#define NEREUS_ERR_ALIGN         -8   /* a shard pointer is not 16-byte aligned                            */
+
+/* device status word (nereus_transition_status) */
+#define NEREUS_DEV_OK             0
+#define NEREUS_DEV_BOUNDS         1   /* a claimed tile did not resolve to a task: corrupted table         */
+#define NEREUS_DEV_TIMEOUT        2   /* a dependency wait gave up after its poll limit                    */
+
+typedef enum { NEREUS_BF16 = 1, NEREUS_FP32 = 2 } nereus_dtype_t;
+
+typedef struct nereus_model_desc_s* nereus_model_desc_t;   /* opaque, host */
+typedef struct nereus_transition_s* nereus_transition_t;   /* opaque, host; owns the task table */
+
+/* A (TP, PP) layout.  dtype 0 means "the descriptor's dtype". */
+typedef struct { int tp; int pp; int dtype; } nereus_plan_t;
+
+/* One rect-copy task of a compiled transition, for inspection and tests.  Buffer indices address the
+ * concatenation [src_ptrs..., dst_ptrs...] that nereus_transition_run receives ("unified index").
+ * The task copies `rows` pieces; piece i is `width_bytes_dst` bytes at dst_off + i*dst_pitch and comes
+ * from `width_bytes_src` bytes at src_off + i*src_pitch (twice as many when cast = 1). */
+typedef struct {
+    int32_t  src_buf, dst_buf;      /* unified buffer indices */
+    int32_t  level;                 /* dependency level: tasks of level k run after all of level k-1 */
+    int32_t  cast;                  /* 1: fp32 -> bf16 RNE, 0: bit copy */
+    uint64_t src_off, dst_off;      /* bytes from the start of the buffer */
+    uint64_t src_pitch, dst_pitch;  /* bytes between consecutive pieces */
+    uint64_t rows;
+    uint64_t width_bytes_src, width_bytes_dst;
+} nereus_rect_t;
+
+/* ---- model descriptor (EMU field M and the shapes of theta; Section 5) -------------------------------- */
+
+/* Describes a Llama-style decoder.  dtype is the element type of plans whose dtype field is 0.
+ * Errors: ARG (non-positive size, bad dtype, null out), INDIVISIBLE (heads does not divide hidden, or
+ * kv_heads does not divide heads). */
+int nereus_model_desc(int layers, int hidden, int heads, int kv_heads, int ffn, int vocab, int dtype,
+                      nereus_model_desc_t* out);
+/* Replaces the LM head [V,H] by a value head [out_dim,H], out_dim = 1 (critic / reward model-stages).
+ * The value head is replicated over TP.  Errors: ARG, UNSUPPORTED (out_dim != 1). */
+int nereus_model_desc_set_value_head(nereus_model_desc_t desc, int out_dim);
+int nereus_model_desc_destroy(nereus_model_desc_t desc);
+
+/* ---- layout queries (theta_i, i = p*tp + r; Section 5) ------------------------------------------------ */
+
+/* Checks the layout contract's divisibility rules for one plan.  Errors: ARG, INDIVISIBLE, UNSUPPORTED. */
+int nereus_plan_check(nereus_model_desc_t desc, nereus_plan_t plan);
+int nereus_plan_num_shards(nereus_model_desc_t desc, nereus_plan_t plan, int* n);            /* tp*pp */
+int nereus_plan_shard_bytes(nereus_model_desc_t desc, nereus_plan_t plan, int shard, size_t* bytes);
+/* Number of stored tensor ids, 6*L + 3. */
+int nereus_model_num_tensors(nereus_model_desc_t desc, int* n);
+/* Where `shard` keeps stored tensor `tensor_id`: byte offset, and the stored block's rows x cols in
+ * elements (row-major, cols contiguous).  rows = cols = 0 when the shard's stage does not own the tensor.
+ * replicated = 1 for tensors that every TP rank of the stage holds whole. */
+int nereus_plan_tensor_slice(nereus_model_desc_t desc, nereus_plan_t plan, int shard, int tensor_id,
+                             size_t* offset, size_t* rows, size_t* cols, int* replicated);
+
+/* ---- transition compiler (the change Delta_M = (E_M -> E*_M) of Section 6.1, at tensor granularity) ---- */
+
+/* Compiles src -> dst for one model-stage into rect-copy tasks by intersecting every destination slice
+ * with the source slices directly (no intermediate layout).  Host work only.
+ * Errors: ARG, INDIVISIBLE, UNSUPPORTED (dtype pair; tp > kv_heads), NOMEM. */
+int nereus_transition_compile(nereus_model_desc_t desc, nereus_plan_t src, nereus_plan_t dst,
+                              nereus_transition_t* out);
+/* Fuses n compiled transitions into one task table that one launch executes (Section 6.2: ready primitives
+ * run concurrently; a primitive is ready only after its predecessors complete).
+ *   chained = 0: the parts are independent model-stages.  run() takes the concatenation of the parts'
+ *                source arrays and the concatenation of their destination arrays.  One level.
+ *   chained = 1: part k+1 reads what part k wrote: its source buffers ARE part k's destination buffers
+ *                (same count and sizes, else MISMATCH).  run() takes part 0's sources and the concatenation
+ *                of all parts' destinations; part k is dependency level k.
+ * The parts stay valid and independent of the fused handle.  Errors: ARG, MISMATCH, UNSUPPORTED, NOMEM. */
+int nereus_transition_fuse(const nereus_transition_t* parts, int n, int chained, nereus_transition_t* out);
+int nereus_transition_destroy(nereus_transition_t t);
+
+/* Number of source / destination buffers run() expects, and the minimum length of each. */
+int nereus_transition_num_buffers(nereus_transition_t t, int* n_src, int* n_dst);
+int nereus_transition_buffer_bytes(nereus_transition_t t, int is_dst, int index, size_t* bytes);
+/* Algorithmic bytes one run reads and writes (sum over tasks; replicated tensors once per replica). */
+int nereus_transition_bytes(nereus_transition_t t, size_t* read, size_t* written);
+/* The task table, in execution order (level, then largest first). */
+int nereus_transition_num_rects(nereus_transition_t t, int* n);
+int nereus_transition_get_rect(nereus_transition_t t, int index, nereus_rect_t* out);
+/* Tiles one run claims, and dependency levels. */
+int nereus_transition_num_tiles(nereus_transition_t t, uint64_t* tiles, int* levels);
+
+/* Launch tuning; 0 keeps the default of a field.  tile_bytes: target bytes per claimed tile (multiple of
+ * 512).  ctas_per_sm, threads: persistent grid = SMs * ctas_per_sm blocks of `threads` threads.
+ * variant: 0 default, 1 register-staged vector copy, 2 bulk-copy shared-memory ring.
+ * Drops the device copy of the table (the next prepare/run uploads it again).  Errors: ARG. */
+int nereus_transition_tune(nereus_transition_t t, int tile_bytes, int ctas_per_sm, int threads, int variant);
+
+/* ---- execution (the local layout change of Section 6.2) ---------------------------------------------- */
+
+/* Uploads the task table to the current device (cudaMalloc + synchronous copy).  Optional: run() does it
+ * on first use.  Call it ahead of time to keep allocation out of a timed or captured region. */
+int nereus_transition_prepare(nereus_transition_t t);
+/* Enqueues the whole transition on `cuda_stream` (a cudaStream_t; NULL = the default stream) as one
+ * persistent kernel and returns without synchronising.
+ *   src_ptrs (host array of device pointers): source shard i = p*tp + r; read-only during the run.
+ *   dst_ptrs (host array of device pointers): destination shards; every byte of every stored tensor is
+ *            written exactly once, padding is untouched.
+ * Both arrays are copied before the call returns.  Every pointer must be 16-byte aligned and address at
+ * least nereus_transition_buffer_bytes bytes.  Sources stay live until the stream reaches the end of the
+ * run (Section 6.2: source buffers live until their readers complete).
+ * Errors: ARG (null), ALIGN, ALIAS, CUDA.  Runs of the same handle must not overlap on the device. */
+int nereus_transition_run(nereus_transition_t t, const void* const* src_ptrs, void* const* dst_ptrs,
+                          void* cuda_stream);
+/* Reads the device status word of the last run (NEREUS_DEV_*).  The caller must have synchronised the
+ * stream first; this call copies 4 bytes from the device synchronously. */
+int nereus_transition_status(nereus_transition_t t, int* device_status);
+/* Kernels this handle has launched since it was created (one per run). */
+int nereus_transition_launches(nereus_transition_t t, uint64_t* n);
+
+const char* nereus_strerror(int code);
+/* cudaError_t of the last failed CUDA call made by this library on the calling thread (0 if none). */
+int nereus_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NEREUS_H_ */

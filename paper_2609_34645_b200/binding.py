@@ -1,0 +1,252 @@
+"""Thin ctypes binding of ``libnereus.so`` (the C ABI of ``include/nereus.h``), same names, argument
+marshalling only: every step of the reshard runs inside the CUDA library.  Importing this module loads the
+library and raises if it has not been built (``python -m paper_2609_34645_b200.build``); there is no CPU
+fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libnereus.so")
+
+BF16 = 1
+FP32 = 2
+DTYPES = {"bf16": BF16, "fp32": FP32}
+
+OK = 0
+ERR_ARG, ERR_INDIVISIBLE, ERR_UNSUPPORTED, ERR_ALIAS = -1, -2, -3, -4
+ERR_CUDA, ERR_NOMEM, ERR_MISMATCH, ERR_ALIGN = -5, -6, -7, -8
+DEV_OK, DEV_BOUNDS, DEV_TIMEOUT = 0, 1, 2
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_34645_b200.build` "
+                      "(nvcc, sm_100a).  The reshard has no CPU fallback.")
+_lib = ctypes.CDLL(LIB_PATH)
+
+
+class NereusError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        msg = _lib.nereus_strerror(code).decode()
+        if code == ERR_CUDA:
+            msg += f" (cudaError {_lib.nereus_last_cuda_error()})"
+        super().__init__(f"{what}: {msg} [{code}]")
+        self.code = code
+
+
+class Plan(ctypes.Structure):
+    """nereus_plan_t: (tp, pp, dtype); dtype 0 = the descriptor's."""
+    _fields_ = [("tp", ctypes.c_int), ("pp", ctypes.c_int), ("dtype", ctypes.c_int)]
+
+    def __init__(self, tp: int, pp: int, dtype: int = 0):
+        super().__init__(tp, pp, dtype)
+
+    def __repr__(self):
+        return f"Plan(tp={self.tp}, pp={self.pp}, dtype={self.dtype})"
+
+
+class Rect(ctypes.Structure):
+    """nereus_rect_t."""
+    _fields_ = [("src_buf", ctypes.c_int32), ("dst_buf", ctypes.c_int32), ("level", ctypes.c_int32),
+                ("cast", ctypes.c_int32), ("src_off", ctypes.c_uint64), ("dst_off", ctypes.c_uint64),
+                ("src_pitch", ctypes.c_uint64), ("dst_pitch", ctypes.c_uint64), ("rows", ctypes.c_uint64),
+                ("width_bytes_src", ctypes.c_uint64), ("width_bytes_dst", ctypes.c_uint64)]
+
+
+_vp, _i, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+_P = ctypes.POINTER
+_SIGS = {
+    "nereus_model_desc": [_i, _i, _i, _i, _i, _i, _i, _P(_vp)],
+    "nereus_model_desc_set_value_head": [_vp, _i],
+    "nereus_model_desc_destroy": [_vp],
+    "nereus_plan_check": [_vp, Plan],
+    "nereus_plan_num_shards": [_vp, Plan, _P(_i)],
+    "nereus_plan_shard_bytes": [_vp, Plan, _i, _P(_sz)],
+    "nereus_model_num_tensors": [_vp, _P(_i)],
+    "nereus_plan_tensor_slice": [_vp, Plan, _i, _i, _P(_sz), _P(_sz), _P(_sz), _P(_i)],
+    "nereus_transition_compile": [_vp, Plan, Plan, _P(_vp)],
+    "nereus_transition_fuse": [_P(_vp), _i, _i, _P(_vp)],
+    "nereus_transition_destroy": [_vp],
+    "nereus_transition_num_buffers": [_vp, _P(_i), _P(_i)],
+    "nereus_transition_buffer_bytes": [_vp, _i, _i, _P(_sz)],
+    "nereus_transition_bytes": [_vp, _P(_sz), _P(_sz)],
+    "nereus_transition_num_rects": [_vp, _P(_i)],
+    "nereus_transition_get_rect": [_vp, _i, _P(Rect)],
+    "nereus_transition_num_tiles": [_vp, _P(ctypes.c_uint64), _P(_i)],
+    "nereus_transition_tune": [_vp, _i, _i, _i, _i],
+    "nereus_transition_prepare": [_vp],
+    "nereus_transition_run": [_vp, _P(_vp), _P(_vp), _vp],
+    "nereus_transition_status": [_vp, _P(_i)],
+    "nereus_transition_launches": [_vp, _P(ctypes.c_uint64)],
+    "nereus_last_cuda_error": [],
+}
+for _name, _args in _SIGS.items():
+    _f = getattr(_lib, _name)          # AttributeError here = the library does not export a declared symbol
+    _f.argtypes = _args
+    _f.restype = _i
+_lib.nereus_strerror.argtypes = [_i]
+_lib.nereus_strerror.restype = ctypes.c_char_p
+EXPORTS = sorted(list(_SIGS) + ["nereus_strerror"])
+
+
+def _ck(rc: int, what: str) -> None:
+    if rc != OK:
+        raise NereusError(rc, what)
+
+
+class ModelDesc:
+    """nereus_model_desc(layers, hidden, heads, kv_heads, ffn, vocab, dtype)."""
+
+    def __init__(self, layers, hidden, heads, kv_heads, ffn, vocab, dtype=BF16, value_head=False):
+        self._h = _vp()
+        _ck(_lib.nereus_model_desc(layers, hidden, heads, kv_heads, ffn, vocab, dtype, ctypes.byref(self._h)),
+            "nereus_model_desc")
+        if value_head:
+            self.set_value_head(1)
+
+    def set_value_head(self, out_dim=1):
+        _ck(_lib.nereus_model_desc_set_value_head(self._h, out_dim), "nereus_model_desc_set_value_head")
+
+    def plan_check(self, plan: Plan) -> int:
+        return _lib.nereus_plan_check(self._h, plan)
+
+    def num_shards(self, plan: Plan) -> int:
+        n = _i()
+        _ck(_lib.nereus_plan_num_shards(self._h, plan, ctypes.byref(n)), "nereus_plan_num_shards")
+        return n.value
+
+    def shard_bytes(self, plan: Plan, shard: int) -> int:
+        n = _sz()
+        _ck(_lib.nereus_plan_shard_bytes(self._h, plan, shard, ctypes.byref(n)), "nereus_plan_shard_bytes")
+        return n.value
+
+    def shard_sizes(self, plan: Plan) -> list:
+        return [self.shard_bytes(plan, s) for s in range(self.num_shards(plan))]
+
+    def num_tensors(self) -> int:
+        n = _i()
+        _ck(_lib.nereus_model_num_tensors(self._h, ctypes.byref(n)), "nereus_model_num_tensors")
+        return n.value
+
+    def tensor_slice(self, plan: Plan, shard: int, tensor_id: int):
+        """(offset, rows, cols, replicated) of a stored tensor in a shard; rows = cols = 0 if not held."""
+        off, r, c, rep = _sz(), _sz(), _sz(), _i()
+        _ck(_lib.nereus_plan_tensor_slice(self._h, plan, shard, tensor_id, ctypes.byref(off), ctypes.byref(r),
+                                          ctypes.byref(c), ctypes.byref(rep)), "nereus_plan_tensor_slice")
+        return off.value, r.value, c.value, bool(rep.value)
+
+    def compile(self, src: Plan, dst: Plan) -> "Transition":
+        h = _vp()
+        _ck(_lib.nereus_transition_compile(self._h, src, dst, ctypes.byref(h)), "nereus_transition_compile")
+        return Transition(h)
+
+    def close(self):
+        if self._h:
+            _lib.nereus_model_desc_destroy(self._h)
+            self._h = _vp()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class Transition:
+    """A compiled transition handle (nereus_transition_t)."""
+
+    def __init__(self, handle):
+        self._h = handle
+
+    @staticmethod
+    def fuse(parts, chained=False) -> "Transition":
+        arr = (_vp * len(parts))(*[p._h for p in parts])
+        h = _vp()
+        _ck(_lib.nereus_transition_fuse(arr, len(parts), int(chained), ctypes.byref(h)), "nereus_transition_fuse")
+        return Transition(h)
+
+    def num_buffers(self):
+        a, b = _i(), _i()
+        _ck(_lib.nereus_transition_num_buffers(self._h, ctypes.byref(a), ctypes.byref(b)),
+            "nereus_transition_num_buffers")
+        return a.value, b.value
+
+    def buffer_bytes(self, is_dst: bool, index: int) -> int:
+        n = _sz()
+        _ck(_lib.nereus_transition_buffer_bytes(self._h, int(is_dst), index, ctypes.byref(n)),
+            "nereus_transition_buffer_bytes")
+        return n.value
+
+    def bytes(self):
+        r, w = _sz(), _sz()
+        _ck(_lib.nereus_transition_bytes(self._h, ctypes.byref(r), ctypes.byref(w)), "nereus_transition_bytes")
+        return r.value, w.value
+
+    def rects(self) -> list:
+        n = _i()
+        _ck(_lib.nereus_transition_num_rects(self._h, ctypes.byref(n)), "nereus_transition_num_rects")
+        out = []
+        for k in range(n.value):
+            r = Rect()
+            _ck(_lib.nereus_transition_get_rect(self._h, k, ctypes.byref(r)), "nereus_transition_get_rect")
+            out.append(r)
+        return out
+
+    def num_tiles(self):
+        t, l = ctypes.c_uint64(), _i()
+        _ck(_lib.nereus_transition_num_tiles(self._h, ctypes.byref(t), ctypes.byref(l)), "nereus_transition_num_tiles")
+        return t.value, l.value
+
+    def tune(self, tile_bytes=0, ctas_per_sm=0, threads=0, variant=0):
+        _ck(_lib.nereus_transition_tune(self._h, tile_bytes, ctas_per_sm, threads, variant), "nereus_transition_tune")
+
+    def prepare(self):
+        _ck(_lib.nereus_transition_prepare(self._h), "nereus_transition_prepare")
+
+    @staticmethod
+    def pointer_array(ptrs):
+        return (_vp * len(ptrs))(*ptrs)
+
+    def run(self, src_ptrs, dst_ptrs, stream=0):
+        """src_ptrs / dst_ptrs: sequences of device addresses (ints) or ready ctypes arrays; stream: a
+        cudaStream_t as an int (e.g. torch.cuda.current_stream().cuda_stream)."""
+        if not isinstance(src_ptrs, ctypes.Array):
+            src_ptrs = self.pointer_array(src_ptrs)
+        if not isinstance(dst_ptrs, ctypes.Array):
+            dst_ptrs = self.pointer_array(dst_ptrs)
+        _ck(_lib.nereus_transition_run(self._h, src_ptrs, dst_ptrs, _vp(stream)), "nereus_transition_run")
+
+    def run_raw(self, src_ptrs, dst_ptrs, stream=0) -> int:
+        """Like run() but returns the error code instead of raising."""
+        if not isinstance(src_ptrs, ctypes.Array):
+            src_ptrs = self.pointer_array(src_ptrs)
+        if not isinstance(dst_ptrs, ctypes.Array):
+            dst_ptrs = self.pointer_array(dst_ptrs)
+        return _lib.nereus_transition_run(self._h, src_ptrs, dst_ptrs, _vp(stream))
+
+    def status(self) -> int:
+        s = _i()
+        _ck(_lib.nereus_transition_status(self._h, ctypes.byref(s)), "nereus_transition_status")
+        return s.value
+
+    def launches(self) -> int:
+        n = ctypes.c_uint64()
+        _ck(_lib.nereus_transition_launches(self._h, ctypes.byref(n)), "nereus_transition_launches")
+        return n.value
+
+    def close(self):
+        if self._h:
+            _lib.nereus_transition_destroy(self._h)
+            self._h = _vp()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def strerror(code: int) -> str:
+    return _lib.nereus_strerror(code).decode()

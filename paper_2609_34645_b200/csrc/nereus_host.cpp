@@ -1,0 +1,474 @@
+// Host side of the EMU reshard: model descriptor, shard layout, and the transition compiler that turns a
+// plan difference (source plan -> target plan, the change Delta_M of Section 6.1 of the Nereus paper at
+// tensor granularity) into rect-copy tasks.  The map is direct: every destination slice is intersected with
+// the source slices that overlap it; no full logical tensor and no intermediate layout is ever formed.
+#include <algorithm>
+#include <cstring>
+#include <new>
+
+#include "nereus_internal.hpp"
+
+using namespace nereus;
+
+namespace nereus {
+
+// ---------------------------------------------------------------------------------------------------
+// catalogue
+// ---------------------------------------------------------------------------------------------------
+
+static StoredTensor whole(int64_t rows, int64_t cols, int layer) {
+    return StoredTensor{Cut::Whole, 1, {rows, 0, 0}, cols, layer};
+}
+static StoredTensor by_rows(int nseg, int64_t r0, int64_t r1, int64_t r2, int64_t cols, int layer) {
+    return StoredTensor{Cut::Rows, nseg, {r0, r1, r2}, cols, layer};
+}
+static StoredTensor by_cols(int64_t rows, int64_t cols, int layer) {
+    return StoredTensor{Cut::Cols, 1, {rows, 0, 0}, cols, layer};
+}
+
+void build_catalogue(nereus_model_desc_s& d) {
+    const int64_t hd = d.H / d.nq;
+    d.catalogue.clear();
+    d.catalogue.reserve(6 * d.L + 3);
+    d.catalogue.push_back(by_rows(1, d.V, 0, 0, d.H, -1));                                   // embed
+    for (int l = 0; l < d.L; ++l) {
+        d.catalogue.push_back(whole(1, d.H, l));                                             // ln1
+        d.catalogue.push_back(by_rows(3, d.nq * hd, d.nkv * hd, d.nkv * hd, d.H, l));        // q;k;v
+        d.catalogue.push_back(by_cols(d.H, d.nq * hd, l));                                   // wo
+        d.catalogue.push_back(whole(1, d.H, l));                                             // ln2
+        d.catalogue.push_back(by_rows(2, d.F, d.F, 0, d.H, l));                              // gate;up
+        d.catalogue.push_back(by_cols(d.H, d.F, l));                                         // wdown
+    }
+    d.catalogue.push_back(whole(1, d.H, -2));                                                // ln_f
+    d.catalogue.push_back(d.value_head ? whole(1, d.H, -2) : by_rows(1, d.V, 0, 0, d.H, -2)); // head
+}
+
+int check_plan(const nereus_model_desc_s& d, nereus_plan_t p) {
+    if (p.tp < 1 || p.pp < 1) return NEREUS_ERR_ARG;
+    if (p.dtype != 0 && p.dtype != NEREUS_BF16 && p.dtype != NEREUS_FP32) return NEREUS_ERR_ARG;
+    if (p.tp > d.nkv) return NEREUS_ERR_UNSUPPORTED;
+    if (d.nkv % p.tp || d.nq % p.tp || d.F % p.tp || d.V % p.tp || d.L % p.pp) return NEREUS_ERR_INDIVISIBLE;
+    return NEREUS_OK;
+}
+
+int owning_stage(const nereus_model_desc_s& d, int id, int pp) {
+    const int layer = d.catalogue[id].layer;
+    if (layer == -1) return 0;
+    if (layer == -2) return pp - 1;
+    return layer / (int)(d.L / pp);
+}
+
+void stored_block(const StoredTensor& t, int tp, int64_t& rows, int64_t& cols) {
+    switch (t.cut) {
+    case Cut::Whole: rows = t.seg_rows[0]; cols = t.cols; break;
+    case Cut::Cols:  rows = t.seg_rows[0]; cols = t.cols / tp; break;
+    case Cut::Rows:
+        rows = 0;
+        for (int s = 0; s < t.nseg; ++s) rows += t.seg_rows[s] / tp;
+        cols = t.cols;
+        break;
+    }
+}
+
+void stage_layout(const nereus_model_desc_s& d, nereus_plan_t p, int stage, StageLayout& out) {
+    const uint64_t es = elem_size(plan_dtype(d, p));
+    const int n = (int)d.catalogue.size();
+    out.offset.assign(n, kNotHeld);
+    uint64_t cur = 0;
+    for (int id = 0; id < n; ++id) {          // the catalogue order is the packing order
+        if (owning_stage(d, id, p.pp) != stage) continue;
+        int64_t rows, cols;
+        stored_block(d.catalogue[id], p.tp, rows, cols);
+        cur = round_up(cur, 256);
+        out.offset[id] = cur;
+        cur += (uint64_t)rows * (uint64_t)cols * es;
+    }
+    out.bytes = round_up(cur, 256);
+}
+
+// ---------------------------------------------------------------------------------------------------
+// compiler
+// ---------------------------------------------------------------------------------------------------
+
+namespace {
+
+struct Emitter {
+    std::vector<Rect>& out;
+    bool               misaligned = false;
+
+    void emit(Rect r) {
+        const uint64_t ws = r.width_dst << r.cast;
+        if (r.rows == 0 || r.width_dst == 0) return;
+        // a rect whose pieces touch on both sides is one contiguous run
+        if (r.rows > 1 && r.src_pitch == ws && r.dst_pitch == r.width_dst) {
+            r.width_dst *= r.rows;
+            r.rows = 1;
+        }
+        if (r.rows == 1) { r.src_pitch = r.width_dst << r.cast; r.dst_pitch = r.width_dst; }
+        if ((r.src_off | r.dst_off | r.width_dst | (r.rows > 1 ? (r.src_pitch | r.dst_pitch) : 0)) & 15)
+            misaligned = true;
+        // extend the previous run when this one continues it on both sides
+        if (!out.empty()) {
+            Rect& p = out.back();
+            if (p.rows == 1 && r.rows == 1 && p.src_buf == r.src_buf && p.dst_buf == r.dst_buf &&
+                p.cast == r.cast && p.level == r.level &&
+                p.src_off + (p.width_dst << p.cast) == r.src_off && p.dst_off + p.width_dst == r.dst_off) {
+                p.width_dst += r.width_dst;
+                p.src_pitch = p.width_dst << p.cast;
+                p.dst_pitch = p.width_dst;
+                return;
+            }
+        }
+        out.push_back(r);
+    }
+};
+
+}  // namespace
+
+static int compile_one(const nereus_model_desc_s& d, nereus_plan_t sp, nereus_plan_t dp, nereus_transition_s& t) {
+    const int      sdt = plan_dtype(d, sp), ddt = plan_dtype(d, dp);
+    const uint64_t ses = elem_size(sdt), des = elem_size(ddt);
+    const int      cast = (sdt != ddt) ? 1 : 0;
+    const int      n_src = sp.tp * sp.pp, n_dst = dp.tp * dp.pp;
+    if (n_src + n_dst > kMaxBuffers) return NEREUS_ERR_UNSUPPORTED;
+
+    std::vector<StageLayout> sl(sp.pp), dl(dp.pp);
+    for (int p = 0; p < sp.pp; ++p) stage_layout(d, sp, p, sl[p]);
+    for (int p = 0; p < dp.pp; ++p) stage_layout(d, dp, p, dl[p]);
+    t.src_bytes.resize(n_src);
+    t.dst_bytes.resize(n_dst);
+    for (int i = 0; i < n_src; ++i) t.src_bytes[i] = sl[i / sp.tp].bytes;
+    for (int i = 0; i < n_dst; ++i) t.dst_bytes[i] = dl[i / dp.tp].bytes;
+    t.dst_level.assign(n_dst, 0);
+    t.dst_read_level.assign(n_dst, -1);
+    t.n_levels = 1;
+
+    Emitter em{t.rects};
+    const int ts = sp.tp, td = dp.tp;
+    for (int pd = 0; pd < dp.pp; ++pd) {
+        for (int rd = 0; rd < td; ++rd) {
+            const int dst_buf = n_src + pd * td + rd;
+            for (int id = 0; id < (int)d.catalogue.size(); ++id) {
+                const uint64_t doff = dl[pd].offset[id];
+                if (doff == kNotHeld) continue;
+                const StoredTensor& x = d.catalogue[id];
+                const int      ps   = owning_stage(d, id, sp.pp);
+                const uint64_t soff = sl[ps].offset[id];
+                Rect r{};
+                r.dst_buf = dst_buf; r.level = 0; r.cast = cast;
+                if (x.cut == Cut::Whole) {
+                    // replicated state: every copy is the same logical state; read TP rank 0's
+                    r.src_buf = ps * ts;
+                    r.src_off = soff; r.dst_off = doff;
+                    r.rows = 1; r.width_dst = (uint64_t)x.seg_rows[0] * x.cols * des;
+                    em.emit(r);
+                } else if (x.cut == Cut::Rows) {
+                    // each stacked segment is cut by rows on both sides: intersect row intervals
+                    uint64_t sbase = 0, dbase = 0;       // rows of earlier segments inside the stored block
+                    for (int s = 0; s < x.nseg; ++s) {
+                        const int64_t N = x.seg_rows[s], ns = N / ts, nd = N / td;
+                        const int64_t d0 = rd * nd, d1 = d0 + nd;
+                        for (int rs = 0; rs < ts; ++rs) {
+                            const int64_t s0 = rs * ns, s1 = s0 + ns;
+                            const int64_t lo = std::max(d0, s0), hi = std::min(d1, s1);
+                            if (lo >= hi) continue;
+                            r.src_buf = ps * ts + rs;
+                            r.src_off = soff + (sbase + (uint64_t)(lo - s0)) * x.cols * ses;
+                            r.dst_off = doff + (dbase + (uint64_t)(lo - d0)) * x.cols * des;
+                            r.rows = 1; r.width_dst = (uint64_t)(hi - lo) * x.cols * des;
+                            em.emit(r);
+                        }
+                        sbase += ns; dbase += nd;
+                    }
+                } else {
+                    // every row is cut into column pieces on both sides: intersect column intervals
+                    const int64_t K = x.cols, ks = K / ts, kd = K / td;
+                    const int64_t d0 = rd * kd, d1 = d0 + kd;
+                    for (int rs = 0; rs < ts; ++rs) {
+                        const int64_t s0 = rs * ks, s1 = s0 + ks;
+                        const int64_t lo = std::max(d0, s0), hi = std::min(d1, s1);
+                        if (lo >= hi) continue;
+                        r.src_buf = ps * ts + rs;
+                        r.src_off = soff + (uint64_t)(lo - s0) * ses;
+                        r.dst_off = doff + (uint64_t)(lo - d0) * des;
+                        r.src_pitch = (uint64_t)ks * ses; r.dst_pitch = (uint64_t)kd * des;
+                        r.rows = (uint64_t)x.seg_rows[0]; r.width_dst = (uint64_t)(hi - lo) * des;
+                        em.emit(r);
+                    }
+                }
+            }
+        }
+    }
+    if (em.misaligned) return NEREUS_ERR_INDIVISIBLE;
+    return NEREUS_OK;
+}
+
+static void finish(nereus_transition_s& t) {
+    // execution order: by level, then largest first (stable, so equal tasks keep destination order)
+    std::stable_sort(t.rects.begin(), t.rects.end(), [](const Rect& a, const Rect& b) {
+        if (a.level != b.level) return a.level < b.level;
+        return a.rows * a.width_dst > b.rows * b.width_dst;
+    });
+    t.bytes_read = t.bytes_written = 0;
+    for (const Rect& r : t.rects) {
+        t.bytes_written += r.rows * r.width_dst;
+        t.bytes_read += r.rows * (r.width_dst << r.cast);
+    }
+}
+
+uint64_t tile_table(const nereus_transition_s& t, uint32_t tile_bytes, std::vector<RectDev>& out,
+                    std::vector<uint32_t>& first, uint32_t level_end[kMaxLevels]) {
+    out.clear(); first.clear();
+    out.reserve(t.rects.size()); first.reserve(t.rects.size() + 1);
+    for (int k = 0; k < kMaxLevels; ++k) level_end[k] = 0;
+    uint64_t total = 0;
+    for (const Rect& r : t.rects) {
+        RectDev q{};
+        q.src_off = r.src_off; q.dst_off = r.dst_off; q.width = r.width_dst;
+        q.src_pitch = (uint32_t)r.src_pitch; q.dst_pitch = (uint32_t)r.dst_pitch;
+        q.rows = (uint32_t)r.rows;
+        q.src_buf = (uint16_t)r.src_buf; q.dst_buf = (uint16_t)r.dst_buf;
+        q.level = (uint16_t)r.level; q.cast = (uint16_t)r.cast;
+        uint64_t ntiles;
+        if (r.rows == 1 || r.width_dst >= tile_bytes) {
+            q.rows_per_tile = 1;
+            q.tile_w = tile_bytes;
+            const uint64_t ct = (r.width_dst + tile_bytes - 1) / tile_bytes;
+            q.col_tiles = (uint32_t)ct;
+            ntiles = ct * r.rows;
+        } else {
+            q.rows_per_tile = (uint32_t)std::max<uint64_t>(1, tile_bytes / r.width_dst);
+            q.tile_w = (uint32_t)r.width_dst;
+            q.col_tiles = 1;
+            ntiles = (r.rows + q.rows_per_tile - 1) / q.rows_per_tile;
+        }
+        if (total + ntiles > 0xFFFFFFF0ull) return 0;
+        q.first_tile = (uint32_t)total;
+        first.push_back((uint32_t)total);
+        total += ntiles;
+        level_end[r.level] = (uint32_t)total;
+        out.push_back(q);
+    }
+    first.push_back((uint32_t)total);
+    for (int k = 1; k < kMaxLevels; ++k) level_end[k] = std::max(level_end[k], level_end[k - 1]);
+    return total;
+}
+
+}  // namespace nereus
+
+// ---------------------------------------------------------------------------------------------------
+// C ABI: descriptor, layout queries, compiler
+// ---------------------------------------------------------------------------------------------------
+
+#define NEREUS_GUARD_BEGIN try {
+#define NEREUS_GUARD_END   } catch (const std::bad_alloc&) { return NEREUS_ERR_NOMEM; } catch (...) { return NEREUS_ERR_ARG; }
+
+extern "C" {
+
+int nereus_model_desc(int layers, int hidden, int heads, int kv_heads, int ffn, int vocab, int dtype,
+                      nereus_model_desc_t* out) {
+    NEREUS_GUARD_BEGIN
+    if (!out || layers < 1 || hidden < 1 || heads < 1 || kv_heads < 1 || ffn < 1 || vocab < 1) return NEREUS_ERR_ARG;
+    if (dtype != NEREUS_BF16 && dtype != NEREUS_FP32) return NEREUS_ERR_ARG;
+    if (hidden % heads || heads % kv_heads) return NEREUS_ERR_INDIVISIBLE;
+    auto* d = new nereus_model_desc_s{layers, hidden, heads, kv_heads, ffn, vocab, dtype, false, {}};
+    build_catalogue(*d);
+    *out = d;
+    return NEREUS_OK;
+    NEREUS_GUARD_END
+}
+
+int nereus_model_desc_set_value_head(nereus_model_desc_t d, int out_dim) {
+    NEREUS_GUARD_BEGIN
+    if (!d) return NEREUS_ERR_ARG;
+    if (out_dim != 1) return NEREUS_ERR_UNSUPPORTED;
+    d->value_head = true;
+    build_catalogue(*d);
+    return NEREUS_OK;
+    NEREUS_GUARD_END
+}
+
+int nereus_model_desc_destroy(nereus_model_desc_t d) {
+    if (!d) return NEREUS_ERR_ARG;
+    delete d;
+    return NEREUS_OK;
+}
+
+int nereus_plan_check(nereus_model_desc_t d, nereus_plan_t p) {
+    if (!d) return NEREUS_ERR_ARG;
+    return check_plan(*d, p);
+}
+
+int nereus_plan_num_shards(nereus_model_desc_t d, nereus_plan_t p, int* n) {
+    if (!d || !n) return NEREUS_ERR_ARG;
+    if (int rc = check_plan(*d, p)) return rc;
+    *n = p.tp * p.pp;
+    return NEREUS_OK;
+}
+
+int nereus_plan_shard_bytes(nereus_model_desc_t d, nereus_plan_t p, int shard, size_t* bytes) {
+    NEREUS_GUARD_BEGIN
+    if (!d || !bytes) return NEREUS_ERR_ARG;
+    if (int rc = check_plan(*d, p)) return rc;
+    if (shard < 0 || shard >= p.tp * p.pp) return NEREUS_ERR_ARG;
+    StageLayout sl;
+    stage_layout(*d, p, shard / p.tp, sl);
+    *bytes = (size_t)sl.bytes;
+    return NEREUS_OK;
+    NEREUS_GUARD_END
+}
+
+int nereus_model_num_tensors(nereus_model_desc_t d, int* n) {
+    if (!d || !n) return NEREUS_ERR_ARG;
+    *n = (int)d->catalogue.size();
+    return NEREUS_OK;
+}
+
+int nereus_plan_tensor_slice(nereus_model_desc_t d, nereus_plan_t p, int shard, int tensor_id, size_t* offset,
+                             size_t* rows, size_t* cols, int* replicated) {
+    NEREUS_GUARD_BEGIN
+    if (!d || !offset || !rows || !cols) return NEREUS_ERR_ARG;
+    if (int rc = check_plan(*d, p)) return rc;
+    if (shard < 0 || shard >= p.tp * p.pp || tensor_id < 0 || tensor_id >= (int)d->catalogue.size())
+        return NEREUS_ERR_ARG;
+    StageLayout sl;
+    stage_layout(*d, p, shard / p.tp, sl);
+    if (replicated) *replicated = d->catalogue[tensor_id].cut == Cut::Whole;
+    if (sl.offset[tensor_id] == kNotHeld) { *offset = 0; *rows = 0; *cols = 0; return NEREUS_OK; }
+    int64_t r, c;
+    stored_block(d->catalogue[tensor_id], p.tp, r, c);
+    *offset = (size_t)sl.offset[tensor_id]; *rows = (size_t)r; *cols = (size_t)c;
+    return NEREUS_OK;
+    NEREUS_GUARD_END
+}
+
+int nereus_transition_compile(nereus_model_desc_t d, nereus_plan_t sp, nereus_plan_t dp, nereus_transition_t* out) {
+    NEREUS_GUARD_BEGIN
+    if (!d || !out) return NEREUS_ERR_ARG;
+    if (int rc = check_plan(*d, sp)) return rc;
+    if (int rc = check_plan(*d, dp)) return rc;
+    const int sdt = plan_dtype(*d, sp), ddt = plan_dtype(*d, dp);
+    if (!(sdt == ddt || (sdt == NEREUS_FP32 && ddt == NEREUS_BF16))) return NEREUS_ERR_UNSUPPORTED;
+    auto* t = new nereus_transition_s();
+    if (int rc = compile_one(*d, sp, dp, *t)) { delete t; return rc; }
+    finish(*t);
+    *out = t;
+    return NEREUS_OK;
+    NEREUS_GUARD_END
+}
+
+int nereus_transition_fuse(const nereus_transition_t* parts, int n, int chained, nereus_transition_t* out) {
+    NEREUS_GUARD_BEGIN
+    if (!parts || n < 1 || !out) return NEREUS_ERR_ARG;
+    for (int i = 0; i < n; ++i)
+        if (!parts[i] || parts[i]->n_levels != 1) return NEREUS_ERR_ARG;     // fuse takes compiled parts only
+    if (chained && n > kMaxLevels) return NEREUS_ERR_UNSUPPORTED;
+    auto* t = new nereus_transition_s();
+    if (!chained) {
+        size_t ns = 0, nd = 0;
+        for (int i = 0; i < n; ++i) { ns += parts[i]->src_bytes.size(); nd += parts[i]->dst_bytes.size(); }
+        if (ns + nd > (size_t)kMaxBuffers) { delete t; return NEREUS_ERR_UNSUPPORTED; }
+        size_t so = 0, dof = 0;
+        for (int i = 0; i < n; ++i) {
+            const nereus_transition_s& p = *parts[i];
+            const int pns = (int)p.src_bytes.size();
+            for (Rect r : p.rects) {
+                r.src_buf = (int32_t)(so + r.src_buf);
+                r.dst_buf = (int32_t)(ns + dof + (r.dst_buf - pns));
+                t->rects.push_back(r);
+            }
+            t->src_bytes.insert(t->src_bytes.end(), p.src_bytes.begin(), p.src_bytes.end());
+            t->dst_bytes.insert(t->dst_bytes.end(), p.dst_bytes.begin(), p.dst_bytes.end());
+            so += p.src_bytes.size(); dof += p.dst_bytes.size();
+        }
+        t->dst_level.assign(nd, 0);
+        t->dst_read_level.assign(nd, -1);
+        t->n_levels = 1;
+    } else {
+        for (int i = 1; i < n; ++i)
+            if (parts[i]->src_bytes != parts[i - 1]->dst_bytes) { delete t; return NEREUS_ERR_MISMATCH; }
+        const size_t ns = parts[0]->src_bytes.size();
+        size_t nd = 0;
+        for (int i = 0; i < n; ++i) nd += parts[i]->dst_bytes.size();
+        if (ns + nd > (size_t)kMaxBuffers) { delete t; return NEREUS_ERR_UNSUPPORTED; }
+        t->src_bytes = parts[0]->src_bytes;
+        size_t prev_base = 0;      // unified index of the buffers level k reads
+        size_t dof = 0;            // destinations emitted so far
+        for (int i = 0; i < n; ++i) {
+            const nereus_transition_s& p = *parts[i];
+            const int pns = (int)p.src_bytes.size();
+            for (Rect r : p.rects) {
+                r.src_buf = (int32_t)(prev_base + r.src_buf);
+                r.dst_buf = (int32_t)(ns + dof + (r.dst_buf - pns));
+                r.level = i;
+                t->rects.push_back(r);
+            }
+            for (size_t j = 0; j < p.dst_bytes.size(); ++j) {
+                t->dst_bytes.push_back(p.dst_bytes[j]);
+                t->dst_level.push_back(i);
+                t->dst_read_level.push_back(i + 1 < n ? i + 1 : -1);
+            }
+            prev_base = ns + dof;
+            dof += p.dst_bytes.size();
+        }
+        t->n_levels = n;
+    }
+    finish(*t);
+    *out = t;
+    return NEREUS_OK;
+    NEREUS_GUARD_END
+}
+
+int nereus_transition_num_buffers(nereus_transition_t t, int* n_src, int* n_dst) {
+    if (!t || !n_src || !n_dst) return NEREUS_ERR_ARG;
+    *n_src = (int)t->src_bytes.size(); *n_dst = (int)t->dst_bytes.size();
+    return NEREUS_OK;
+}
+
+int nereus_transition_buffer_bytes(nereus_transition_t t, int is_dst, int index, size_t* bytes) {
+    if (!t || !bytes || index < 0) return NEREUS_ERR_ARG;
+    const std::vector<uint64_t>& v = is_dst ? t->dst_bytes : t->src_bytes;
+    if ((size_t)index >= v.size()) return NEREUS_ERR_ARG;
+    *bytes = (size_t)v[index];
+    return NEREUS_OK;
+}
+
+int nereus_transition_bytes(nereus_transition_t t, size_t* read, size_t* written) {
+    if (!t || !read || !written) return NEREUS_ERR_ARG;
+    *read = (size_t)t->bytes_read; *written = (size_t)t->bytes_written;
+    return NEREUS_OK;
+}
+
+int nereus_transition_num_rects(nereus_transition_t t, int* n) {
+    if (!t || !n) return NEREUS_ERR_ARG;
+    *n = (int)t->rects.size();
+    return NEREUS_OK;
+}
+
+int nereus_transition_get_rect(nereus_transition_t t, int index, nereus_rect_t* out) {
+    if (!t || !out || index < 0 || (size_t)index >= t->rects.size()) return NEREUS_ERR_ARG;
+    const Rect& r = t->rects[index];
+    out->src_buf = r.src_buf; out->dst_buf = r.dst_buf; out->level = r.level; out->cast = r.cast;
+    out->src_off = r.src_off; out->dst_off = r.dst_off;
+    out->src_pitch = r.src_pitch; out->dst_pitch = r.dst_pitch;
+    out->rows = r.rows;
+    out->width_bytes_dst = r.width_dst; out->width_bytes_src = r.width_dst << r.cast;
+    return NEREUS_OK;
+}
+
+const char* nereus_strerror(int code) {
+    switch (code) {
+    case NEREUS_OK:              return "ok";
+    case NEREUS_ERR_ARG:         return "invalid argument";
+    case NEREUS_ERR_INDIVISIBLE: return "plan does not divide the model, or a piece is not a multiple of 16 bytes";
+    case NEREUS_ERR_UNSUPPORTED: return "unsupported dtype pair, tp > kv_heads, or too many buffers";
+    case NEREUS_ERR_ALIAS:       return "a destination buffer overlaps a source or another destination";
+    case NEREUS_ERR_CUDA:        return "a CUDA call failed";
+    case NEREUS_ERR_NOMEM:       return "out of host memory";
+    case NEREUS_ERR_MISMATCH:    return "chained parts do not connect";
+    case NEREUS_ERR_ALIGN:       return "a shard pointer is not 16-byte aligned";
+    default:                     return "unknown error";
+    }
+}
+
+}  // extern "C"

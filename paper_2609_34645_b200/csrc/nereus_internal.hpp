@@ -1,0 +1,147 @@
+// Internal types shared by the layout, the transition compiler and the launcher.  Not installed.
+#pragma once
+
+#include <cstdint>
+#include <cstddef>
+#include <vector>
+
+#include "nereus.h"
+
+namespace nereus {
+
+// ---------------------------------------------------------------------------------------------------
+// Model descriptor and the catalogue of stored tensors
+// ---------------------------------------------------------------------------------------------------
+
+// How a stored tensor is cut over TP ranks.
+enum class Cut : int {
+    Whole = 0,   // replicated: every TP rank stores the whole tensor            (norms, value head)
+    Rows  = 1,   // dim-0: one or more stacked segments, each cut by rows         (embed, head, qkv, gate_up)
+    Cols  = 2,   // dim-1: every row is cut into tp column pieces                 (wo, wdown)
+};
+
+// A stored tensor of the catalogue, before any plan is applied.
+struct StoredTensor {
+    Cut     cut;
+    int     nseg;        // Rows: number of stacked segments (1, 2 or 3); otherwise 1
+    int64_t seg_rows[3]; // Rows: logical rows of each segment; Whole/Cols: seg_rows[0] = rows
+    int64_t cols;        // logical columns (the contiguous dimension)
+    int     layer;       // owning layer, -1 embed (first stage), -2 final norm / head (last stage)
+};
+
+}  // namespace nereus
+
+struct nereus_model_desc_s {
+    int64_t L, H, nq, nkv, F, V;
+    int     dtype;
+    bool    value_head;
+    std::vector<nereus::StoredTensor> catalogue;   // 6L + 3 entries, in stored-id order
+};
+
+namespace nereus {
+
+inline int      elem_size(int dtype) { return dtype == NEREUS_FP32 ? 4 : 2; }
+inline int      plan_dtype(const nereus_model_desc_s& d, nereus_plan_t p) { return p.dtype ? p.dtype : d.dtype; }
+inline uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+
+void build_catalogue(nereus_model_desc_s& d);
+int  check_plan(const nereus_model_desc_s& d, nereus_plan_t p);
+
+// Byte layout of the shards of one pipeline stage under one plan (identical for all TP ranks of the stage).
+struct StageLayout {
+    std::vector<uint64_t> offset;   // per stored id; kNotHeld when the stage does not own the tensor
+    uint64_t              bytes;    // buffer length
+};
+constexpr uint64_t kNotHeld = ~0ull;
+
+// Stage that owns stored tensor `id` under a plan with `pp` stages.
+int  owning_stage(const nereus_model_desc_s& d, int id, int pp);
+void stage_layout(const nereus_model_desc_s& d, nereus_plan_t p, int stage, StageLayout& out);
+// Rows x cols (elements) of the block one TP rank of `tp` stores for tensor `t`.
+void stored_block(const StoredTensor& t, int tp, int64_t& rows, int64_t& cols);
+
+// ---------------------------------------------------------------------------------------------------
+// Task table
+// ---------------------------------------------------------------------------------------------------
+
+// Host form of one rect-copy task.  Widths and pitches in bytes; width_src = width_dst << cast.
+struct Rect {
+    int32_t  src_buf, dst_buf;   // unified buffer indices: [sources..., destinations...]
+    int32_t  level;
+    int32_t  cast;
+    uint64_t src_off, dst_off;
+    uint64_t src_pitch, dst_pitch;
+    uint64_t rows;
+    uint64_t width_dst;
+};
+
+// Device form, 64 bytes.  A rect is cut into tiles of rows_per_tile rows x tile_w bytes (dst side);
+// tile g of the table belongs to the rect with first_tile <= g < first_tile of the next rect.
+struct alignas(16) RectDev {
+    uint64_t src_off, dst_off;
+    uint64_t width;          // dst bytes per row piece
+    uint32_t src_pitch, dst_pitch;
+    uint32_t rows, rows_per_tile;
+    uint32_t tile_w;         // dst bytes per column tile
+    uint32_t col_tiles;
+    uint32_t first_tile;
+    uint16_t src_buf, dst_buf;
+    uint16_t level, cast;
+    uint32_t pad_;
+};
+static_assert(sizeof(RectDev) == 64, "RectDev must stay 64 bytes");
+
+// Control words on the device.
+struct Ctrl {
+    uint32_t cursor;      // next tile to claim
+    uint32_t done;        // tiles completed (only maintained for multi-level tables)
+    uint32_t status;      // NEREUS_DEV_*
+    uint32_t detail;      // tile index that raised the status
+};
+
+constexpr int kMaxBuffers = 448;      // pointers carried in the kernel's parameter block
+constexpr int kMaxLevels  = 8;
+
+struct Tuning {
+    int tile_bytes  = 0;
+    int ctas_per_sm = 0;
+    int threads     = 0;
+    int variant     = 0;
+};
+
+struct DeviceTable {                  // one per prepare()
+    int       device    = -1;
+    RectDev*  rects     = nullptr;
+    uint32_t* first     = nullptr;    // n_rects + 1 tile prefix
+    Ctrl*     ctrl      = nullptr;
+    uint32_t  n_tiles   = 0;
+    uint32_t  level_end[kMaxLevels] = {0};   // tiles up to and including each level
+    int       sm_count  = 0;
+    int       tile_bytes = 0, ctas_per_sm = 0, threads = 0, variant = 0;
+};
+
+}  // namespace nereus
+
+struct nereus_transition_s {
+    std::vector<nereus::Rect> rects;          // execution order
+    std::vector<uint64_t>     src_bytes;      // required length of each source buffer
+    std::vector<uint64_t>     dst_bytes;      // ... of each destination buffer
+    std::vector<int>          dst_level;      // level that writes destination buffer j
+    std::vector<int>          dst_read_level; // level that reads destination j (chained), -1 if none
+    int                       n_levels = 1;
+    uint64_t                  bytes_read = 0, bytes_written = 0;
+    nereus::Tuning            tuning;
+    nereus::DeviceTable       dev;
+    uint64_t                  launches = 0;
+};
+
+namespace nereus {
+
+// Cuts rects into tiles for a tile size; fills RectDev entries, the prefix and level ends.
+// Returns the number of tiles, or 0 with *overflow = true when it exceeds 32 bits.
+uint64_t tile_table(const nereus_transition_s& t, uint32_t tile_bytes, std::vector<RectDev>& out,
+                    std::vector<uint32_t>& first, uint32_t level_end[kMaxLevels]);
+
+void set_cuda_error(int e);
+
+}  // namespace nereus

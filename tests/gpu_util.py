@@ -1,0 +1,99 @@
+"""Helpers of the GPU parity tests: seeded device inputs laid out through the library's own layout query,
+destination buffers with sentinel fill and guard zones, and the comparison with the CPU oracle."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from oracle import oracle as O
+from paper_2609_34645_b200 import binding as B
+from paper_2609_34645_b200 import inputs as I
+
+GUARD = 4096
+SENTINEL = 0xA5
+ODT = {"bf16": O.BF16, "fp32": O.FP32}
+
+
+def desc_of(sh, dtype="bf16", value_head=False):
+    return B.ModelDesc(sh.layers, sh.hidden, sh.heads, sh.kv_heads, sh.ffn, sh.vocab, B.DTYPES[dtype], value_head)
+
+
+def omodel_of(sh, dtype="bf16", value_head=False):
+    return O.Model(sh.layers, sh.hidden, sh.heads, sh.kv_heads, sh.ffn, sh.vocab, ODT[dtype], value_head)
+
+
+def replica_groups(desc, plan):
+    """Byte ranges of replicated tensors, grouped per tensor and pipeline stage, from the library's query."""
+    n = desc.num_shards(plan)
+    groups = []
+    for tid in range(desc.num_tensors()):
+        grp = []
+        for s in range(n):
+            off, rows, cols, rep = desc.tensor_slice(plan, s, tid)
+            if rep and rows:
+                grp.append((s, off, rows * cols))        # (shard, byte offset, elements)
+        if len(grp) > 1:
+            groups.append(grp)
+    return groups
+
+
+def device_sources(desc, plan, dtype, seed, device="cuda"):
+    """Seeded N(0, 0.02) source shards on the device with replicated tensors tied."""
+    sizes = desc.shard_sizes(plan)
+    bufs = I.make_shards(sizes, dtype, seed, device)
+    es = I.element_size(dtype)
+    groups = [[(s, off, n * es) for s, off, n in g] for g in replica_groups(desc, plan)]
+    I.tie_replicas(bufs, groups)
+    return bufs
+
+
+class Guarded:
+    """Destination buffers with a guard zone on both sides, all pre-filled with a sentinel byte."""
+
+    def __init__(self, sizes, device="cuda"):
+        self.sizes = [int(s) for s in sizes]
+        self.raw = [torch.full((s + 2 * GUARD,), SENTINEL, dtype=torch.uint8, device=device) for s in self.sizes]
+        self.bufs = [r[GUARD:GUARD + s] for r, s in zip(self.raw, self.sizes)]
+
+    def ptrs(self):
+        return [b.data_ptr() for b in self.bufs]
+
+    def guards_intact(self):
+        for r, s in zip(self.raw, self.sizes):
+            if not bool((r[:GUARD] == SENTINEL).all()) or not bool((r[GUARD + s:] == SENTINEL).all()):
+                return False
+        return True
+
+
+def run_transition(t, src_bufs, dst_bufs, stream=None):
+    stream = stream or torch.cuda.current_stream()
+    t.run([b.data_ptr() for b in src_bufs], [b.data_ptr() for b in dst_bufs], stream.cuda_stream)
+    stream.synchronize()
+    assert t.status() == B.DEV_OK
+
+
+def oracle_expected(sh, a, b, sdt, ddt, vh, src_host):
+    m = omodel_of(sh, sdt, vh)
+    return O.reshard(m, O.Plan(*a), O.Plan(b[0], b[1], ODT[ddt]), src_host, fill=SENTINEL)
+
+
+def check_against_oracle(sh, a, b, sdt="bf16", ddt="bf16", vh=False, seed=0, tune=None):
+    """Full element-by-element parity of one transition, padding and guard zones included."""
+    desc = desc_of(sh, sdt, vh)
+    pa, pb = B.Plan(*a), B.Plan(b[0], b[1], B.DTYPES[ddt])
+    t = desc.compile(pa, pb)
+    if tune:
+        t.tune(**tune)
+    src = device_sources(desc, pa, sdt, seed)
+    dst = Guarded([t.buffer_bytes(True, j) for j in range(t.num_buffers()[1])])
+    before = t.launches()
+    run_transition(t, src, dst.bufs)
+    assert t.launches() == before + 1
+    want = oracle_expected(sh, a, b, sdt, ddt, vh, [s.cpu().numpy() for s in src])
+    for j, (g, w) in enumerate(zip(dst.bufs, want)):
+        g = g.cpu().numpy()
+        if not np.array_equal(g, w):
+            bad = np.flatnonzero(g != w)
+            raise AssertionError(f"{a}->{b} shard {j}: {bad.size} bytes differ, first at {bad[0]}")
+    assert dst.guards_intact()
+    return t

@@ -1,0 +1,303 @@
+"""Host logic of the CUDA library, checked without a GPU: exported symbols, layout queries, and the
+transition compiler's task table executed by a byte-loop interpreter (test scaffolding only) against the
+oracle."""
+import itertools
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import oracle as O
+from paper_2609_34645_b200 import binding as B
+from paper_2609_34645_b200 import inputs as I
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def desc_of(sh, dtype=B.BF16, value_head=False):
+    return B.ModelDesc(sh.layers, sh.hidden, sh.heads, sh.kv_heads, sh.ffn, sh.vocab, dtype, value_head)
+
+
+def omodel_of(sh, dtype=O.BF16, value_head=False):
+    return O.Model(sh.layers, sh.hidden, sh.heads, sh.kv_heads, sh.ffn, sh.vocab, dtype, value_head)
+
+
+def random_src(m, plan, seed, dtype):
+    """Seeded N(0, 0.02) source shards with replicated tensors tied, laid out by the oracle's layout."""
+    sizes = [O.shard_bytes(m, plan, s) for s in range(O.num_shards(m, plan))]
+    bufs = I.make_shards(sizes, dtype, seed)
+    groups = []
+    for t in range(O.num_logical(m)):
+        rows, cols = O.logical_shape(m, t)
+        held = [(s, O.locate(m, plan, s, t)) for s in range(len(sizes))]
+        held = [(s, p) for s, p in held if p.held]
+        if len(held) > 1 and all(p.nr * p.nc == rows * cols for _, p in held):
+            groups.append([(s, p.offset, p.nr * p.nc * O.es(m, plan)) for s, p in held])
+    I.tie_replicas(bufs, groups)
+    return [b.numpy() for b in bufs]
+
+
+def interpret(rects, src, dst, counts=None):
+    """Executes rect tasks on host byte arrays, level by level, in table order."""
+    bufs = list(src) + list(dst)
+    for r in rects:
+        s, d = bufs[r.src_buf], bufs[r.dst_buf]
+        for i in range(r.rows):
+            so, do = r.src_off + i * r.src_pitch, r.dst_off + i * r.dst_pitch
+            piece = s[so:so + r.width_bytes_src]
+            if r.cast:
+                piece = O.rne_bf16_array(piece.view(np.uint32)).view(np.uint8)
+            assert piece.size == r.width_bytes_dst
+            d[do:do + r.width_bytes_dst] = piece
+            if counts is not None:
+                counts[r.dst_buf - len(src)][do:do + r.width_bytes_dst] += 1
+
+
+def payload_mask(m, plan):
+    masks = [np.zeros(O.shard_bytes(m, plan, s), bool) for s in range(O.num_shards(m, plan))]
+    e = O.es(m, plan)
+    for s in range(len(masks)):
+        for t in range(O.num_logical(m)):
+            p = O.locate(m, plan, s, t)
+            if p.held:
+                masks[s][p.offset:p.offset + p.nr * p.nc * e] = True
+    return masks
+
+
+def plans_for(sh):
+    return [(tp, pp) for tp in (1, 2, 4, 8) for pp in (1, 2, 4, 8)
+            if tp <= sh.kv_heads and sh.kv_heads % tp == 0 and sh.ffn % tp == 0 and sh.vocab % tp == 0
+            and sh.layers % pp == 0]
+
+
+# ---------------------------------------------------------------- the boundary
+
+def test_library_exports_every_declared_symbol():
+    with open(os.path.join(ROOT, "include", "nereus.h")) as f:
+        text = re.sub(r"/\*.*?\*/", "", f.read(), flags=re.S)
+    declared = set(re.findall(r"\b(nereus_[a-z_0-9]+)\s*\(", text))
+    assert declared, "no declarations found"
+    assert declared == set(B.EXPORTS)
+    import ctypes
+    lib = ctypes.CDLL(B.LIB_PATH)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_argument_errors():
+    d = desc_of(I.TINY)
+    assert d.plan_check(B.Plan(4, 1)) == B.ERR_UNSUPPORTED
+    assert d.plan_check(B.Plan(1, 4)) == B.ERR_INDIVISIBLE
+    assert d.plan_check(B.Plan(0, 1)) == B.ERR_ARG
+    assert d.plan_check(B.Plan(1, 1, 7)) == B.ERR_ARG
+    with pytest.raises(B.NereusError) as e:
+        B.ModelDesc(2, 256, 3, 2, 688, 1024)
+    assert e.value.code == B.ERR_INDIVISIBLE
+    with pytest.raises(B.NereusError) as e:
+        B.ModelDesc(0, 256, 4, 2, 688, 1024)
+    assert e.value.code == B.ERR_ARG
+    with pytest.raises(B.NereusError) as e:
+        d.compile(B.Plan(1, 1, B.BF16), B.Plan(1, 1, B.FP32))      # bf16 -> fp32 is not a transition
+    assert e.value.code == B.ERR_UNSUPPORTED
+    with pytest.raises(B.NereusError) as e:
+        d.set_value_head(2)
+    assert e.value.code == B.ERR_UNSUPPORTED
+    # F/tp = 86 elements = 172 bytes: not a multiple of 16
+    with pytest.raises(B.NereusError) as e:
+        desc_of(I.Shape(2, 256, 4, 2, 172, 1024)).compile(B.Plan(1, 1), B.Plan(2, 1))
+    assert e.value.code == B.ERR_INDIVISIBLE
+    assert "16 bytes" in B.strerror(B.ERR_INDIVISIBLE)
+
+
+# ---------------------------------------------------------------- layout
+
+@pytest.mark.parametrize("sh,vh", [(I.TINY, False), (I.MICRO, True), (I.LLAMA_8B, False), (I.LLAMA_8B, True),
+                                   (I.DENSE_32B, False)])
+def test_layout_agrees_with_oracle(sh, vh):
+    """Shard sizes and every stored tensor's offset and extent equal the oracle's independent derivation."""
+    for es, bdt, odt in ((2, B.BF16, O.BF16), (4, B.FP32, O.FP32)):
+        d, m = desc_of(sh, bdt, vh), omodel_of(sh, odt, vh)
+        L = sh.layers
+        assert d.num_tensors() == 6 * L + 3
+        pls = plans_for(sh) if sh.layers <= 8 else [(1, 1), (4, 2), (2, 2), (4, 1), (8, 1), (2, 4)]
+        pls = [p for p in pls if p in plans_for(sh)]
+        for tp, pp in pls:
+            bp, op = B.Plan(tp, pp), O.Plan(tp, pp)
+            assert d.num_shards(bp) == O.num_shards(m, op)
+            layers = range(L) if L <= 8 else (0, 1, L // 2 - 1, L // 2, L - 1)
+            for s in range(tp * pp):
+                assert d.shard_bytes(bp, s) == O.shard_bytes(m, op, s)
+                # stored id -> the oracle's logical ids that make it up
+                pairs = [(0, [0]), (1 + 6 * L, [9 * L + 1]), (2 + 6 * L, [9 * L + 2])]
+                for l in layers:
+                    b6, b9 = 1 + 6 * l, 1 + 9 * l
+                    pairs += [(b6, [b9]), (b6 + 1, [b9 + 1, b9 + 2, b9 + 3]), (b6 + 2, [b9 + 4]), (b6 + 3, [b9 + 5]),
+                              (b6 + 4, [b9 + 6, b9 + 7]), (b6 + 5, [b9 + 8])]
+                for sid, lids in pairs:
+                    off, rows, cols, rep = d.tensor_slice(bp, s, sid)
+                    parts = [O.locate(m, op, s, t) for t in lids]
+                    if not parts[0].held:
+                        assert rows == 0 and cols == 0
+                        continue
+                    assert off == parts[0].offset
+                    assert rows * cols == sum(p.nr * p.nc for p in parts)
+                    assert cols == parts[0].nc
+                    cur = off
+                    for p in parts:                      # fused parts are stacked back to back
+                        assert p.offset == cur
+                        cur += p.nr * p.nc * es
+
+
+# ---------------------------------------------------------------- the compiler, executed on the host
+
+def check_transition(sh, a, b, sdt="bf16", ddt="bf16", vh=False, seed=0):
+    odt = {"bf16": O.BF16, "fp32": O.FP32}
+    d = desc_of(sh, B.DTYPES[sdt], vh)
+    m = omodel_of(sh, odt[sdt], vh)
+    oa, ob = O.Plan(*a), O.Plan(b[0], b[1], odt[ddt])
+    src = random_src(m, oa, seed, sdt)
+    want = O.reshard(m, oa, ob, src, fill=0xA5)
+    t = d.compile(B.Plan(*a), B.Plan(b[0], b[1], B.DTYPES[ddt]))
+    n_src, n_dst = t.num_buffers()
+    assert (n_src, n_dst) == (len(src), len(want))
+    for i, s in enumerate(src):
+        assert t.buffer_bytes(False, i) == s.size
+    got = [np.full(t.buffer_bytes(True, j), 0xA5, np.uint8) for j in range(n_dst)]
+    counts = [np.zeros(g.size, np.uint8) for g in got]
+    rects = t.rects()
+    interpret(rects, src, got, counts)
+    m_dst = omodel_of(sh, odt[ddt], vh)
+    for j, (g, w, c, mask) in enumerate(zip(got, want, counts, payload_mask(m_dst, O.Plan(b[0], b[1])))):
+        assert np.array_equal(g, w), (a, b, j)
+        assert np.array_equal(c == 1, mask), "every payload byte written exactly once, padding never"
+    rd, wr = t.bytes()
+    assert wr == sum(int(mk.sum()) for mk in payload_mask(m_dst, O.Plan(b[0], b[1])))
+    assert rd == wr * (2 if sdt != ddt else 1)
+    for r in rects:
+        assert r.src_off % 16 == 0 and r.dst_off % 16 == 0 and r.width_bytes_dst % 16 == 0
+        if r.rows > 1:
+            assert r.src_pitch % 16 == 0 and r.dst_pitch % 16 == 0
+    return t
+
+
+@pytest.mark.parametrize("a,b", list(itertools.product([(1, 1), (2, 1), (1, 2), (2, 2)], repeat=2)))
+def test_tiny_all_plan_pairs(a, b):
+    check_transition(I.TINY, a, b)
+
+
+def test_micro_plan_pairs_including_paper_example():
+    pls = plans_for(I.MICRO)
+    rng = np.random.default_rng(0)
+    pairs = [((4, 8), (8, 2)), ((4, 8), (4, 2)), ((4, 2), (8, 2)), ((1, 4), (2, 4)), ((8, 1), (1, 8))]
+    pairs += [(pls[i], pls[j]) for i, j in rng.integers(0, len(pls), (12, 2))]
+    for a, b in pairs:
+        check_transition(I.MICRO, a, b, seed=3)
+
+
+@pytest.mark.parametrize("a,b", [((2, 2), (4, 1)), ((1, 1), (2, 2)), ((4, 4), (1, 1)), ((2, 1), (2, 1))])
+def test_cast_transitions(a, b):
+    check_transition(I.SMALL, a, b, "fp32", "bf16", seed=2)
+
+
+def test_value_head_and_fp32():
+    check_transition(I.SMALL, (2, 1), (4, 2), vh=True, seed=5)
+    check_transition(I.SMALL, (4, 1), (2, 1), vh=True, seed=7)
+    check_transition(I.TINY, (1, 1), (2, 2), "fp32", "fp32", seed=1)
+
+
+def test_rect_counts_and_bytes_closed_form_8b():
+    d = desc_of(I.LLAMA_8B)
+    t = d.compile(B.Plan(1, 1), B.Plan(4, 2))
+    rd, wr = t.bytes()
+    repl = (2 * 32 + 1) * 4096 * 2 * 3                 # norms written once per extra TP replica
+    assert rd == wr == 8_030_261_248 * 2 + repl
+    rects = t.rects()
+    assert all(r.level == 0 and r.cast == 0 for r in rects)
+    sizes = [r.rows * r.width_bytes_dst for r in rects]
+    assert sizes == sorted(sizes, reverse=True)        # largest first
+    pitched = [r for r in rects if r.rows > 1]
+    assert len(pitched) == 32 * 4 * 2                  # wo and wdown, per layer and destination rank
+    assert {r.width_bytes_dst for r in pitched} == {2048, 7168}
+    t3 = desc_of(I.LLAMA_8B, B.FP32).compile(B.Plan(2, 2), B.Plan(4, 1, B.BF16))
+    rd, wr = t3.bytes()
+    assert rd == 2 * wr and wr == 8_030_261_248 * 2 + repl
+    assert all(r.cast == 1 for r in t3.rects())
+
+
+def test_identity_collapses_to_runs():
+    """Equal plans: every task is a contiguous run, adjacent tensors merged where no padding separates them."""
+    t = desc_of(I.TINY).compile(B.Plan(2, 1), B.Plan(2, 1))
+    assert all(r.rows == 1 for r in t.rects())
+
+
+def test_tiles_cover_tasks():
+    t = desc_of(I.SMALL).compile(B.Plan(1, 1), B.Plan(4, 2))
+    for tile in (512, 4096, 16384, 1 << 20):
+        t.tune(tile_bytes=tile)
+        tiles, levels = t.num_tiles()
+        want = 0
+        for r in t.rects():
+            if r.rows == 1 or r.width_bytes_dst >= tile:
+                want += r.rows * -(-r.width_bytes_dst // tile)
+            else:
+                want += -(-r.rows // max(1, tile // r.width_bytes_dst))
+        assert tiles == want and levels == 1
+    with pytest.raises(B.NereusError):
+        t.tune(tile_bytes=1000)
+
+
+# ---------------------------------------------------------------- fuse
+
+def test_fuse_independent_and_chained():
+    sh = I.TINY
+    d, m = desc_of(sh), omodel_of(sh)
+    a, b = (2, 1), (1, 2)
+    t_ab = d.compile(B.Plan(*a), B.Plan(*b))
+    t_ba = d.compile(B.Plan(*b), B.Plan(*a))
+    src = random_src(m, O.Plan(*a), 4, "bf16")
+    mid_want = O.reshard(m, O.Plan(*a), O.Plan(*b), src, fill=0xA5)
+
+    # chained round trip: level 0 writes `mid`, level 1 reads it and writes `back`
+    ch = B.Transition.fuse([t_ab, t_ba], chained=True)
+    assert ch.num_buffers() == (2, 4)
+    assert ch.num_tiles()[1] == 2
+    rects = ch.rects()
+    assert [r.level for r in rects] == sorted(r.level for r in rects)
+    mid = [np.full(ch.buffer_bytes(True, j), 0xA5, np.uint8) for j in range(2)]
+    back = [np.full(ch.buffer_bytes(True, 2 + j), 0xA5, np.uint8) for j in range(2)]
+    interpret(rects, src, mid + back)
+    for g, w in zip(mid, mid_want):
+        assert np.array_equal(g, w)
+    for mk, g, s in zip(payload_mask(m, O.Plan(*a)), back, src):
+        assert np.array_equal(g[mk], s[mk])
+    rd, wr = ch.bytes()
+    assert rd == wr == sum(t_ab.bytes()[1:]) + sum(t_ba.bytes()[1:])
+
+    # independent: two model-stages side by side
+    ind = B.Transition.fuse([t_ab, t_ba], chained=False)
+    assert ind.num_buffers() == (4, 4)
+    src2 = random_src(m, O.Plan(*b), 6, "bf16")
+    out = [np.full(ind.buffer_bytes(True, j), 0xA5, np.uint8) for j in range(4)]
+    interpret(ind.rects(), src + src2, out)
+    for g, w in zip(out, mid_want + O.reshard(m, O.Plan(*b), O.Plan(*a), src2, fill=0xA5)):
+        assert np.array_equal(g, w)
+
+    # parts that do not connect
+    with pytest.raises(B.NereusError) as e:
+        B.Transition.fuse([t_ab, t_ab], chained=True)
+    assert e.value.code == B.ERR_MISMATCH
+    with pytest.raises(B.NereusError) as e:
+        B.Transition.fuse([ch, t_ab], chained=False)          # only compiled parts fuse
+    assert e.value.code == B.ERR_ARG
+
+
+def test_run_rejects_bad_pointers_before_any_cuda_call():
+    t = desc_of(I.TINY).compile(B.Plan(2, 1), B.Plan(1, 1))
+    sizes = [t.buffer_bytes(False, 0), t.buffer_bytes(False, 1)]
+    base = 1 << 40
+    src = [base, base + (1 << 30)]
+    assert t.run_raw([0, src[1]], [base + (2 << 30)]) == B.ERR_ARG
+    assert t.run_raw([src[0] + 8, src[1]], [base + (2 << 30)]) == B.ERR_ALIGN
+    assert t.run_raw(src, [src[1] + sizes[1] - 256]) == B.ERR_ALIAS        # dst overlaps a source's tail
+    assert t.run_raw(src, [src[0] - 16]) == B.ERR_ALIAS

@@ -74,6 +74,16 @@ WORKLOADS = {
         Stage("32b", DENSE_32B, 8, (2, 4, "bf16"), (8, 1, "bf16")),), round_trip=True),
 }
 
+# profiling stand-in: the 8B shape cut to 4 layers (3.85 GB each side: larger than L2, small enough for a
+# multi-pass profiler capture); same tensor classes and piece sizes as the full Split
+LLAMA_8B_4L = Shape(4, 4096, 32, 8, 14336, 128256)
+WORKLOADS["8b4l_tp1pp1_to_tp4pp2"] = Workload("8b4l_tp1pp1_to_tp4pp2", (
+    Stage("8b4l", LLAMA_8B_4L, 1, (1, 1, "bf16"), (4, 2, "bf16")),))
+WORKLOADS["8b4l_tp4pp2_to_tp1pp1"] = Workload("8b4l_tp4pp2_to_tp1pp1", (
+    Stage("8b4l", LLAMA_8B_4L, 1, (4, 2, "bf16"), (1, 1, "bf16")),))
+WORKLOADS["8b4l_fp32_tp2pp2_to_bf16_tp4pp1"] = Workload("8b4l_fp32_tp2pp2_to_bf16_tp4pp1", (
+    Stage("8b4l_master", LLAMA_8B_4L, 2, (2, 2, "fp32"), (4, 1, "bf16")),))
+
 # scaled-down stand-ins with the same structure, for parity tests the oracle finishes in seconds
 SMALL = Shape(4, 512, 8, 4, 1376, 2048)            # head_dim 64; several tiles and ragged tails
 MICRO = Shape(8, 64, 8, 8, 128, 128)               # head_dim 8; brute-force sized, TP up to 8, PP up to 8

@@ -66,6 +66,7 @@ extern "C" {
 #define NEREUS_ERR_NOMEM         -6   /* host allocation failed                                            */
 #define NEREUS_ERR_MISMATCH      -7   /* parts of a chained fuse do not connect (buffer count or sizes)    */
 #define NEREUS_ERR_ALIGN         -8   /* a shard pointer is not 16-byte aligned                            */
+#define NEREUS_ERR_TOO_LARGE     -9   /* more tasks than the fixed scratch of nereus_transition_run_static */
 
 /* device status word (nereus_transition_status) */
 #define NEREUS_DEV_OK             0
@@ -176,6 +177,30 @@ int nereus_transition_run(nereus_transition_t t, const void* const* src_ptrs, vo
 int nereus_transition_status(nereus_transition_t t, int* device_status);
 /* Kernels this handle has launched since it was created (one per run). */
 int nereus_transition_launches(nereus_transition_t t, uint64_t* n);
+
+/* ---- execution without allocation --------------------------------------------------------------------- */
+
+/* The paper has no counterpart of this entry point; it exists for callers that cannot allocate device
+ * memory when a transition is due: a process that gave all of HBM to its own pool (a server with a
+ * pre-sized KV cache, a trainer whose caching allocator owns the device) has nothing left for cudaMalloc,
+ * and at a near-capacity boundary the table upload of nereus_transition_prepare may fail.
+ *
+ * Same contract, arguments and result as nereus_transition_run, but it calls no cudaMalloc, cudaFree or any
+ * other allocating routine and never touches the handle's device copy: the task table and the control
+ * words go into one fixed array in the library's device image, NEREUS_STATIC_MAX_RECTS tasks at most
+ * (about 272 KiB, held on every GPU the process uses until it exits).  The table is copied there on
+ * `cuda_stream` by every call (two small cudaMemcpyAsync and a memset ahead of the kernel).
+ *   - A transition with more tasks (nereus_transition_num_rects) is refused with NEREUS_ERR_TOO_LARGE.
+ *   - The first call on a device looks the array's device address up (cudaGetSymbolAddress) and reads the
+ *     SM count; make that first call outside any stream capture.
+ *   - All handles and all calls on one device share the array, which keeps the previous call's contents
+ *     until the next one overwrites it: two calls whose work overlaps on the GPU (different streams, or
+ *     different threads) race on it.  Issue them on one stream, or order them with events.
+ *   - nereus_transition_status does not see these runs: their status word lives in the shared array and is
+ *     not exported.  It only ever matters for chained tables (a dependency wait that gives up). */
+#define NEREUS_STATIC_MAX_RECTS 4096
+int nereus_transition_run_static(nereus_transition_t t, const void* const* src_ptrs, void* const* dst_ptrs,
+                                 void* cuda_stream);
 
 const char* nereus_strerror(int code);
 /* cudaError_t of the last failed CUDA call made by this library on the calling thread (0 if none). */

@@ -19,6 +19,8 @@ DTYPES = {"bf16": BF16, "fp32": FP32}
 OK = 0
 ERR_ARG, ERR_INDIVISIBLE, ERR_UNSUPPORTED, ERR_ALIAS = -1, -2, -3, -4
 ERR_CUDA, ERR_NOMEM, ERR_MISMATCH, ERR_ALIGN = -5, -6, -7, -8
+ERR_TOO_LARGE = -9
+STATIC_MAX_RECTS = 4096
 DEV_OK, DEV_BOUNDS, DEV_TIMEOUT = 0, 1, 2
 
 if not os.path.exists(LIB_PATH):
@@ -81,6 +83,7 @@ _SIGS = {
     "nereus_transition_status": [_vp, _P(_i)],
     "nereus_transition_launches": [_vp, _P(ctypes.c_uint64)],
     "nereus_last_cuda_error": [],
+    "nereus_transition_run_static": [_vp, _P(_vp), _P(_vp), _vp],
 }
 for _name, _args in _SIGS.items():
     _f = getattr(_lib, _name)          # AttributeError here = the library does not export a declared symbol
@@ -225,6 +228,24 @@ class Transition:
         if not isinstance(dst_ptrs, ctypes.Array):
             dst_ptrs = self.pointer_array(dst_ptrs)
         return _lib.nereus_transition_run(self._h, src_ptrs, dst_ptrs, _vp(stream))
+
+    def run_static(self, src_ptrs, dst_ptrs, stream=0):
+        """nereus_transition_run_static: the same transition without any device allocation, for callers
+        whose memory pool owns the whole GPU.  At most STATIC_MAX_RECTS tasks; calls that overlap on the
+        device race on the shared table; make the first call on a device outside stream capture."""
+        if not isinstance(src_ptrs, ctypes.Array):
+            src_ptrs = self.pointer_array(src_ptrs)
+        if not isinstance(dst_ptrs, ctypes.Array):
+            dst_ptrs = self.pointer_array(dst_ptrs)
+        _ck(_lib.nereus_transition_run_static(self._h, src_ptrs, dst_ptrs, _vp(stream)),
+            "nereus_transition_run_static")
+
+    def run_static_raw(self, src_ptrs, dst_ptrs, stream=0) -> int:
+        if not isinstance(src_ptrs, ctypes.Array):
+            src_ptrs = self.pointer_array(src_ptrs)
+        if not isinstance(dst_ptrs, ctypes.Array):
+            dst_ptrs = self.pointer_array(dst_ptrs)
+        return _lib.nereus_transition_run_static(self._h, src_ptrs, dst_ptrs, _vp(stream))
 
     def status(self) -> int:
         s = _i()

@@ -434,3 +434,98 @@ int nereus_transition_destroy(nereus_transition_t t) {
 int nereus_last_cuda_error(void) { return g_last_cuda_error; }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------------
+// run without any allocation: the task table lives in a fixed device array
+// ---------------------------------------------------------------------------------------------------
+//
+// Some callers cannot allocate device memory at the moment they need a transition: an engine that handed
+// all of HBM to its own pool (a serving process with a pre-sized KV cache, a trainer whose caching
+// allocator owns the device) has nothing left for cudaMalloc to give, and at a near-capacity safe boundary
+// the allocation that prepare() makes may simply fail.  For them the table and the control words sit in
+// this file-scope array, which every process that loads the library holds on every GPU it touches until
+// it exits.
+
+namespace nereus {
+
+constexpr int    kStaticMaxRects    = 4096;
+constexpr size_t kStaticRectBytes   = (size_t)kStaticMaxRects * sizeof(RectDev);              // 256 KiB
+constexpr size_t kStaticFirstBytes  = ((size_t)kStaticMaxRects + 1 + 63) / 64 * 64 * sizeof(uint32_t);
+constexpr size_t kStaticScratchBytes = kStaticRectBytes + kStaticFirstBytes + 256;            // ~272 KiB
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kStaticMaxDevices = 64;
+static unsigned char* g_static_ptr[kStaticMaxDevices];   // device address of the array, per device
+static int            g_static_sms[kStaticMaxDevices];
+
+// Once per device, with that device current: the array's name is only a host-side handle of the symbol;
+// the address a kernel can use comes from cudaGetSymbolAddress.
+static int static_scratch(int device, unsigned char** ptr, int* sms) {
+    if (device < 0 || device >= kStaticMaxDevices) return NEREUS_ERR_UNSUPPORTED;
+    if (!g_static_ptr[device]) {
+        unsigned char* p = nullptr;
+        NEREUS_CUDA(cudaGetSymbolAddress((void**)&p, g_static_scratch));
+        int n = 0;
+        NEREUS_CUDA(cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, device));
+        g_static_sms[device] = n;
+        g_static_ptr[device] = p;
+    }
+    *ptr = g_static_ptr[device];
+    *sms = g_static_sms[device];
+    return NEREUS_OK;
+}
+
+}  // namespace nereus
+
+extern "C" int nereus_transition_run_static(nereus_transition_t t, const void* const* src_ptrs,
+                                            void* const* dst_ptrs, void* cuda_stream) {
+    try {
+        if (!t || !src_ptrs || !dst_ptrs) return NEREUS_ERR_ARG;
+        if (t->rects.size() > (size_t)kStaticMaxRects) return NEREUS_ERR_TOO_LARGE;
+        if (int rc = check_buffers(*t, src_ptrs, dst_ptrs)) return rc;
+        int device = 0;
+        NEREUS_CUDA(cudaGetDevice(&device));
+        unsigned char* scratch = nullptr;
+        int sms = 0;
+        if (int rc = static_scratch(device, &scratch, &sms)) return rc;
+        cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+
+        const int tile_bytes  = t->tuning.tile_bytes  ? t->tuning.tile_bytes  : env_int("NEREUS_TILE_BYTES", 16384);
+        const int ctas_per_sm = t->tuning.ctas_per_sm ? t->tuning.ctas_per_sm : env_int("NEREUS_CTAS_PER_SM", 2);
+        const int threads     = t->tuning.threads     ? t->tuning.threads     : env_int("NEREUS_THREADS", 512);
+        if (tile_bytes < 512 || tile_bytes % 512 || ctas_per_sm < 1 || ctas_per_sm > 2 || threads < 32 ||
+            threads > 512 || threads % 32)
+            return NEREUS_ERR_ARG;
+
+        WalkParams p;
+        std::vector<RectDev>  rects;        // host memory only
+        std::vector<uint32_t> first;
+        const uint64_t n_tiles = tile_table(*t, (uint32_t)tile_bytes, rects, first, p.level_end);
+        if (n_tiles == 0 && !t->rects.empty()) return NEREUS_ERR_UNSUPPORTED;
+
+        RectDev*  d_rects = reinterpret_cast<RectDev*>(scratch);
+        uint32_t* d_first = reinterpret_cast<uint32_t*>(scratch + kStaticRectBytes);
+        Ctrl*     d_ctrl  = reinterpret_cast<Ctrl*>(scratch + kStaticRectBytes + kStaticFirstBytes);
+        // the array keeps whatever the previous call left: overwrite the table, zero the control words
+        NEREUS_CUDA(cudaMemcpyAsync(d_rects, rects.data(), rects.size() * sizeof(RectDev), cudaMemcpyHostToDevice, stream));
+        NEREUS_CUDA(cudaMemcpyAsync(d_first, first.data(), first.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, stream));
+        NEREUS_CUDA(cudaMemsetAsync(d_ctrl, 0, sizeof(Ctrl), stream));
+
+        p.rects = d_rects; p.first = d_first; p.ctrl = d_ctrl;
+        p.n_rects = (uint32_t)t->rects.size(); p.n_tiles = (uint32_t)n_tiles; p.n_levels = (uint32_t)t->n_levels;
+        const size_t ns = t->src_bytes.size(), nd = t->dst_bytes.size();
+        for (size_t i = 0; i < ns; ++i) p.bufs[i] = (char*)const_cast<void*>(src_ptrs[i]);
+        for (size_t j = 0; j < nd; ++j) p.bufs[ns + j] = (char*)dst_ptrs[j];
+        for (size_t k = ns + nd; k < (size_t)kMaxBuffers; ++k) p.bufs[k] = nullptr;
+        if (n_tiles > 0) {
+            const unsigned warps_per_cta = (unsigned)threads / 32;
+            unsigned grid = (unsigned)(sms * ctas_per_sm);
+            grid = std::max(1u, std::min(grid, ((unsigned)n_tiles + warps_per_cta - 1) / warps_per_cta));
+            nereus_walk_vec<<<grid, threads, 0, stream>>>(p);
+            NEREUS_CUDA(cudaGetLastError());
+            t->launches += 1;
+        }
+        return NEREUS_OK;
+    } catch (const std::bad_alloc&) { return NEREUS_ERR_NOMEM; }
+}

@@ -337,7 +337,7 @@ def run_ours(args):
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": NCU_TRAFFIC_PER_ALGORITHMIC_BYTE * (rd + wr),
                      "traffic_note": "ncu capture on the 4-layer stand-in, scaled by bytes moved",
-                     "peak_kind": f"of {peak_kind}", "kernel": "nereus_walk",
+                     "peak_kind": f"of {peak_kind}", "kernel": t.launch_info()["kernel"], "launch": t.launch_info(),
                      "kernel_ms": kernel_ms, "kernel_ms_min": min(per_step)},
         "clocks": clocks, "gpu_launches": launches,
     }

@@ -152,9 +152,15 @@ int nereus_transition_num_tiles(nereus_transition_t t, uint64_t* tiles, int* lev
 
 /* Launch tuning; 0 keeps the default of a field.  tile_bytes: target bytes per claimed tile (multiple of
  * 512).  ctas_per_sm, threads: persistent grid = SMs * ctas_per_sm blocks of `threads` threads.
- * variant: 0 default, 1 register-staged vector copy, 2 bulk-copy shared-memory ring.
+ * variant: 0 default (the ring where it applies), 1 register-staged vector copy, 2 bulk-copy shared-memory
+ * ring (tables with a cast or with several levels always run on the vector kernel).  tile_bytes 0 = 16 KiB (32 KiB per ring stage),
+ * halved for small tables until every claimer gets a few tiles.
  * Drops the device copy of the table (the next prepare/run uploads it again).  Errors: ARG. */
 int nereus_transition_tune(nereus_transition_t t, int tile_bytes, int ctas_per_sm, int threads, int variant);
+
+/* The launch shape the next run on the current device will use (after nereus_transition_prepare; before it,
+ * what a 148-SM device would get): kernel variant (1 vector copy, 2 bulk ring), tile bytes, grid, block. */
+int nereus_transition_launch_info(nereus_transition_t t, int* variant, int* tile_bytes, int* grid, int* threads);
 
 /* ---- execution (the local layout change of Section 6.2) ---------------------------------------------- */
 

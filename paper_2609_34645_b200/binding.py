@@ -79,6 +79,7 @@ _SIGS = {
     "nereus_transition_num_tiles": [_vp, _P(ctypes.c_uint64), _P(_i)],
     "nereus_transition_tune": [_vp, _i, _i, _i, _i],
     "nereus_transition_prepare": [_vp],
+    "nereus_transition_launch_info": [_vp, _P(_i), _P(_i), _P(_i), _P(_i)],
     "nereus_transition_run": [_vp, _P(_vp), _P(_vp), _vp],
     "nereus_transition_status": [_vp, _P(_i)],
     "nereus_transition_launches": [_vp, _P(ctypes.c_uint64)],
@@ -204,6 +205,13 @@ class Transition:
 
     def tune(self, tile_bytes=0, ctas_per_sm=0, threads=0, variant=0):
         _ck(_lib.nereus_transition_tune(self._h, tile_bytes, ctas_per_sm, threads, variant), "nereus_transition_tune")
+
+    def launch_info(self) -> dict:
+        v, tb, g, th = _i(), _i(), _i(), _i()
+        _ck(_lib.nereus_transition_launch_info(self._h, ctypes.byref(v), ctypes.byref(tb), ctypes.byref(g),
+                                               ctypes.byref(th)), "nereus_transition_launch_info")
+        return {"kernel": {1: "nereus_walk_vec", 2: "nereus_walk_bulk"}[v.value], "tile_bytes": tb.value,
+                "grid": g.value, "threads": th.value}
 
     def prepare(self):
         _ck(_lib.nereus_transition_prepare(self._h), "nereus_transition_prepare")

@@ -12,7 +12,12 @@
 //     contiguous per instruction, kUnroll independent loads in flight per lane before the first store.
 //   * tables with several dependency levels (chained transitions): a tile of level k waits, with a poll
 //     limit, until every tile of level k-1 has completed; on giving up it records NEREUS_DEV_TIMEOUT and the
-//     warp leaves.  Loads bypass L1 (ld.global.cg) so a level reads what another SM wrote before it.
+//     warp leaves.  A warp publishes its completed tiles once per level (one fence, one atomic), not per
+//     tile.  Loads bypass L1 (ld.global.cg) so a level reads what another SM wrote before it.
+//   * second kernel, nereus_walk_bulk, for single-level bit-copy tables: one CTA per SM, a producer warp
+//     that claims tiles and issues cp.async.bulk global -> shared copies into a ring of stages, and a
+//     consumer warp that issues cp.async.bulk shared -> global stores; mbarriers track both directions and
+//     every wait has an iteration limit.
 #include <cuda_runtime.h>
 
 #include <algorithm>
@@ -58,6 +63,12 @@ constexpr uint32_t kGatePolls   = 1u << 21;     // x ~200 ns sleep: gives up aft
 __device__ __forceinline__ uint32_t claim_tile(Ctrl* ctrl, unsigned lane) {
     uint32_t g = 0;
     if (lane == 0) g = atomicAdd(&ctrl->cursor, 1u);
+    return __shfl_sync(0xffffffffu, g, 0);
+}
+
+__device__ __forceinline__ uint32_t claim_tiles(Ctrl* ctrl, unsigned lane, uint32_t n) {
+    uint32_t g = 0;
+    if (lane == 0) g = atomicAdd(&ctrl->cursor, n);
     return __shfl_sync(0xffffffffu, g, 0);
 }
 
@@ -169,82 +180,289 @@ __device__ __forceinline__ void cast_tile(const char* __restrict__ s, char* __re
 }
 
 // ---------------------------------------------------------------------------------------------------
-// the persistent walker (register-staged vector copy)
+// tile index -> addresses
 // ---------------------------------------------------------------------------------------------------
 
-__global__ void __launch_bounds__(512, 2) nereus_walk_vec(const __grid_constant__ WalkParams p) {
-    const unsigned lane = threadIdx.x & 31;
-    Ctrl* const    ctrl = p.ctrl;
+struct Tile {
+    const char* s;
+    char*       d;
+    uint32_t    nr, w, sp, dp;     // row pieces, dst bytes per piece, pitches
+    uint32_t    level, cast;
+};
 
-    uint32_t g = claim_tile(ctrl, lane);
-    while (g < p.n_tiles) {
-        const uint32_t g_next = claim_tile(ctrl, lane);      // in flight while this tile is copied
+// The rect a claimer resolved last: consecutive claims of one warp usually fall into the same rect (a rect
+// has thousands of tiles), so the binary search is skipped while first <= g < next_first.
+struct RectRange {
+    uint32_t index = 0, first = 1, next_first = 0;            // empty range
+};
 
-        // tile -> rect: largest i with first[i] <= g
+// Resolves tile g: binary search for the rect (largest i with first[i] <= g), then row block x column block.
+// Returns false when the table does not resolve (corrupted).
+template <bool kUseRange>
+__device__ __forceinline__ bool resolve_tile(const WalkParams& p, uint32_t g, RectRange& rr, Tile& t) {
+    if (!kUseRange || g < rr.first || g >= rr.next_first) {
         uint32_t lo = 0, hi = p.n_rects;                       // invariant: first[lo] <= g < first[hi]
         while (hi - lo > 1) {
             const uint32_t mid = (lo + hi) >> 1;
             if (__ldg(p.first + mid) <= g) lo = mid; else hi = mid;
         }
-        const RectDev* rp = p.rects + lo;
-        const uint4 q0 = __ldg(reinterpret_cast<const uint4*>(rp));          // src_off, dst_off
-        const uint4 q1 = __ldg(reinterpret_cast<const uint4*>(rp) + 1);      // width, src_pitch, dst_pitch
-        const uint4 q2 = __ldg(reinterpret_cast<const uint4*>(rp) + 2);      // rows, rows_per_tile, tile_w, col_tiles
-        const uint4 q3 = __ldg(reinterpret_cast<const uint4*>(rp) + 3);      // first_tile, bufs, level|cast
-        const uint64_t src_off = ((uint64_t)q0.y << 32) | q0.x, dst_off = ((uint64_t)q0.w << 32) | q0.z;
-        const uint64_t width   = ((uint64_t)q1.y << 32) | q1.x;
-        const uint32_t sp = q1.z, dp = q1.w;
-        const uint32_t rows = q2.x, rpt = q2.y, tile_w = q2.z, col_tiles = q2.w;
-        const uint32_t first_tile = q3.x;
-        const uint32_t src_buf = q3.y & 0xFFFFu, dst_buf = q3.y >> 16;
-        const uint32_t level = q3.z & 0xFFFFu, cast = q3.z >> 16;
+        rr.index = lo;
+        if (kUseRange) {
+            rr.first = __ldg(p.first + lo);
+            rr.next_first = __ldg(p.first + lo + 1);
+        }
+    }
+    const RectDev* rp = p.rects + rr.index;
+    const uint4 q0 = __ldg(reinterpret_cast<const uint4*>(rp));          // src_off, dst_off
+    const uint4 q1 = __ldg(reinterpret_cast<const uint4*>(rp) + 1);      // width, src_pitch, dst_pitch
+    const uint4 q2 = __ldg(reinterpret_cast<const uint4*>(rp) + 2);      // rows, rows_per_tile, tile_w, col_tiles
+    const uint4 q3 = __ldg(reinterpret_cast<const uint4*>(rp) + 3);      // first_tile, bufs, level|cast
+    const uint64_t src_off = ((uint64_t)q0.y << 32) | q0.x, dst_off = ((uint64_t)q0.w << 32) | q0.z;
+    const uint64_t width   = ((uint64_t)q1.y << 32) | q1.x;
+    const uint32_t rows = q2.x, rpt = q2.y, tile_w = q2.z, col_tiles = q2.w;
+    const uint32_t first_tile = q3.x;
+    const uint32_t src_buf = q3.y & 0xFFFFu, dst_buf = q3.y >> 16;
+    t.sp = q1.z; t.dp = q1.w;
+    t.level = q3.z & 0xFFFFu; t.cast = q3.z >> 16;
+    if (first_tile > g || src_buf >= (uint32_t)kMaxBuffers || dst_buf >= (uint32_t)kMaxBuffers || col_tiles == 0)
+        return false;
+    const uint32_t k  = g - first_tile;
+    const uint32_t rb = k / col_tiles, cb = k - rb * col_tiles;
+    const uint32_t r0 = rb * rpt;
+    if (r0 >= rows) return false;
+    const uint64_t c0 = (uint64_t)cb * tile_w;                 // dst bytes into the row piece
+    t.nr = min(rpt, rows - r0);
+    t.w  = (uint32_t)min((uint64_t)tile_w, width - c0);
+    t.s  = p.bufs[src_buf] + src_off + (uint64_t)r0 * t.sp + (c0 << t.cast);
+    t.d  = p.bufs[dst_buf] + dst_off + (uint64_t)r0 * t.dp + c0;
+    return true;
+}
 
-        if (first_tile > g || src_buf >= (uint32_t)kMaxBuffers || dst_buf >= (uint32_t)kMaxBuffers) {
-            if (lane == 0) { atomicCAS(&ctrl->status, NEREUS_DEV_OK, NEREUS_DEV_BOUNDS); ctrl->detail = g; }
+__device__ __forceinline__ void raise_status(Ctrl* ctrl, uint32_t status, uint32_t detail) {
+    if (atomicCAS(&ctrl->status, (uint32_t)NEREUS_DEV_OK, status) == (uint32_t)NEREUS_DEV_OK) ctrl->detail = detail;
+}
+
+// ---------------------------------------------------------------------------------------------------
+// the persistent walker, register-staged vector copy (every table)
+// ---------------------------------------------------------------------------------------------------
+
+__global__ void __launch_bounds__(512, 2) nereus_walk_vec(const __grid_constant__ WalkParams p) {
+    const unsigned lane = threadIdx.x & 31;
+    Ctrl* const    ctrl = p.ctrl;
+    uint32_t       my_done = 0, my_level = 0;                  // tiles completed and not yet published
+    uint32_t       open_level = 0;                             // highest level whose gate this warp has passed
+    RectRange      rr;
+
+    uint32_t g = claim_tile(ctrl, lane);
+    while (g < p.n_tiles) {
+        const uint32_t g_next = claim_tile(ctrl, lane);        // in flight while this tile is copied
+        Tile t;
+        if (!resolve_tile<false>(p, g, rr, t)) {
+            if (lane == 0) raise_status(ctrl, NEREUS_DEV_BOUNDS, g);
             return;
         }
 
-        // dependency gate
-        if (level > 0) {
-            const uint32_t need = p.level_end[level - 1];
-            uint32_t polls = 0;
+        if (t.level != my_level) {
+            // leaving a level: make this warp's stores visible, publish its tiles, then wait for the level
+            // below this tile's to be complete everywhere
+            if (my_done) {
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) atomicAdd(&ctrl->done, my_done);
+                my_done = 0;
+            }
+            my_level = t.level;
+        }
+        if (t.level > open_level) {
+            const uint32_t need = p.level_end[t.level - 1];
             bool ok = true;
             if (lane == 0) {
+                uint32_t polls = 0;
                 while (ld_acquire_u32(&ctrl->done) < need) {
                     if (++polls > kGatePolls) { ok = false; break; }
                     __nanosleep(200);
                 }
-                if (!ok) { atomicCAS(&ctrl->status, NEREUS_DEV_OK, NEREUS_DEV_TIMEOUT); ctrl->detail = g; }
+                if (!ok) raise_status(ctrl, NEREUS_DEV_TIMEOUT, g);
             }
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) return;
             __threadfence();
+            open_level = t.level;
         }
 
-        // tile -> row block x column block
-        const uint32_t t  = g - first_tile;
-        const uint32_t rb = t / col_tiles, cb = t - rb * col_tiles;
-        const uint32_t r0 = rb * rpt;
-        const uint32_t nr = min(rpt, rows - r0);
-        const uint64_t c0 = (uint64_t)cb * tile_w;                     // dst bytes into the row piece
-        const uint32_t w  = (uint32_t)min((uint64_t)tile_w, width - c0);
-        const char* s = p.bufs[src_buf] + src_off + (uint64_t)r0 * sp + (c0 << cast);
-        char*       d = p.bufs[dst_buf] + dst_off + (uint64_t)r0 * dp + c0;
-
-        if (cast) {
-            cast_tile<kUnrollRect>(s, d, nr, w >> 3, sp, dp, lane);
-        } else if (nr == 1) {
-            copy_run<kUnrollRun>(s, d, w >> 4, lane);
+        if (t.cast) {
+            cast_tile<kUnrollRect>(t.s, t.d, t.nr, t.w >> 3, t.sp, t.dp, lane);
+        } else if (t.nr == 1) {
+            copy_run<kUnrollRun>(t.s, t.d, t.w >> 4, lane);
         } else {
-            copy_rect<kUnrollRect>(s, d, nr, w >> 4, sp, dp, lane);
+            copy_rect<kUnrollRect>(t.s, t.d, t.nr, t.w >> 4, t.sp, t.dp, lane);
         }
-
-        if (p.n_levels > 1) {
-            __threadfence();
-            __syncwarp();
-            if (lane == 0) atomicAdd(&ctrl->done, 1u);
-        }
+        if (p.n_levels > 1) ++my_done;
         g = g_next;
+    }
+    if (my_done) {
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) atomicAdd(&ctrl->done, my_done);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// the persistent walker, bulk-copy ring (single-level bit-copy tables)
+// ---------------------------------------------------------------------------------------------------
+//
+// Shared memory: n_stages x stage_bytes of data, then per stage one "full" mbarrier (1 arrival + the
+// bytes the bulk loads deliver), one "empty" mbarrier (32 arrivals: the consumer lanes) and the tile's
+// destination record.  Data never passes through registers.
+
+struct StageMeta {
+    char*    d;
+    uint32_t nr, w, dp, end;
+};
+
+constexpr uint32_t kBulkMaxStages = 28;
+constexpr uint32_t kBulkPiece     = 4096;       // contiguous tiles are issued in pieces of this many bytes
+constexpr uint32_t kClaimBatch    = 4;          // consecutive tiles per claim of the ring's producer
+constexpr uint32_t kBulkLag       = 2;          // stages whose stores may still be reading shared memory
+constexpr uint32_t kBarrierTries  = 1u << 22;   // try_wait attempts before a wait gives up
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Bounded wait for the phase with the given parity; false when it gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kBarrierTries; ++i) {
+        uint32_t ok;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                     "selp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst_smem, const char* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void bulk_store(char* dst, uint32_t src_smem, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 ::"l"(dst), "r"(src_smem), "r"(bytes) : "memory");
+}
+
+__global__ void __launch_bounds__(64, 2) nereus_walk_bulk(const __grid_constant__ WalkParams p,
+                                                          const uint32_t stage_bytes, const uint32_t n_stages) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    uint64_t*  full  = reinterpret_cast<uint64_t*>(smem + (size_t)stage_bytes * n_stages);
+    uint64_t*  empty = full + n_stages;
+    StageMeta* meta  = reinterpret_cast<StageMeta*>(empty + n_stages);
+    const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    Ctrl* const    ctrl = p.ctrl;
+
+    if (threadIdx.x == 0) {
+        for (uint32_t i = 0; i < n_stages; ++i) {
+            mbar_init(smem_addr(full + i), 1);
+            mbar_init(smem_addr(empty + i), 32);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    if (warp == 0) {
+        // ---------------- producer: claim kClaimBatch consecutive tiles at a time, resolve, load into the ring
+        uint32_t  stage = 0, phase = 0;
+        RectRange rr;
+        uint32_t  g0 = claim_tiles(ctrl, lane, kClaimBatch);
+        bool      running = true;
+        while (running) {
+            const bool     last    = g0 >= p.n_tiles;
+            const uint32_t g0_next = last ? g0 : claim_tiles(ctrl, lane, kClaimBatch);   // hidden behind this batch
+            for (uint32_t g = g0; running && g < g0 + kClaimBatch; ++g) {
+                const bool end = g >= p.n_tiles;
+                Tile t;
+                bool ok = true;
+                if (!end) {
+                    ok = resolve_tile<true>(p, g, rr, t) && t.level == 0 && t.cast == 0 &&
+                         (uint64_t)t.nr * t.w <= stage_bytes;
+                    if (!ok && lane == 0) raise_status(ctrl, NEREUS_DEV_BOUNDS, g);
+                }
+                // the stage is free once the consumer's stores of its previous use have read it
+                bool freed = true;
+                if (lane == 0) freed = mbar_wait(smem_addr(empty + stage), phase ^ 1);
+                freed = __shfl_sync(0xffffffffu, freed, 0);
+                if (!freed) {
+                    if (lane == 0) raise_status(ctrl, NEREUS_DEV_TIMEOUT, g);
+                    running = false;
+                    break;
+                }
+                if (end || !ok) {
+                    if (lane == 0) {
+                        meta[stage].end = 1;
+                        mbar_arrive(smem_addr(full + stage));
+                    }
+                    running = false;
+                    break;
+                }
+                const uint32_t base = smem_addr(smem + (size_t)stage * stage_bytes);
+                const uint32_t bar  = smem_addr(full + stage);
+                if (lane == 0) {
+                    meta[stage].d = t.d; meta[stage].nr = t.nr; meta[stage].w = t.w; meta[stage].dp = t.dp;
+                    meta[stage].end = 0;
+                    mbar_arrive_expect_tx(bar, t.nr * t.w);
+                }
+                __syncwarp();
+                if (t.nr == 1) {
+                    for (uint32_t off = lane * kBulkPiece; off < t.w; off += 32 * kBulkPiece)
+                        bulk_load(base + off, t.s + off, min(kBulkPiece, t.w - off), bar);
+                } else {
+                    for (uint32_t r = lane; r < t.nr; r += 32)
+                        bulk_load(base + r * t.w, t.s + (size_t)r * t.sp, t.w, bar);
+                }
+                if (++stage == n_stages) { stage = 0; phase ^= 1; }
+            }
+            g0 = g0_next;
+        }
+    } else {
+        // ---------------- consumer: store full stages, hand them back kBulkLag stages later
+        uint32_t stage = 0, phase = 0, issued = 0;
+        while (true) {
+            bool ready = true;
+            if (lane == 0) ready = mbar_wait(smem_addr(full + stage), phase);
+            ready = __shfl_sync(0xffffffffu, ready, 0);
+            if (!ready) {
+                if (lane == 0) raise_status(ctrl, NEREUS_DEV_TIMEOUT, 0xFFFFFFFFu);
+                break;
+            }
+            const StageMeta m = meta[stage];
+            if (m.end) break;
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            const uint32_t base = smem_addr(smem + (size_t)stage * stage_bytes);
+            if (m.nr == 1) {
+                for (uint32_t off = lane * kBulkPiece; off < m.w; off += 32 * kBulkPiece)
+                    bulk_store(m.d + off, base + off, min(kBulkPiece, m.w - off));
+            } else {
+                for (uint32_t r = lane; r < m.nr; r += 32)
+                    bulk_store(m.d + (size_t)r * m.dp, base + r * m.w, m.w);
+            }
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            ++issued;
+            if (issued > kBulkLag) {
+                // all but the kBulkLag newest groups of this lane have finished reading shared memory
+                asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kBulkLag) : "memory");
+                const uint32_t rel = (stage + n_stages - kBulkLag) % n_stages;
+                mbar_arrive(smem_addr(empty + rel));
+            }
+            if (++stage == n_stages) { stage = 0; phase ^= 1; }
+        }
+        // shared memory must outlive the stores that read it
+        asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
 }
 
@@ -270,6 +488,69 @@ static int env_int(const char* name, int dflt) {
     return (v && *v) ? atoi(v) : dflt;
 }
 
+// Launch shape of one run, from the handle's tuning, the environment and the table.
+struct Launch {
+    int      variant = 1;           // 1 vector copy, 2 bulk-copy ring
+    int      tile_bytes = 0, ctas_per_sm = 0, threads = 0;
+    uint32_t n_stages = 0;          // bulk ring
+    size_t   smem = 0;
+};
+
+static bool bulk_eligible(const nereus_transition_s& t) {
+    if (t.n_levels != 1) return false;
+    for (const Rect& r : t.rects)
+        if (r.cast) return false;
+    return true;
+}
+
+static int resolve_launch(const nereus_transition_s& t, int sms, Launch& L) {
+    const int want = t.tuning.variant ? t.tuning.variant : env_int("NEREUS_VARIANT", 0);
+    const int asked_tile = t.tuning.tile_bytes ? t.tuning.tile_bytes : env_int("NEREUS_TILE_BYTES", 0);
+    // default: the ring for large single-level bit-copy tables (its per-CTA start-up costs more than it gains
+    // below a few tens of MB), the vector kernel for everything else
+    if (want == 2)      L.variant = bulk_eligible(t) ? 2 : 1;
+    else if (want == 1) L.variant = 1;
+    else                L.variant = (bulk_eligible(t) && t.bytes_written >= (64ull << 20) && asked_tile <= 49152) ? 2 : 1;
+    L.ctas_per_sm = t.tuning.ctas_per_sm ? t.tuning.ctas_per_sm : env_int("NEREUS_CTAS_PER_SM", 2);
+    L.threads     = t.tuning.threads     ? t.tuning.threads     : env_int("NEREUS_THREADS", 512);
+    L.tile_bytes  = t.tuning.tile_bytes  ? t.tuning.tile_bytes  : env_int("NEREUS_TILE_BYTES", 0);
+    if (L.variant == 2) { L.ctas_per_sm = t.tuning.ctas_per_sm ? t.tuning.ctas_per_sm : 1; L.threads = 64; }
+    if (L.ctas_per_sm < 1 || L.ctas_per_sm > 2 || L.threads < 32 || L.threads > 512 || L.threads % 32)
+        return NEREUS_ERR_ARG;
+    if (L.tile_bytes == 0) {
+        // default: 16 KiB per warp tile (32 KiB per ring stage); smaller tiles for small tables, so that every
+        // claimer still gets a few tiles
+        L.tile_bytes = L.variant == 2 ? 32768 : 16384;
+        const uint64_t claimers = (uint64_t)sms * L.ctas_per_sm * (L.variant == 2 ? 8 : L.threads / 32);
+        while (L.tile_bytes > 1024 && t.bytes_written / L.tile_bytes < 4 * claimers) L.tile_bytes /= 2;
+    }
+    if (L.tile_bytes < 512 || L.tile_bytes % 512) return NEREUS_ERR_ARG;
+    if (L.variant == 2) {
+        const size_t budget = (227 * 1024) / L.ctas_per_sm - 1024;          // per CTA
+        if ((size_t)L.tile_bytes > budget / 4) return NEREUS_ERR_ARG;
+        const size_t per_stage = (size_t)L.tile_bytes + 2 * sizeof(uint64_t) + sizeof(StageMeta);
+        L.n_stages = (uint32_t)std::min<size_t>(kBulkMaxStages, budget / per_stage);
+        L.smem = L.n_stages * per_stage;
+    }
+    return NEREUS_OK;
+}
+
+static int launch_walk(const Launch& L, int sms, const WalkParams& p, cudaStream_t stream) {
+    if (p.n_tiles == 0) return NEREUS_OK;
+    if (L.variant == 2) {
+        NEREUS_CUDA(cudaFuncSetAttribute(nereus_walk_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.smem));
+        const unsigned grid = std::max(1u, std::min((unsigned)(sms * L.ctas_per_sm), p.n_tiles));
+        nereus_walk_bulk<<<grid, 64, L.smem, stream>>>(p, (uint32_t)L.tile_bytes, L.n_stages);
+    } else {
+        const unsigned warps_per_cta = (unsigned)L.threads / 32;
+        unsigned grid = (unsigned)(sms * L.ctas_per_sm);
+        grid = std::max(1u, std::min(grid, (p.n_tiles + warps_per_cta - 1) / warps_per_cta));
+        nereus_walk_vec<<<grid, L.threads, 0, stream>>>(p);
+    }
+    NEREUS_CUDA(cudaGetLastError());
+    return NEREUS_OK;
+}
+
 static int prepare(nereus_transition_s& t) {
     int device = 0;
     NEREUS_CUDA(cudaGetDevice(&device));
@@ -278,17 +559,13 @@ static int prepare(nereus_transition_s& t) {
 
     int sms = 0;
     NEREUS_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
+    Launch L;
+    if (int rc = resolve_launch(t, sms, L)) return rc;
 
     DeviceTable dv;
     dv.device = device;
     dv.sm_count = sms;
-    dv.tile_bytes  = t.tuning.tile_bytes  ? t.tuning.tile_bytes  : env_int("NEREUS_TILE_BYTES", 16384);
-    dv.ctas_per_sm = t.tuning.ctas_per_sm ? t.tuning.ctas_per_sm : env_int("NEREUS_CTAS_PER_SM", 2);
-    dv.threads     = t.tuning.threads     ? t.tuning.threads     : env_int("NEREUS_THREADS", 512);
-    dv.variant     = t.tuning.variant     ? t.tuning.variant     : env_int("NEREUS_VARIANT", 1);
-    if (dv.tile_bytes < 512 || dv.tile_bytes % 512 || dv.ctas_per_sm < 1 || dv.ctas_per_sm > 2 ||
-        dv.threads < 32 || dv.threads > 512 || dv.threads % 32)
-        return NEREUS_ERR_ARG;
+    dv.tile_bytes = L.tile_bytes; dv.ctas_per_sm = L.ctas_per_sm; dv.threads = L.threads; dv.variant = L.variant;
 
     std::vector<RectDev>  rects;
     std::vector<uint32_t> first;
@@ -310,6 +587,16 @@ static int prepare(nereus_transition_s& t) {
     if (e != cudaSuccess) { cudaFree(base); set_cuda_error((int)e); (void)cudaGetLastError(); return NEREUS_ERR_CUDA; }
     t.dev = dv;
     return NEREUS_OK;
+}
+
+static void fill_params(const nereus_transition_s& t, const void* const* src_ptrs, void* const* dst_ptrs,
+                        WalkParams& p) {
+    p.n_rects = (uint32_t)t.rects.size();
+    p.n_levels = (uint32_t)t.n_levels;
+    const size_t ns = t.src_bytes.size(), nd = t.dst_bytes.size();
+    for (size_t i = 0; i < ns; ++i) p.bufs[i] = (char*)const_cast<void*>(src_ptrs[i]);
+    for (size_t j = 0; j < nd; ++j) p.bufs[ns + j] = (char*)dst_ptrs[j];
+    for (size_t k = ns + nd; k < (size_t)kMaxBuffers; ++k) p.bufs[k] = nullptr;
 }
 
 static bool overlap(const char* a, uint64_t na, const char* b, uint64_t nb) {
@@ -349,7 +636,7 @@ static int check_buffers(const nereus_transition_s& t, const void* const* src, v
 extern "C" {
 
 int nereus_transition_tune(nereus_transition_t t, int tile_bytes, int ctas_per_sm, int threads, int variant) {
-    if (!t || tile_bytes < 0 || ctas_per_sm < 0 || threads < 0 || variant < 0) return NEREUS_ERR_ARG;
+    if (!t || tile_bytes < 0 || ctas_per_sm < 0 || threads < 0 || variant < 0 || variant > 2) return NEREUS_ERR_ARG;
     if (tile_bytes && (tile_bytes < 512 || tile_bytes % 512)) return NEREUS_ERR_ARG;
     if (ctas_per_sm > 2 || threads > 512 || threads % 32) return NEREUS_ERR_ARG;
     t->tuning.tile_bytes = tile_bytes; t->tuning.ctas_per_sm = ctas_per_sm;
@@ -362,12 +649,26 @@ int nereus_transition_num_tiles(nereus_transition_t t, uint64_t* tiles, int* lev
     try {
         if (!t || !tiles || !levels) return NEREUS_ERR_ARG;
         std::vector<RectDev> rects; std::vector<uint32_t> first; uint32_t le[kMaxLevels];
-        const int tb = t->dev.rects ? t->dev.tile_bytes
-                                    : (t->tuning.tile_bytes ? t->tuning.tile_bytes : env_int("NEREUS_TILE_BYTES", 16384));
+        int tb = t->dev.tile_bytes;
+        if (!t->dev.rects) {                      // not prepared: what a 148-SM device would get
+            Launch L;
+            if (int rc = resolve_launch(*t, 148, L)) return rc;
+            tb = L.tile_bytes;
+        }
         *tiles = tile_table(*t, (uint32_t)tb, rects, first, le);
         *levels = t->n_levels;
         return NEREUS_OK;
     } catch (const std::bad_alloc&) { return NEREUS_ERR_NOMEM; }
+}
+
+int nereus_transition_launch_info(nereus_transition_t t, int* variant, int* tile_bytes, int* grid, int* threads) {
+    if (!t || !variant || !tile_bytes || !grid || !threads) return NEREUS_ERR_ARG;
+    const int sms = t->dev.rects ? t->dev.sm_count : 148;
+    Launch L;
+    if (int rc = resolve_launch(*t, sms, L)) return rc;
+    if (t->dev.rects) L.tile_bytes = t->dev.tile_bytes;
+    *variant = L.variant; *tile_bytes = L.tile_bytes; *grid = sms * L.ctas_per_sm; *threads = L.threads;
+    return NEREUS_OK;
 }
 
 int nereus_transition_prepare(nereus_transition_t t) {
@@ -386,25 +687,18 @@ int nereus_transition_run(nereus_transition_t t, const void* const* src_ptrs, vo
         const DeviceTable& dv = t->dev;
         cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
 
+        Launch L;
+        if (int rc = resolve_launch(*t, dv.sm_count, L)) return rc;
+        L.tile_bytes = dv.tile_bytes;
         WalkParams p;
         p.rects = dv.rects; p.first = dv.first; p.ctrl = dv.ctrl;
-        p.n_rects = (uint32_t)t->rects.size(); p.n_tiles = dv.n_tiles; p.n_levels = (uint32_t)t->n_levels;
+        p.n_tiles = dv.n_tiles;
         for (int k = 0; k < kMaxLevels; ++k) p.level_end[k] = dv.level_end[k];
-        const size_t ns = t->src_bytes.size(), nd = t->dst_bytes.size();
-        for (size_t i = 0; i < ns; ++i) p.bufs[i] = (char*)const_cast<void*>(src_ptrs[i]);
-        for (size_t j = 0; j < nd; ++j) p.bufs[ns + j] = (char*)dst_ptrs[j];
-        for (size_t k = ns + nd; k < (size_t)kMaxBuffers; ++k) p.bufs[k] = nullptr;
+        fill_params(*t, src_ptrs, dst_ptrs, p);
 
         NEREUS_CUDA(cudaMemsetAsync(dv.ctrl, 0, sizeof(Ctrl), stream));
-        if (dv.n_tiles > 0) {
-            const unsigned warps_needed = dv.n_tiles;
-            unsigned grid = (unsigned)(dv.sm_count * dv.ctas_per_sm);
-            const unsigned warps_per_cta = (unsigned)dv.threads / 32;
-            grid = std::max(1u, std::min(grid, (warps_needed + warps_per_cta - 1) / warps_per_cta));
-            nereus_walk_vec<<<grid, dv.threads, 0, stream>>>(p);
-            NEREUS_CUDA(cudaGetLastError());
-            t->launches += 1;
-        }
+        if (int rc = launch_walk(L, dv.sm_count, p, stream)) return rc;
+        if (dv.n_tiles > 0) t->launches += 1;
         return NEREUS_OK;
     } catch (const std::bad_alloc&) { return NEREUS_ERR_NOMEM; }
 }
@@ -491,17 +785,13 @@ extern "C" int nereus_transition_run_static(nereus_transition_t t, const void* c
         if (int rc = static_scratch(device, &scratch, &sms)) return rc;
         cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
 
-        const int tile_bytes  = t->tuning.tile_bytes  ? t->tuning.tile_bytes  : env_int("NEREUS_TILE_BYTES", 16384);
-        const int ctas_per_sm = t->tuning.ctas_per_sm ? t->tuning.ctas_per_sm : env_int("NEREUS_CTAS_PER_SM", 2);
-        const int threads     = t->tuning.threads     ? t->tuning.threads     : env_int("NEREUS_THREADS", 512);
-        if (tile_bytes < 512 || tile_bytes % 512 || ctas_per_sm < 1 || ctas_per_sm > 2 || threads < 32 ||
-            threads > 512 || threads % 32)
-            return NEREUS_ERR_ARG;
+        Launch L;
+        if (int rc = resolve_launch(*t, sms, L)) return rc;
 
         WalkParams p;
         std::vector<RectDev>  rects;        // host memory only
         std::vector<uint32_t> first;
-        const uint64_t n_tiles = tile_table(*t, (uint32_t)tile_bytes, rects, first, p.level_end);
+        const uint64_t n_tiles = tile_table(*t, (uint32_t)L.tile_bytes, rects, first, p.level_end);
         if (n_tiles == 0 && !t->rects.empty()) return NEREUS_ERR_UNSUPPORTED;
 
         RectDev*  d_rects = reinterpret_cast<RectDev*>(scratch);
@@ -513,19 +803,10 @@ extern "C" int nereus_transition_run_static(nereus_transition_t t, const void* c
         NEREUS_CUDA(cudaMemsetAsync(d_ctrl, 0, sizeof(Ctrl), stream));
 
         p.rects = d_rects; p.first = d_first; p.ctrl = d_ctrl;
-        p.n_rects = (uint32_t)t->rects.size(); p.n_tiles = (uint32_t)n_tiles; p.n_levels = (uint32_t)t->n_levels;
-        const size_t ns = t->src_bytes.size(), nd = t->dst_bytes.size();
-        for (size_t i = 0; i < ns; ++i) p.bufs[i] = (char*)const_cast<void*>(src_ptrs[i]);
-        for (size_t j = 0; j < nd; ++j) p.bufs[ns + j] = (char*)dst_ptrs[j];
-        for (size_t k = ns + nd; k < (size_t)kMaxBuffers; ++k) p.bufs[k] = nullptr;
-        if (n_tiles > 0) {
-            const unsigned warps_per_cta = (unsigned)threads / 32;
-            unsigned grid = (unsigned)(sms * ctas_per_sm);
-            grid = std::max(1u, std::min(grid, ((unsigned)n_tiles + warps_per_cta - 1) / warps_per_cta));
-            nereus_walk_vec<<<grid, threads, 0, stream>>>(p);
-            NEREUS_CUDA(cudaGetLastError());
-            t->launches += 1;
-        }
+        p.n_tiles = (uint32_t)n_tiles;
+        fill_params(*t, src_ptrs, dst_ptrs, p);
+        if (int rc = launch_walk(L, sms, p, stream)) return rc;
+        if (n_tiles > 0) t->launches += 1;
         return NEREUS_OK;
     } catch (const std::bad_alloc&) { return NEREUS_ERR_NOMEM; }
 }

@@ -31,12 +31,29 @@ def test_small_plan_pairs_and_tile_sizes(tile):
     rng = np.random.default_rng(tile)
     pairs = [(pls[i], pls[j]) for i, j in rng.integers(0, len(pls), (6, 2))] + [((1, 1), (4, 2)), ((4, 2), (1, 1))]
     for a, b in pairs:
-        G.check_against_oracle(I.SMALL, a, b, seed=tile, tune=dict(tile_bytes=tile))
+        G.check_against_oracle(I.SMALL, a, b, seed=tile, tune=dict(tile_bytes=tile, variant=1))
+
+
+@pytest.mark.parametrize("tile", [512, 2048, 8192, 32768])
+def test_bulk_ring_kernel(tile):
+    """The bulk-copy ring (cp.async.bulk through shared memory) on the same plan pairs, incl. 16-byte pieces."""
+    tune = dict(tile_bytes=tile, variant=2)
+    for a, b in [((1, 1), (4, 2)), ((4, 2), (1, 1)), ((2, 4), (4, 1)), ((4, 4), (2, 2)), ((2, 1), (2, 1))]:
+        G.check_against_oracle(I.SMALL, a, b, seed=tile + 1, tune=tune)
+    G.check_against_oracle(I.SMALL, (2, 1), (4, 2), vh=True, seed=5, tune=tune)
+    G.check_against_oracle(I.SMALL, (1, 2), (4, 1), "fp32", "fp32", seed=3, tune=tune)
+    for a, b in [((4, 8), (8, 2)), ((8, 1), (1, 8))]:
+        G.check_against_oracle(I.MICRO, a, b, seed=9, tune=tune)
+    st = I.WORKLOADS["tiny_tp2pp1_to_tp1pp1"].stages[0]
+    G.check_against_oracle(st.shape, st.src[:2], st.dst[:2], seed=0, tune=tune)
+    # a cast or a chained table asks for the ring and silently gets the vector kernel
+    G.check_against_oracle(I.SMALL, (2, 2), (4, 1), "fp32", "bf16", seed=2, tune=tune)
 
 
 @pytest.mark.parametrize("threads,ctas", [(512, 2), (256, 1), (32, 1)])
 def test_launch_shapes(threads, ctas):
-    G.check_against_oracle(I.SMALL, (2, 2), (4, 1), seed=1, tune=dict(threads=threads, ctas_per_sm=ctas))
+    G.check_against_oracle(I.SMALL, (2, 2), (4, 1), seed=1, tune=dict(threads=threads, ctas_per_sm=ctas, variant=1))
+    G.check_against_oracle(I.SMALL, (2, 2), (4, 1), seed=1, tune=dict(ctas_per_sm=ctas, variant=2))
 
 
 def test_micro_paper_example_and_tp8():

@@ -34,7 +34,8 @@ DEFAULT_WORKLOAD = "8b_tp1pp1_to_tp4pp2"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic bytes of one nereus_walk launch, from the ncu
-# capture on the 4-layer 8B stand-in summarised in profiles/nereus_walk_vec__8b_split.md; traffic grows in
+# captures on the 4-layer 8B stand-in summarised in profiles/nereus_walk_bulk__8b_split.md and
+# profiles/nereus_walk_vec__8b_split.md (both kernels: 0.993); traffic grows in
 # proportion to the bytes moved (same tensor classes and piece sizes), so a full launch is scaled by it.
 NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 0.993
 
@@ -249,6 +250,19 @@ def run_reference(args):
 
 # ------------------------------------------------------------------------------------------------ ours
 
+def aggregate_over_ranks(total_ms, steps, bytes_per_step, world, device):
+    """Replicas only: every rank moved `bytes_per_step` per step; the job's time is the slowest rank's.
+    Returns (ms per step, GB/s summed over ranks)."""
+    import torch
+    import torch.distributed as dist
+
+    tm = torch.tensor([total_ms], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+    ms_per_step = float(tm.item()) / steps
+    return ms_per_step, world * bytes_per_step / 1e9 / (ms_per_step / 1e3)
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -302,12 +316,7 @@ def run_ours(args):
     clocks = sampler.stop() if rank == 0 else None
     assert t.status() == B.DEV_OK
 
-    tm = torch.tensor([total_ms], dtype=torch.float64, device=device)
-    if world > 1:
-        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-    total_ms_max = float(tm.item())
-    ms_per_step = total_ms_max / args.steps
-    value = world * (rd + wr) / 1e9 / (ms_per_step / 1e3)
+    ms_per_step, value = aggregate_over_ranks(total_ms, args.steps, rd + wr, world, device)
 
     # end to end: host buffers in, host buffers out, copies inside the timed region
     e2e = None

@@ -308,7 +308,7 @@ __global__ void __launch_bounds__(512, 2) nereus_walk_vec(const __grid_constant_
 }
 
 // ---------------------------------------------------------------------------------------------------
-// the persistent walker, bulk-copy ring (single-level bit-copy tables)
+// the persistent walker, bulk-copy ring (bit-copy tables)
 // ---------------------------------------------------------------------------------------------------
 //
 // Shared memory: n_stages x stage_bytes of data, then per stage one "full" mbarrier (1 arrival + the
@@ -317,8 +317,10 @@ __global__ void __launch_bounds__(512, 2) nereus_walk_vec(const __grid_constant_
 
 struct StageMeta {
     char*    d;
-    uint32_t nr, w, dp, end;
+    uint32_t nr, w, dp;
+    uint32_t kind;          // kStageData, kStageEnd or kStageFlush
 };
+constexpr uint32_t kStageData = 0, kStageEnd = 1, kStageFlush = 2;
 
 constexpr uint32_t kBulkMaxStages = 28;
 constexpr uint32_t kBulkPiece     = 4096;       // contiguous tiles are issued in pieces of this many bytes
@@ -377,7 +379,7 @@ __global__ void __launch_bounds__(64, 2) nereus_walk_bulk(const __grid_constant_
 
     if (warp == 0) {
         // ---------------- producer: claim kClaimBatch consecutive tiles at a time, resolve, load into the ring
-        uint32_t  stage = 0, phase = 0;
+        uint32_t  stage = 0, phase = 0, level = 0;
         RectRange rr;
         uint32_t  g0 = claim_tiles(ctrl, lane, kClaimBatch);
         bool      running = true;
@@ -389,49 +391,78 @@ __global__ void __launch_bounds__(64, 2) nereus_walk_bulk(const __grid_constant_
                 Tile t;
                 bool ok = true;
                 if (!end) {
-                    ok = resolve_tile<true>(p, g, rr, t) && t.level == 0 && t.cast == 0 &&
-                         (uint64_t)t.nr * t.w <= stage_bytes;
+                    ok = resolve_tile<true>(p, g, rr, t) && t.cast == 0 && (uint64_t)t.nr * t.w <= stage_bytes;
                     if (!ok && lane == 0) raise_status(ctrl, NEREUS_DEV_BOUNDS, g);
                 }
-                // the stage is free once the consumer's stores of its previous use have read it
-                bool freed = true;
-                if (lane == 0) freed = mbar_wait(smem_addr(empty + stage), phase ^ 1);
-                freed = __shfl_sync(0xffffffffu, freed, 0);
-                if (!freed) {
-                    if (lane == 0) raise_status(ctrl, NEREUS_DEV_TIMEOUT, g);
-                    running = false;
-                    break;
-                }
-                if (end || !ok) {
-                    if (lane == 0) {
-                        meta[stage].end = 1;
-                        mbar_arrive(smem_addr(full + stage));
+                // a tile of a higher level: first have the consumer publish this CTA's finished tiles (a flush
+                // stage), only then wait for the level below to be complete everywhere
+                const bool climb = !end && ok && t.level > level;
+                for (int pass = climb ? 0 : 1; running && pass < 2; ++pass) {
+                    // the stage is free once the consumer's stores of its previous use have read it
+                    bool freed = true;
+                    if (lane == 0) freed = mbar_wait(smem_addr(empty + stage), phase ^ 1);
+                    freed = __shfl_sync(0xffffffffu, freed, 0);
+                    if (!freed) {
+                        if (lane == 0) raise_status(ctrl, NEREUS_DEV_TIMEOUT, g);
+                        running = false;
+                        break;
                     }
-                    running = false;
-                    break;
+                    const uint32_t base = smem_addr(smem + (size_t)stage * stage_bytes);
+                    const uint32_t bar  = smem_addr(full + stage);
+                    if (pass == 0) {
+                        if (lane == 0) {
+                            meta[stage].kind = kStageFlush;
+                            mbar_arrive(bar);
+                        }
+                        if (++stage == n_stages) { stage = 0; phase ^= 1; }
+                        // dependency gate, bounded
+                        bool open = true;
+                        if (lane == 0) {
+                            const uint32_t need = p.level_end[t.level - 1];
+                            uint32_t polls = 0;
+                            while (ld_acquire_u32(&ctrl->done) < need) {
+                                if (++polls > kGatePolls) { open = false; break; }
+                                __nanosleep(200);
+                            }
+                            if (!open) raise_status(ctrl, NEREUS_DEV_TIMEOUT, g);
+                        }
+                        open = __shfl_sync(0xffffffffu, open, 0);
+                        if (!open) { ok = false; }
+                        // what other SMs wrote (through the async proxy, published after a proxy fence) is read
+                        // below through the async proxy again
+                        asm volatile("fence.proxy.async.global;" ::: "memory");
+                        level = t.level;
+                        continue;
+                    }
+                    if (end || !ok) {
+                        if (lane == 0) {
+                            meta[stage].kind = kStageEnd;
+                            mbar_arrive(bar);
+                        }
+                        running = false;
+                        break;
+                    }
+                    if (lane == 0) {
+                        meta[stage].d = t.d; meta[stage].nr = t.nr; meta[stage].w = t.w; meta[stage].dp = t.dp;
+                        meta[stage].kind = kStageData;
+                        mbar_arrive_expect_tx(bar, t.nr * t.w);
+                    }
+                    __syncwarp();
+                    if (t.nr == 1) {
+                        for (uint32_t off = lane * kBulkPiece; off < t.w; off += 32 * kBulkPiece)
+                            bulk_load(base + off, t.s + off, min(kBulkPiece, t.w - off), bar);
+                    } else {
+                        for (uint32_t r = lane; r < t.nr; r += 32)
+                            bulk_load(base + r * t.w, t.s + (size_t)r * t.sp, t.w, bar);
+                    }
+                    if (++stage == n_stages) { stage = 0; phase ^= 1; }
                 }
-                const uint32_t base = smem_addr(smem + (size_t)stage * stage_bytes);
-                const uint32_t bar  = smem_addr(full + stage);
-                if (lane == 0) {
-                    meta[stage].d = t.d; meta[stage].nr = t.nr; meta[stage].w = t.w; meta[stage].dp = t.dp;
-                    meta[stage].end = 0;
-                    mbar_arrive_expect_tx(bar, t.nr * t.w);
-                }
-                __syncwarp();
-                if (t.nr == 1) {
-                    for (uint32_t off = lane * kBulkPiece; off < t.w; off += 32 * kBulkPiece)
-                        bulk_load(base + off, t.s + off, min(kBulkPiece, t.w - off), bar);
-                } else {
-                    for (uint32_t r = lane; r < t.nr; r += 32)
-                        bulk_load(base + r * t.w, t.s + (size_t)r * t.sp, t.w, bar);
-                }
-                if (++stage == n_stages) { stage = 0; phase ^= 1; }
             }
             g0 = g0_next;
         }
     } else {
         // ---------------- consumer: store full stages, hand them back kBulkLag stages later
-        uint32_t stage = 0, phase = 0, issued = 0;
+        uint32_t stage = 0, phase = 0, issued = 0, unpublished = 0;
         while (true) {
             bool ready = true;
             if (lane == 0) ready = mbar_wait(smem_addr(full + stage), phase);
@@ -441,17 +472,29 @@ __global__ void __launch_bounds__(64, 2) nereus_walk_bulk(const __grid_constant_
                 break;
             }
             const StageMeta m = meta[stage];
-            if (m.end) break;
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            const uint32_t base = smem_addr(smem + (size_t)stage * stage_bytes);
-            if (m.nr == 1) {
-                for (uint32_t off = lane * kBulkPiece; off < m.w; off += 32 * kBulkPiece)
-                    bulk_store(m.d + off, base + off, min(kBulkPiece, m.w - off));
+            if (m.kind == kStageEnd) break;
+            if (m.kind == kStageFlush) {
+                // this CTA leaves a level: all its stores must have landed and be visible device-wide before
+                // the tiles are counted as done
+                asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+                asm volatile("fence.proxy.async.global;" ::: "memory");
+                __threadfence();
+                __syncwarp();
+                if (lane == 0 && unpublished) atomicAdd(&ctrl->done, unpublished);
+                unpublished = 0;
             } else {
-                for (uint32_t r = lane; r < m.nr; r += 32)
-                    bulk_store(m.d + (size_t)r * m.dp, base + r * m.w, m.w);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                const uint32_t base = smem_addr(smem + (size_t)stage * stage_bytes);
+                if (m.nr == 1) {
+                    for (uint32_t off = lane * kBulkPiece; off < m.w; off += 32 * kBulkPiece)
+                        bulk_store(m.d + off, base + off, min(kBulkPiece, m.w - off));
+                } else {
+                    for (uint32_t r = lane; r < m.nr; r += 32)
+                        bulk_store(m.d + (size_t)r * m.dp, base + r * m.w, m.w);
+                }
+                ++unpublished;
             }
-            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");        // a flush commits an empty group
             ++issued;
             if (issued > kBulkLag) {
                 // all but the kBulkLag newest groups of this lane have finished reading shared memory
@@ -461,8 +504,14 @@ __global__ void __launch_bounds__(64, 2) nereus_walk_bulk(const __grid_constant_
             }
             if (++stage == n_stages) { stage = 0; phase ^= 1; }
         }
-        // shared memory must outlive the stores that read it
+        // shared memory must outlive the stores that read it; other CTAs may be waiting for this one's tiles
         asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        if (p.n_levels > 1 && unpublished) {
+            asm volatile("fence.proxy.async.global;" ::: "memory");
+            __threadfence();
+            __syncwarp();
+            if (lane == 0) atomicAdd(&ctrl->done, unpublished);
+        }
     }
 }
 
@@ -497,7 +546,6 @@ struct Launch {
 };
 
 static bool bulk_eligible(const nereus_transition_s& t) {
-    if (t.n_levels != 1) return false;
     for (const Rect& r : t.rects)
         if (r.cast) return false;
     return true;

@@ -127,8 +127,9 @@ def test_fused_independent_stages():
     assert t.launches() == 1
 
 
+@pytest.mark.parametrize("variant", [1, 2])
 @pytest.mark.parametrize("tile", [2048, 16384])
-def test_chained_round_trip_into_the_sources(tile):
+def test_chained_round_trip_into_the_sources(tile, variant):
     """A -> B -> A in one launch with dependency levels; the way back overwrites the original source
     buffers (poisoned by the test between checks), as the 32B round-trip workload does."""
     sh = I.SMALL
@@ -136,7 +137,7 @@ def test_chained_round_trip_into_the_sources(tile):
     a, b = (2, 4), (4, 1)
     ab, ba = d.compile(B.Plan(*a), B.Plan(*b)), d.compile(B.Plan(*b), B.Plan(*a))
     t = B.Transition.fuse([ab, ba], chained=True)
-    t.tune(tile_bytes=tile)
+    t.tune(tile_bytes=tile, variant=variant)
     src = G.device_sources(d, B.Plan(*a), "bf16", 8)
     keep = [s.cpu().numpy().copy() for s in src]
     mid = G.Guarded([t.buffer_bytes(True, j) for j in range(4)])
@@ -150,7 +151,7 @@ def test_chained_round_trip_into_the_sources(tile):
     assert mid.guards_intact()
     # three levels: A -> B -> A -> B into fresh buffers
     t3 = B.Transition.fuse([ab, ba, ab], chained=True)
-    t3.tune(tile_bytes=tile)
+    t3.tune(tile_bytes=tile, variant=variant)
     back = G.Guarded([t3.buffer_bytes(True, 4 + j) for j in range(8)])
     again = G.Guarded([t3.buffer_bytes(True, 12 + j) for j in range(4)])
     for m in mid.bufs:
@@ -158,6 +159,9 @@ def test_chained_round_trip_into_the_sources(tile):
     G.run_transition(t3, src, mid.bufs + back.bufs + again.bufs)
     for g, w in zip(again.bufs, mid_want):
         assert np.array_equal(g.cpu().numpy(), w)
+    back_fresh = O.reshard(G.omodel_of(sh), O.Plan(*b), O.Plan(*a), mid_want, fill=G.SENTINEL)
+    for g, w in zip(back.bufs, back_fresh):
+        assert np.array_equal(g.cpu().numpy(), w)           # level 1 really wrote its fresh buffers
     assert again.guards_intact() and back.guards_intact()
 
 

@@ -141,21 +141,33 @@ def build_workload(name, device, tune):
         d = B.ModelDesc(sh.layers, sh.hidden, sh.heads, sh.kv_heads, sh.ffn, sh.vocab, B.DTYPES[st.src[2]],
                         st.value_head)
         pa, pb = B.Plan(st.src[0], st.src[1], B.DTYPES[st.src[2]]), B.Plan(st.dst[0], st.dst[1], B.DTYPES[st.dst[2]])
-        t = d.compile(pa, pb)
-        s = I.make_shards(d.shard_sizes(pa), st.src[2], st.seed, device)
-        es = I.element_size(st.src[2])
-        groups = []
-        for tid in range(d.num_tensors()):
-            g = []
-            for k in range(d.num_shards(pa)):
-                off, rows, cols, rep = d.tensor_slice(pa, k, tid)
-                if rep and rows:
-                    g.append((k, off, rows * cols * es))
-            if len(g) > 1:
-                groups.append(g)
-        I.tie_replicas(s, groups)
-        srcs += s
-        dsts += I.sentinel_shards(d.shard_sizes(pb), device)
+        if st.replicas > 1:
+            t = d.compile_replicated(pa, pb, st.replicas)
+        elif st.n_opt:
+            t = d.compile_state(pa, pb, st.n_opt)
+        else:
+            t = d.compile(pa, pb)
+
+        def tied_sources(plan, dtype, seed):
+            s = I.make_shards(d.shard_sizes(plan), dtype, seed, device)
+            es = I.element_size(dtype)
+            groups = []
+            for tid in range(d.num_tensors()):
+                g = []
+                for k in range(d.num_shards(plan)):
+                    off, rows, cols, rep = d.tensor_slice(plan, k, tid)
+                    if rep and rows:
+                        g.append((k, off, rows * cols * es))
+                if len(g) > 1:
+                    groups.append(g)
+            I.tie_replicas(s, groups)
+            return s
+
+        srcs += tied_sources(pa, st.src[2], st.seed)
+        for k in range(st.n_opt):                      # optimizer tensors: fp32, same (tp, pp)
+            srcs += tied_sources(B.Plan(pa.tp, pa.pp, B.FP32), "fp32", st.seed * 101 + k)
+        n_dst = t.num_buffers()[1]
+        dsts += I.sentinel_shards([t.buffer_bytes(True, j) for j in range(n_dst)], device)
         parts.append(t)
         descs.append((d, pa, pb))
         keep.append(d)

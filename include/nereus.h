@@ -93,6 +93,8 @@ typedef struct {
     uint64_t src_pitch, dst_pitch;  /* bytes between consecutive pieces */
     uint64_t rows;
     uint64_t width_bytes_src, width_bytes_dst;
+    int32_t  replicas;              /* the piece is written `replicas` times: to buffers dst_buf + j*replica_stride */
+    int32_t  replica_stride;
 } nereus_rect_t;
 
 /* ---- model descriptor (EMU field M and the shapes of theta; Section 5) -------------------------------- */
@@ -128,6 +130,20 @@ int nereus_plan_tensor_slice(nereus_model_desc_t desc, nereus_plan_t plan, int s
  * Errors: ARG, INDIVISIBLE, UNSUPPORTED (dtype pair; tp > kv_heads), NOMEM. */
 int nereus_transition_compile(nereus_model_desc_t desc, nereus_plan_t src, nereus_plan_t dst,
                               nereus_transition_t* out);
+/* Same, with `replicas` identical destination units (1..16): every source byte is read once and written
+ * `replicas` times.  This is the data movement of Extend (Section 5.2(c): replicate a unit onto new GPUs,
+ * rank-aligned, each shard sent once; use src == dst) and of a Split that yields k replica units (Section
+ * 5.2(a)).  run() takes replicas * tp*pp destination pointers, replica-major: unit 0's shards, unit 1's, ...
+ * Errors: as nereus_transition_compile, plus ARG (replicas out of range). */
+int nereus_transition_compile_replicated(nereus_model_desc_t desc, nereus_plan_t src, nereus_plan_t dst,
+                                         int replicas, nereus_transition_t* out);
+/* The EMU's full state (theta, omega) in one table: the parameters src -> dst as above, plus `n_opt`
+ * optimizer tensors per parameter (Adam: 2), held in fp32 and following the same layout (Section 5: "optimizer
+ * shards omega follow the same layout").  run() takes, on either side, the parameter shards followed by the
+ * shards of optimizer tensor 0, then of tensor 1, ...; optimizer shards have the sizes of an fp32 plan with
+ * the same tp and pp.  Optimizer state is never cast.  Errors: as nereus_transition_compile, ARG (n_opt < 0). */
+int nereus_transition_compile_state(nereus_model_desc_t desc, nereus_plan_t src, nereus_plan_t dst, int n_opt,
+                                    nereus_transition_t* out);
 /* Fuses n compiled transitions into one task table that one launch executes (Section 6.2: ready primitives
  * run concurrently; a primitive is ready only after its predecessors complete).
  *   chained = 0: the parts are independent model-stages.  run() takes the concatenation of the parts'

@@ -360,3 +360,17 @@ int oracle_reshard(const oracle_model* m, oracle_plan sp, oracle_plan dp,
         if ((rc = oracle_reshard_tensor(m, sp, dp, id, src_bufs, dst_bufs))) return rc;
     return ORACLE_OK;
 }
+
+/* k identical target units: what Extend leaves behind (Section 5.2(c): the new unit "holds replicated copies"
+ * of theta and omega; use sp == dp) and what a Split into k replica units produces (Section 5.2(a)).  By
+ * definition every unit is the plain reshard, so the oracle runs it once per unit.
+ * dst_bufs is replica-major: unit 0's tp*pp shards, then unit 1's, ... */
+int oracle_reshard_replicated(const oracle_model* m, oracle_plan sp, oracle_plan dp, int replicas,
+                              const void* const* src_bufs, void* const* dst_bufs) {
+    int rc;
+    if (replicas < 1) return ORACLE_ERR_ARG;
+    if ((rc = oracle_check_plan(m, dp))) return rc;
+    for (int r = 0; r < replicas; ++r)
+        if ((rc = oracle_reshard(m, sp, dp, src_bufs, dst_bufs + (int64_t)r * dp.tp * dp.pp))) return rc;
+    return ORACLE_OK;
+}

@@ -110,6 +110,7 @@ def lib():
         L.oracle_reshard_tensor_parts.argtypes = [p(_Model), _Plan, _Plan, i64, pp_, pp_]
         L.oracle_reshard_tensor.argtypes = [p(_Model), _Plan, _Plan, i64, pp_, pp_]
         L.oracle_reshard.argtypes = [p(_Model), _Plan, _Plan, pp_, pp_]
+        L.oracle_reshard_replicated.argtypes = [p(_Model), _Plan, _Plan, ctypes.c_int, pp_, pp_]
         _lib = L
     return _lib
 
@@ -227,3 +228,28 @@ def reshard_tensor_parts(model: Model, src: Plan, dst: Plan, tid: int, src_parts
     m = model.c()
     _check(lib().oracle_reshard_tensor_parts(ctypes.byref(m), src.c(), dst.c(), tid, _ptr_array(src_parts),
                                              _ptr_array(dst_parts)), "reshard_tensor_parts")
+
+
+def reshard_replicated(model: Model, src: Plan, dst: Plan, replicas: int, src_bufs: list[np.ndarray],
+                       fill: int = 0) -> list[np.ndarray]:
+    """k identical target units (Extend; Split into k replica units), replica-major list of shard buffers."""
+    m = model.c()
+    dst_bufs = [b for _ in range(replicas) for b in new_shards(model, dst, fill)]
+    _check(lib().oracle_reshard_replicated(ctypes.byref(m), src.c(), dst.c(), replicas, _ptr_array(src_bufs),
+                                           _ptr_array(dst_bufs)), "reshard_replicated")
+    return dst_bufs
+
+
+def reshard_state(model: Model, src: Plan, dst: Plan, n_opt: int, src_bufs: list[np.ndarray],
+                  fill: int = 0) -> list[np.ndarray]:
+    """The EMU's state (theta, omega): the parameters src -> dst, and n_opt optimizer tensors per parameter that
+    "follow the same layout" (Section 5), held in fp32 on both sides and never cast.  Buffers on either side:
+    parameter shards, then the shards of optimizer tensor 0, then of tensor 1, ..."""
+    ns = num_shards(model, src)
+    out = reshard(model, src, dst, src_bufs[:ns], fill=fill)
+    m32 = Model(model.layers, model.hidden, model.heads, model.kv_heads, model.ffn, model.vocab, FP32,
+                model.value_head)
+    s32, d32 = Plan(src.tp, src.pp, FP32), Plan(dst.tp, dst.pp, FP32)
+    for k in range(n_opt):
+        out += reshard(m32, s32, d32, src_bufs[ns * (1 + k):ns * (2 + k)], fill=fill)
+    return out

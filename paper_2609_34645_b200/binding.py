@@ -54,7 +54,8 @@ class Rect(ctypes.Structure):
     _fields_ = [("src_buf", ctypes.c_int32), ("dst_buf", ctypes.c_int32), ("level", ctypes.c_int32),
                 ("cast", ctypes.c_int32), ("src_off", ctypes.c_uint64), ("dst_off", ctypes.c_uint64),
                 ("src_pitch", ctypes.c_uint64), ("dst_pitch", ctypes.c_uint64), ("rows", ctypes.c_uint64),
-                ("width_bytes_src", ctypes.c_uint64), ("width_bytes_dst", ctypes.c_uint64)]
+                ("width_bytes_src", ctypes.c_uint64), ("width_bytes_dst", ctypes.c_uint64),
+                ("replicas", ctypes.c_int32), ("replica_stride", ctypes.c_int32)]
 
 
 _vp, _i, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
@@ -69,6 +70,8 @@ _SIGS = {
     "nereus_model_num_tensors": [_vp, _P(_i)],
     "nereus_plan_tensor_slice": [_vp, Plan, _i, _i, _P(_sz), _P(_sz), _P(_sz), _P(_i)],
     "nereus_transition_compile": [_vp, Plan, Plan, _P(_vp)],
+    "nereus_transition_compile_replicated": [_vp, Plan, Plan, _i, _P(_vp)],
+    "nereus_transition_compile_state": [_vp, Plan, Plan, _i, _P(_vp)],
     "nereus_transition_fuse": [_P(_vp), _i, _i, _P(_vp)],
     "nereus_transition_destroy": [_vp],
     "nereus_transition_num_buffers": [_vp, _P(_i), _P(_i)],
@@ -144,6 +147,20 @@ class ModelDesc:
     def compile(self, src: Plan, dst: Plan) -> "Transition":
         h = _vp()
         _ck(_lib.nereus_transition_compile(self._h, src, dst, ctypes.byref(h)), "nereus_transition_compile")
+        return Transition(h)
+
+    def compile_replicated(self, src: Plan, dst: Plan, replicas: int) -> "Transition":
+        """k identical destination units, every source byte read once (Extend when src == dst)."""
+        h = _vp()
+        _ck(_lib.nereus_transition_compile_replicated(self._h, src, dst, replicas, ctypes.byref(h)),
+            "nereus_transition_compile_replicated")
+        return Transition(h)
+
+    def compile_state(self, src: Plan, dst: Plan, n_opt: int) -> "Transition":
+        """Parameters plus n_opt fp32 optimizer tensors per parameter, all in one table."""
+        h = _vp()
+        _ck(_lib.nereus_transition_compile_state(self._h, src, dst, n_opt, ctypes.byref(h)),
+            "nereus_transition_compile_state")
         return Transition(h)
 
     def close(self):

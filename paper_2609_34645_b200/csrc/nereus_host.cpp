@@ -111,7 +111,7 @@ struct Emitter {
         if (!out.empty()) {
             Rect& p = out.back();
             if (p.rows == 1 && r.rows == 1 && p.src_buf == r.src_buf && p.dst_buf == r.dst_buf &&
-                p.cast == r.cast && p.level == r.level &&
+                p.cast == r.cast && p.level == r.level && p.replicas == r.replicas &&
                 p.src_off + (p.width_dst << p.cast) == r.src_off && p.dst_off + p.width_dst == r.dst_off) {
                 p.width_dst += r.width_dst;
                 p.src_pitch = p.width_dst << p.cast;
@@ -125,11 +125,12 @@ struct Emitter {
 
 }  // namespace
 
-static int compile_one(const nereus_model_desc_s& d, nereus_plan_t sp, nereus_plan_t dp, nereus_transition_s& t) {
+static int compile_one(const nereus_model_desc_s& d, nereus_plan_t sp, nereus_plan_t dp, int replicas,
+                       nereus_transition_s& t) {
     const int      sdt = plan_dtype(d, sp), ddt = plan_dtype(d, dp);
     const uint64_t ses = elem_size(sdt), des = elem_size(ddt);
     const int      cast = (sdt != ddt) ? 1 : 0;
-    const int      n_src = sp.tp * sp.pp, n_dst = dp.tp * dp.pp;
+    const int      n_src = sp.tp * sp.pp, n_unit = dp.tp * dp.pp, n_dst = n_unit * replicas;
     if (n_src + n_dst > kMaxBuffers) return NEREUS_ERR_UNSUPPORTED;
 
     std::vector<StageLayout> sl(sp.pp), dl(dp.pp);
@@ -138,7 +139,7 @@ static int compile_one(const nereus_model_desc_s& d, nereus_plan_t sp, nereus_pl
     t.src_bytes.resize(n_src);
     t.dst_bytes.resize(n_dst);
     for (int i = 0; i < n_src; ++i) t.src_bytes[i] = sl[i / sp.tp].bytes;
-    for (int i = 0; i < n_dst; ++i) t.dst_bytes[i] = dl[i / dp.tp].bytes;
+    for (int i = 0; i < n_dst; ++i) t.dst_bytes[i] = dl[(i % n_unit) / dp.tp].bytes;
     t.dst_level.assign(n_dst, 0);
     t.dst_read_level.assign(n_dst, -1);
     t.n_levels = 1;
@@ -156,6 +157,7 @@ static int compile_one(const nereus_model_desc_s& d, nereus_plan_t sp, nereus_pl
                 const uint64_t soff = sl[ps].offset[id];
                 Rect r{};
                 r.dst_buf = dst_buf; r.level = 0; r.cast = cast;
+                r.replicas = replicas; r.replica_stride = replicas > 1 ? n_unit : 0;
                 if (x.cut == Cut::Whole) {
                     // replicated state: every copy is the same logical state; read TP rank 0's
                     r.src_buf = ps * ts;
@@ -211,7 +213,7 @@ static void finish(nereus_transition_s& t) {
     });
     t.bytes_read = t.bytes_written = 0;
     for (const Rect& r : t.rects) {
-        t.bytes_written += r.rows * r.width_dst;
+        t.bytes_written += r.rows * r.width_dst * (uint64_t)r.replicas;
         t.bytes_read += r.rows * (r.width_dst << r.cast);
     }
 }
@@ -229,6 +231,7 @@ uint64_t tile_table(const nereus_transition_s& t, uint32_t tile_bytes, std::vect
         q.rows = (uint32_t)r.rows;
         q.src_buf = (uint16_t)r.src_buf; q.dst_buf = (uint16_t)r.dst_buf;
         q.level = (uint16_t)r.level; q.cast = (uint16_t)r.cast;
+        q.replicas = (uint16_t)r.replicas; q.replica_stride = (uint16_t)r.replica_stride;
         uint64_t ntiles;
         if (r.rows == 1 || r.width_dst >= tile_bytes) {
             q.rows_per_tile = 1;
@@ -350,10 +353,42 @@ int nereus_transition_compile(nereus_model_desc_t d, nereus_plan_t sp, nereus_pl
     const int sdt = plan_dtype(*d, sp), ddt = plan_dtype(*d, dp);
     if (!(sdt == ddt || (sdt == NEREUS_FP32 && ddt == NEREUS_BF16))) return NEREUS_ERR_UNSUPPORTED;
     auto* t = new nereus_transition_s();
-    if (int rc = compile_one(*d, sp, dp, *t)) { delete t; return rc; }
+    if (int rc = compile_one(*d, sp, dp, 1, *t)) { delete t; return rc; }
     finish(*t);
     *out = t;
     return NEREUS_OK;
+    NEREUS_GUARD_END
+}
+
+int nereus_transition_compile_replicated(nereus_model_desc_t d, nereus_plan_t sp, nereus_plan_t dp, int replicas,
+                                         nereus_transition_t* out) {
+    NEREUS_GUARD_BEGIN
+    if (!d || !out || replicas < 1 || replicas > kMaxReplicas) return NEREUS_ERR_ARG;
+    if (int rc = check_plan(*d, sp)) return rc;
+    if (int rc = check_plan(*d, dp)) return rc;
+    const int sdt = plan_dtype(*d, sp), ddt = plan_dtype(*d, dp);
+    if (!(sdt == ddt || (sdt == NEREUS_FP32 && ddt == NEREUS_BF16))) return NEREUS_ERR_UNSUPPORTED;
+    auto* t = new nereus_transition_s();
+    if (int rc = compile_one(*d, sp, dp, replicas, *t)) { delete t; return rc; }
+    finish(*t);
+    *out = t;
+    return NEREUS_OK;
+    NEREUS_GUARD_END
+}
+
+int nereus_transition_compile_state(nereus_model_desc_t d, nereus_plan_t sp, nereus_plan_t dp, int n_opt,
+                                    nereus_transition_t* out) {
+    NEREUS_GUARD_BEGIN
+    if (!d || !out || n_opt < 0 || n_opt > 8) return NEREUS_ERR_ARG;
+    nereus_transition_t parts[9] = {nullptr};
+    int rc = nereus_transition_compile(d, sp, dp, &parts[0]);
+    nereus_plan_t so = sp, dO = dp;
+    so.dtype = NEREUS_FP32; dO.dtype = NEREUS_FP32;                 // omega: fp32 on both sides, same (tp, pp)
+    for (int k = 0; rc == NEREUS_OK && k < n_opt; ++k) rc = nereus_transition_compile(d, so, dO, &parts[1 + k]);
+    if (rc == NEREUS_OK) rc = nereus_transition_fuse(parts, 1 + n_opt, 0, out);
+    for (int k = 0; k < 9; ++k)
+        if (parts[k]) nereus_transition_destroy(parts[k]);
+    return rc;
     NEREUS_GUARD_END
 }
 
@@ -453,6 +488,7 @@ int nereus_transition_get_rect(nereus_transition_t t, int index, nereus_rect_t* 
     out->src_pitch = r.src_pitch; out->dst_pitch = r.dst_pitch;
     out->rows = r.rows;
     out->width_bytes_dst = r.width_dst; out->width_bytes_src = r.width_dst << r.cast;
+    out->replicas = r.replicas; out->replica_stride = r.replica_stride;
     return NEREUS_OK;
 }
 

@@ -73,6 +73,8 @@ struct Rect {
     uint64_t src_pitch, dst_pitch;
     uint64_t rows;
     uint64_t width_dst;
+    int32_t  replicas = 1;       // the piece is written to `replicas` buffers: dst_buf + j * replica_stride
+    int32_t  replica_stride = 0;
 };
 
 // Device form, 64 bytes.  A rect is cut into tiles of rows_per_tile rows x tile_w bytes (dst side);
@@ -87,7 +89,7 @@ struct alignas(16) RectDev {
     uint32_t first_tile;
     uint16_t src_buf, dst_buf;
     uint16_t level, cast;
-    uint32_t pad_;
+    uint16_t replicas, replica_stride;
 };
 static_assert(sizeof(RectDev) == 64, "RectDev must stay 64 bytes");
 
@@ -101,6 +103,7 @@ struct Ctrl {
 
 constexpr int kMaxBuffers = 448;      // pointers carried in the kernel's parameter block
 constexpr int kMaxLevels  = 8;
+constexpr int kMaxReplicas = 16;
 
 struct Tuning {
     int tile_bytes  = 0;

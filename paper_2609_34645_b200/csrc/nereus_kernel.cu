@@ -53,7 +53,8 @@ struct WalkParams {
 static_assert(sizeof(WalkParams) <= 4000, "kernel parameter block too large");
 
 constexpr int      kUnrollRun   = 8;            // 16-byte loads in flight per lane, contiguous runs
-constexpr int      kUnrollRect  = 8;            // ... pitched rects and the cast
+constexpr int      kUnrollRect  = 6;            // ... pitched rects (their index math needs registers)
+constexpr int      kUnrollCast  = 8;            // ... the cast
 constexpr uint32_t kGatePolls   = 1u << 21;     // x ~200 ns sleep: gives up after roughly half a second
 
 // ---------------------------------------------------------------------------------------------------
@@ -91,35 +92,44 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return r;
 }
 
+// The three tile bodies below load a batch of vectors once and store it to every destination replica
+// (`reps` is 1 except for replicated transitions); D(j) yields replica j's base pointer for the tile.
+
 // Bit copy of a contiguous run of `nvec` 16-byte vectors.
-template <int kUnroll>
-__device__ __forceinline__ void copy_run(const char* __restrict__ s, char* __restrict__ d, uint32_t nvec,
+template <int kUnroll, class Dst>
+__device__ __forceinline__ void copy_run(const char* __restrict__ s, Dst D, uint32_t reps, uint32_t nvec,
                                          unsigned lane) {
     s += lane * 16;
-    d += lane * 16;
+    uint32_t off = lane * 16;
     uint32_t left = nvec;
 #pragma unroll 1
     for (; left >= 32 * kUnroll; left -= 32 * kUnroll) {          // full batches: no predicates
         uint4 v[kUnroll];
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) v[u] = ld_stream(s + u * 512);
+#pragma unroll 1
+        for (uint32_t j = 0; j < reps; ++j) {
+            char* d = D(j) + off;
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) st_stream(d + u * 512, v[u]);
+            for (int u = 0; u < kUnroll; ++u) st_stream(d + u * 512, v[u]);
+        }
         s += 512 * kUnroll;
-        d += 512 * kUnroll;
+        off += 512 * kUnroll;
     }
 #pragma unroll 1
     for (uint32_t i = lane; i < left; i += 32) {                  // ragged tail, one vector at a time
-        st_stream(d, ld_stream(s));
+        const uint4 v = ld_stream(s);
+#pragma unroll 1
+        for (uint32_t j = 0; j < reps; ++j) st_stream(D(j) + off, v);
         s += 512;
-        d += 512;
+        off += 512;
     }
 }
 
 // Bit copy of a pitched tile: `rows` pieces of `vpr` 16-byte vectors each.  Offsets inside a tile fit
 // 32 bits (rows_per_tile x pitch is far below 4 GiB).
-template <int kUnroll>
-__device__ __forceinline__ void copy_rect(const char* __restrict__ s, char* __restrict__ d, uint32_t rows,
+template <int kUnroll, class Dst>
+__device__ __forceinline__ void copy_rect(const char* __restrict__ s, Dst D, uint32_t reps, uint32_t rows,
                                           uint32_t vpr, uint32_t sp, uint32_t dp, unsigned lane) {
     const uint32_t nvec = rows * vpr;
     uint32_t       base = lane;
@@ -134,13 +144,19 @@ __device__ __forceinline__ void copy_rect(const char* __restrict__ s, char* __re
             doff[u] = r * dp + c * 16;
             v[u] = ld_stream(s + (r * sp + c * 16));
         }
+#pragma unroll 1
+        for (uint32_t j = 0; j < reps; ++j) {
+            char* d = D(j);
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) st_stream(d + doff[u], v[u]);
+            for (int u = 0; u < kUnroll; ++u) st_stream(d + doff[u], v[u]);
+        }
     }
 #pragma unroll 1
     for (; base < nvec; base += 32) {                                  // ragged tail
         const uint32_t r = base / vpr, c = base - r * vpr;
-        st_stream(d + (r * dp + c * 16), ld_stream(s + (r * sp + c * 16)));
+        const uint4 v = ld_stream(s + (r * sp + c * 16));
+#pragma unroll 1
+        for (uint32_t j = 0; j < reps; ++j) st_stream(D(j) + (r * dp + c * 16), v);
     }
 }
 
@@ -153,29 +169,40 @@ __device__ __forceinline__ uint2 cast_unit(uint4 v) {
     return o;
 }
 
-template <int kUnroll>
-__device__ __forceinline__ void cast_tile(const char* __restrict__ s, char* __restrict__ d, uint32_t rows,
+template <int kUnroll, class Dst>
+__device__ __forceinline__ void cast_tile(const char* __restrict__ s, Dst D, uint32_t reps, uint32_t rows,
                                           uint32_t upr, uint32_t sp, uint32_t dp, unsigned lane) {
     const uint32_t nunit = rows * upr;
     uint32_t       base = lane;
 #pragma unroll 1
     for (; base + 32 * (kUnroll - 1) < nunit; base += 32 * kUnroll) {
-        uint4    v[kUnroll];
+        uint2    o[kUnroll];
         uint32_t doff[kUnroll];
+        {
+            uint4 v[kUnroll];
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-            const uint32_t idx = base + u * 32;
-            const uint32_t r = idx / upr, c = idx - r * upr;
-            doff[u] = r * dp + c * 8;
-            v[u] = ld_stream(s + (r * sp + c * 16));
+            for (int u = 0; u < kUnroll; ++u) {
+                const uint32_t idx = base + u * 32;
+                const uint32_t r = idx / upr, c = idx - r * upr;
+                doff[u] = r * dp + c * 8;
+                v[u] = ld_stream(s + (r * sp + c * 16));
+            }
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) o[u] = cast_unit(v[u]);
         }
+#pragma unroll 1
+        for (uint32_t j = 0; j < reps; ++j) {
+            char* d = D(j);
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) st_stream8(d + doff[u], cast_unit(v[u]));
+            for (int u = 0; u < kUnroll; ++u) st_stream8(d + doff[u], o[u]);
+        }
     }
 #pragma unroll 1
     for (; base < nunit; base += 32) {
         const uint32_t r = base / upr, c = base - r * upr;
-        st_stream8(d + (r * dp + c * 8), cast_unit(ld_stream(s + (r * sp + c * 16))));
+        const uint2 o = cast_unit(ld_stream(s + (r * sp + c * 16)));
+#pragma unroll 1
+        for (uint32_t j = 0; j < reps; ++j) st_stream8(D(j) + (r * dp + c * 8), o);
     }
 }
 
@@ -185,10 +212,17 @@ __device__ __forceinline__ void cast_tile(const char* __restrict__ s, char* __re
 
 struct Tile {
     const char* s;
-    char*       d;
+    uint64_t    d_off;             // byte offset of the tile inside each destination buffer
+    uint32_t    dst_buf, reps, rstride;   // destinations: bufs[dst_buf + j * rstride], j < reps
     uint32_t    nr, w, sp, dp;     // row pieces, dst bytes per piece, pitches
     uint32_t    level, cast;
 };
+
+// Destination j of a tile.  The pointer table lives in the kernel's parameter block (constant bank).
+__device__ __forceinline__ char* tile_dst(const WalkParams& p, uint32_t dst_buf, uint32_t rstride, uint64_t d_off,
+                                          uint32_t j) {
+    return p.bufs[dst_buf + j * rstride] + d_off;
+}
 
 // The rect a claimer resolved last: consecutive claims of one warp usually fall into the same rect (a rect
 // has thousands of tiles), so the binary search is skipped while first <= g < next_first.
@@ -224,7 +258,10 @@ __device__ __forceinline__ bool resolve_tile(const WalkParams& p, uint32_t g, Re
     const uint32_t src_buf = q3.y & 0xFFFFu, dst_buf = q3.y >> 16;
     t.sp = q1.z; t.dp = q1.w;
     t.level = q3.z & 0xFFFFu; t.cast = q3.z >> 16;
-    if (first_tile > g || src_buf >= (uint32_t)kMaxBuffers || dst_buf >= (uint32_t)kMaxBuffers || col_tiles == 0)
+    t.reps = q3.w & 0xFFFFu; t.rstride = q3.w >> 16;
+    t.dst_buf = dst_buf;
+    if (first_tile > g || src_buf >= (uint32_t)kMaxBuffers || col_tiles == 0 || t.reps == 0 ||
+        dst_buf + (t.reps - 1) * t.rstride >= (uint32_t)kMaxBuffers)
         return false;
     const uint32_t k  = g - first_tile;
     const uint32_t rb = k / col_tiles, cb = k - rb * col_tiles;
@@ -234,7 +271,7 @@ __device__ __forceinline__ bool resolve_tile(const WalkParams& p, uint32_t g, Re
     t.nr = min(rpt, rows - r0);
     t.w  = (uint32_t)min((uint64_t)tile_w, width - c0);
     t.s  = p.bufs[src_buf] + src_off + (uint64_t)r0 * t.sp + (c0 << t.cast);
-    t.d  = p.bufs[dst_buf] + dst_off + (uint64_t)r0 * t.dp + c0;
+    t.d_off = dst_off + (uint64_t)r0 * t.dp + c0;
     return true;
 }
 
@@ -290,12 +327,15 @@ __global__ void __launch_bounds__(512, 2) nereus_walk_vec(const __grid_constant_
             open_level = t.level;
         }
 
+        const uint32_t dst_buf = t.dst_buf, rstride = t.rstride;
+        const uint64_t d_off = t.d_off;
+        auto D = [&p, dst_buf, rstride, d_off](uint32_t j) { return tile_dst(p, dst_buf, rstride, d_off, j); };
         if (t.cast) {
-            cast_tile<kUnrollRect>(t.s, t.d, t.nr, t.w >> 3, t.sp, t.dp, lane);
+            cast_tile<kUnrollCast>(t.s, D, t.reps, t.nr, t.w >> 3, t.sp, t.dp, lane);
         } else if (t.nr == 1) {
-            copy_run<kUnrollRun>(t.s, t.d, t.w >> 4, lane);
+            copy_run<kUnrollRun>(t.s, D, t.reps, t.w >> 4, lane);
         } else {
-            copy_rect<kUnrollRect>(t.s, t.d, t.nr, t.w >> 4, t.sp, t.dp, lane);
+            copy_rect<kUnrollRect>(t.s, D, t.reps, t.nr, t.w >> 4, t.sp, t.dp, lane);
         }
         if (p.n_levels > 1) ++my_done;
         g = g_next;
@@ -316,9 +356,10 @@ __global__ void __launch_bounds__(512, 2) nereus_walk_vec(const __grid_constant_
 // destination record.  Data never passes through registers.
 
 struct StageMeta {
-    char*    d;
+    uint64_t d_off;
     uint32_t nr, w, dp;
     uint32_t kind;          // kStageData, kStageEnd or kStageFlush
+    uint16_t dst_buf, reps, rstride, pad_;
 };
 constexpr uint32_t kStageData = 0, kStageEnd = 1, kStageFlush = 2;
 
@@ -443,7 +484,9 @@ __global__ void __launch_bounds__(64, 2) nereus_walk_bulk(const __grid_constant_
                         break;
                     }
                     if (lane == 0) {
-                        meta[stage].d = t.d; meta[stage].nr = t.nr; meta[stage].w = t.w; meta[stage].dp = t.dp;
+                        meta[stage].d_off = t.d_off; meta[stage].nr = t.nr; meta[stage].w = t.w; meta[stage].dp = t.dp;
+                        meta[stage].dst_buf = (uint16_t)t.dst_buf; meta[stage].reps = (uint16_t)t.reps;
+                        meta[stage].rstride = (uint16_t)t.rstride;
                         meta[stage].kind = kStageData;
                         mbar_arrive_expect_tx(bar, t.nr * t.w);
                     }
@@ -485,12 +528,15 @@ __global__ void __launch_bounds__(64, 2) nereus_walk_bulk(const __grid_constant_
             } else {
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 const uint32_t base = smem_addr(smem + (size_t)stage * stage_bytes);
-                if (m.nr == 1) {
-                    for (uint32_t off = lane * kBulkPiece; off < m.w; off += 32 * kBulkPiece)
-                        bulk_store(m.d + off, base + off, min(kBulkPiece, m.w - off));
-                } else {
-                    for (uint32_t r = lane; r < m.nr; r += 32)
-                        bulk_store(m.d + (size_t)r * m.dp, base + r * m.w, m.w);
+                for (uint32_t j = 0; j < m.reps; ++j) {              // one load, `reps` stores
+                    char* d = tile_dst(p, m.dst_buf, m.rstride, m.d_off, j);
+                    if (m.nr == 1) {
+                        for (uint32_t off = lane * kBulkPiece; off < m.w; off += 32 * kBulkPiece)
+                            bulk_store(d + off, base + off, min(kBulkPiece, m.w - off));
+                    } else {
+                        for (uint32_t r = lane; r < m.nr; r += 32)
+                            bulk_store(d + (size_t)r * m.dp, base + r * m.w, m.w);
+                    }
                 }
                 ++unpublished;
             }
@@ -560,7 +606,7 @@ static int resolve_launch(const nereus_transition_s& t, int sms, Launch& L) {
     else if (want == 1) L.variant = 1;
     else                L.variant = (bulk_eligible(t) && t.bytes_written >= (64ull << 20) && asked_tile <= 49152) ? 2 : 1;
     L.ctas_per_sm = t.tuning.ctas_per_sm ? t.tuning.ctas_per_sm : env_int("NEREUS_CTAS_PER_SM", 2);
-    L.threads     = t.tuning.threads     ? t.tuning.threads     : env_int("NEREUS_THREADS", 512);
+    L.threads     = t.tuning.threads     ? t.tuning.threads     : env_int("NEREUS_THREADS", 384);
     L.tile_bytes  = t.tuning.tile_bytes  ? t.tuning.tile_bytes  : env_int("NEREUS_TILE_BYTES", 0);
     if (L.variant == 2) { L.ctas_per_sm = t.tuning.ctas_per_sm ? t.tuning.ctas_per_sm : 1; L.threads = 64; }
     if (L.ctas_per_sm < 1 || L.ctas_per_sm > 2 || L.threads < 32 || L.threads > 512 || L.threads % 32)

@@ -38,6 +38,8 @@ class Stage:
     src: tuple
     dst: tuple
     value_head: bool = False
+    replicas: int = 1          # identical destination units (Extend, Split into replica units)
+    n_opt: int = 0             # fp32 optimizer tensors per parameter that follow the same layout (Adam: 2)
 
 
 @dataclass(frozen=True)
@@ -83,6 +85,17 @@ WORKLOADS["8b4l_tp4pp2_to_tp1pp1"] = Workload("8b4l_tp4pp2_to_tp1pp1", (
     Stage("8b4l", LLAMA_8B_4L, 1, (4, 2, "bf16"), (1, 1, "bf16")),))
 WORKLOADS["8b4l_fp32_tp2pp2_to_bf16_tp4pp1"] = Workload("8b4l_fp32_tp2pp2_to_bf16_tp4pp1", (
     Stage("8b4l_master", LLAMA_8B_4L, 2, (2, 2, "fp32"), (4, 1, "bf16")),))
+
+# the next rows: k destination units (Extend / replica units) and the EMU's optimizer state
+WORKLOADS["8b_extend_tp4pp2_x2"] = Workload("8b_extend_tp4pp2_x2", (
+    Stage("8b", LLAMA_8B, 11, (4, 2, "bf16"), (4, 2, "bf16"), replicas=2),),
+    note="Extend: two new rank-aligned replicas of a TP4PP2 unit, every shard read once")
+WORKLOADS["8b_fp32_tp2pp2_to_bf16_tp4pp1_x2"] = Workload("8b_fp32_tp2pp2_to_bf16_tp4pp1_x2", (
+    Stage("8b_master", LLAMA_8B, 12, (2, 2, "fp32"), (4, 1, "bf16"), replicas=2),),
+    note="weight sync of fp32 master weights to two bf16 generation units")
+WORKLOADS["8b_state_adam_tp2pp2_to_tp4pp1"] = Workload("8b_state_adam_tp2pp2_to_tp4pp1", (
+    Stage("8b_train", LLAMA_8B, 13, (2, 2, "bf16"), (4, 1, "bf16"), n_opt=2),),
+    note="parameters (bf16) plus Adam's two fp32 moments, same layout, one table")
 
 # scaled-down stand-ins with the same structure, for parity tests the oracle finishes in seconds
 SMALL = Shape(4, 512, 8, 4, 1376, 2048)            # head_dim 64; several tiles and ragged tails

@@ -42,16 +42,18 @@ def interpret(rects, src, dst, counts=None):
     """Executes rect tasks on host byte arrays, level by level, in table order."""
     bufs = list(src) + list(dst)
     for r in rects:
-        s, d = bufs[r.src_buf], bufs[r.dst_buf]
+        s = bufs[r.src_buf]
         for i in range(r.rows):
             so, do = r.src_off + i * r.src_pitch, r.dst_off + i * r.dst_pitch
             piece = s[so:so + r.width_bytes_src]
             if r.cast:
                 piece = O.rne_bf16_array(piece.view(np.uint32)).view(np.uint8)
             assert piece.size == r.width_bytes_dst
-            d[do:do + r.width_bytes_dst] = piece
-            if counts is not None:
-                counts[r.dst_buf - len(src)][do:do + r.width_bytes_dst] += 1
+            for j in range(r.replicas):
+                k = r.dst_buf + j * r.replica_stride
+                bufs[k][do:do + r.width_bytes_dst] = piece
+                if counts is not None:
+                    counts[k - len(src)][do:do + r.width_bytes_dst] += 1
 
 
 def payload_mask(m, plan):
@@ -301,3 +303,55 @@ def test_run_rejects_bad_pointers_before_any_cuda_call():
     assert t.run_raw([src[0] + 8, src[1]], [base + (2 << 30)]) == B.ERR_ALIGN
     assert t.run_raw(src, [src[1] + sizes[1] - 256]) == B.ERR_ALIAS        # dst overlaps a source's tail
     assert t.run_raw(src, [src[0] - 16]) == B.ERR_ALIAS
+
+
+# ---------------------------------------------------------------- replicas (Extend) and optimizer state
+
+@pytest.mark.parametrize("a,b,k,sdt,ddt", [((2, 2), (2, 2), 3, "bf16", "bf16"),      # Extend: same layout, 3 new units
+                                           ((4, 1), (2, 2), 2, "bf16", "bf16"),      # Split into 2 replica units
+                                           ((2, 2), (4, 1), 2, "fp32", "bf16")])     # weight sync to 2 rollout units
+def test_replicated_destinations(a, b, k, sdt, ddt):
+    sh = I.SMALL
+    odt = {"bf16": O.BF16, "fp32": O.FP32}
+    d, m = desc_of(sh, B.DTYPES[sdt]), omodel_of(sh, odt[sdt])
+    src = random_src(m, O.Plan(*a), 11, sdt)
+    want = O.reshard_replicated(m, O.Plan(*a), O.Plan(b[0], b[1], odt[ddt]), k, src, fill=0xA5)
+    t = d.compile_replicated(B.Plan(*a), B.Plan(b[0], b[1], B.DTYPES[ddt]), k)
+    n_src, n_dst = t.num_buffers()
+    assert n_dst == k * b[0] * b[1] == len(want)
+    got = [np.full(t.buffer_bytes(True, j), 0xA5, np.uint8) for j in range(n_dst)]
+    counts = [np.zeros(g.size, np.uint8) for g in got]
+    interpret(t.rects(), src, got, counts)
+    for g, w in zip(got, want):
+        assert np.array_equal(g, w)
+    rd, wr = t.bytes()
+    one = d.compile(B.Plan(*a), B.Plan(b[0], b[1], B.DTYPES[ddt])).bytes()
+    assert rd == one[0] and wr == k * one[1]          # read once, written k times
+    if a == b and sdt == ddt:                          # Extend: every unit is a copy of the source unit
+        masks = payload_mask(m, O.Plan(*a))
+        for j, g in enumerate(got):
+            mk = masks[j % len(src)]
+            assert np.array_equal(g[mk], src[j % len(src)][mk])
+    with pytest.raises(B.NereusError) as e:
+        d.compile_replicated(B.Plan(*a), B.Plan(*b), 0)
+    assert e.value.code == B.ERR_ARG
+
+
+def test_state_with_optimizer_tensors():
+    """theta (bf16) plus Adam's two fp32 moments, all following the same layout, in one table."""
+    sh = I.SMALL
+    d, m = desc_of(sh), omodel_of(sh)
+    a, b = (2, 2), (4, 1)
+    m32 = omodel_of(sh, O.FP32)
+    src = random_src(m, O.Plan(*a), 1, "bf16") + random_src(m32, O.Plan(*a), 2, "fp32") + \
+        random_src(m32, O.Plan(*a), 3, "fp32")
+    want = O.reshard_state(m, O.Plan(*a), O.Plan(*b), 2, src, fill=0xA5)
+    t = d.compile_state(B.Plan(*a), B.Plan(*b), 2)
+    assert t.num_buffers() == (12, 12)
+    got = [np.full(t.buffer_bytes(True, j), 0xA5, np.uint8) for j in range(12)]
+    interpret(t.rects(), src, got)
+    for g, w in zip(got, want):
+        assert np.array_equal(g, w)
+    rd, wr = t.bytes()
+    theta = d.compile(B.Plan(*a), B.Plan(*b)).bytes()[0]
+    assert rd == wr == theta * (1 + 2 * 2)            # fp32 moments are twice the bf16 parameters, each

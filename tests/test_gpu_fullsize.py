@@ -23,6 +23,7 @@ TDT = {"bf16": torch.int16, "fp32": torch.int32}
 
 
 def _need(bytes_needed):
+    torch.cuda.empty_cache()                     # blocks cached from earlier tests count as used otherwise
     free, _ = torch.cuda.mem_get_info()
     if free < bytes_needed * 1.02 + (2 << 30):
         pytest.skip(f"needs {bytes_needed / 1e9:.1f} GB of device memory, {free / 1e9:.1f} GB free")

@@ -1,0 +1,133 @@
+"""GPU parity of the rows after the core path: k destination units (Extend; Split into replica units) and the
+EMU's optimizer state, both through the C ABI against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import bench
+import gpu_util as G
+import test_gpu_fullsize as F
+from oracle import oracle as O
+from paper_2609_34645_b200 import binding as B
+from paper_2609_34645_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("variant", [1, 2])
+@pytest.mark.parametrize("a,b,k,sdt,ddt", [((2, 2), (2, 2), 3, "bf16", "bf16"),      # Extend
+                                           ((4, 1), (2, 2), 2, "bf16", "bf16"),      # Split into 2 replica units
+                                           ((1, 1), (4, 2), 4, "bf16", "bf16"),
+                                           ((2, 2), (4, 1), 2, "fp32", "bf16")])     # weight sync to 2 units
+def test_replicated_destinations(a, b, k, sdt, ddt, variant):
+    sh = I.SMALL
+    desc = G.desc_of(sh, sdt)
+    pa, pb = B.Plan(*a), B.Plan(b[0], b[1], B.DTYPES[ddt])
+    for tile in (1024, 16384):
+        t = desc.compile_replicated(pa, pb, k)
+        t.tune(tile_bytes=tile, variant=variant)
+        src = G.device_sources(desc, pa, sdt, 17)
+        dst = G.Guarded([t.buffer_bytes(True, j) for j in range(t.num_buffers()[1])])
+        G.run_transition(t, src, dst.bufs)
+        want = O.reshard_replicated(G.omodel_of(sh, sdt), O.Plan(*a), O.Plan(b[0], b[1], G.ODT[ddt]), k,
+                                    [s.cpu().numpy() for s in src], fill=G.SENTINEL)
+        assert len(want) == len(dst.bufs) == k * b[0] * b[1]
+        for g, w in zip(dst.bufs, want):
+            assert np.array_equal(g.cpu().numpy(), w)
+        assert dst.guards_intact()
+
+
+@pytest.mark.parametrize("variant", [1, 2])
+def test_state_with_adam_moments(variant):
+    sh = I.SMALL
+    desc = G.desc_of(sh)
+    a, b = (2, 2), (4, 1)
+    pa, pb = B.Plan(*a), B.Plan(*b)
+    t = desc.compile_state(pa, pb, 2)
+    t.tune(variant=variant)
+    p32 = B.Plan(a[0], a[1], B.FP32)
+    src = G.device_sources(desc, pa, "bf16", 1) + G.device_sources(desc, p32, "fp32", 2) + \
+        G.device_sources(desc, p32, "fp32", 3)
+    dst = G.Guarded([t.buffer_bytes(True, j) for j in range(t.num_buffers()[1])])
+    G.run_transition(t, src, dst.bufs)
+    want = O.reshard_state(G.omodel_of(sh), O.Plan(*a), O.Plan(*b), 2, [s.cpu().numpy() for s in src],
+                           fill=G.SENTINEL)
+    for g, w in zip(dst.bufs, want):
+        assert np.array_equal(g.cpu().numpy(), w)
+    assert dst.guards_intact()
+
+
+def _bytes_of(name):
+    wl, t = I.WORKLOADS[name], None
+    st = wl.stages[0]
+    sh = st.shape
+    d = B.ModelDesc(sh.layers, sh.hidden, sh.heads, sh.kv_heads, sh.ffn, sh.vocab, B.DTYPES[st.src[2]], st.value_head)
+    pa = B.Plan(st.src[0], st.src[1], B.DTYPES[st.src[2]])
+    pb = B.Plan(st.dst[0], st.dst[1], B.DTYPES[st.dst[2]])
+    tot = sum(d.shard_sizes(pa)) + st.replicas * sum(d.shard_sizes(pb))
+    tot += st.n_opt * (sum(d.shard_sizes(B.Plan(pa.tp, pa.pp, B.FP32))) + sum(d.shard_sizes(B.Plan(pb.tp, pb.pp, B.FP32))))
+    return tot
+
+
+def _run(name):
+    F._need(_bytes_of(name))
+    wl, t, srcs, dsts, (parts, keep, descs) = bench.build_workload(name, torch.device("cuda"), dict(
+        tile_bytes=0, ctas_per_sm=0, threads=0, variant=0))
+    stream = torch.cuda.current_stream()
+    t.run([b.data_ptr() for b in srcs], [b.data_ptr() for b in dsts], stream.cuda_stream)
+    stream.synchronize()
+    assert t.status() == B.DEV_OK
+    return wl, t, srcs, dsts, descs
+
+
+def test_8b_extend_two_replicas_full_size():
+    """Extend at full size: each new unit's shard equals the source shard, every byte (the 8B shape has no
+    padding), which is the definition of a replica."""
+    wl, t, srcs, dsts, descs = _run("8b_extend_tp4pp2_x2")
+    n = len(srcs)
+    assert len(dsts) == 2 * n
+    for j, d in enumerate(dsts):
+        assert torch.equal(d, srcs[j % n]), f"replica {j // n} shard {j % n}"
+    rd, wr = t.bytes()
+    assert wr == 2 * rd == 2 * sum(b.numel() for b in srcs)
+    assert t.launch_info()["kernel"] == "nereus_walk_bulk"
+    del srcs, dsts
+    torch.cuda.empty_cache()
+
+
+def test_8b_weight_sync_to_two_generation_units_full_size():
+    wl, t, srcs, dsts, descs = _run("8b_fp32_tp2pp2_to_bf16_tp4pp1_x2")
+    st = wl.stages[0]
+    desc, pa, pb = descs[0]
+    n = desc.num_shards(pb)
+    for j in range(n):
+        assert torch.equal(dsts[j], dsts[n + j])                      # the two units are identical
+    F._check_stage_sums(st, desc, srcs, dsts[:n], pa, pb, "fp32", "bf16")
+    F._check_stage_sampled(st, srcs, dsts[:n], st.src, st.dst, list(range(1, 10)) + [9 * 32 + 1])
+    rd, wr = t.bytes()
+    assert rd == wr                                                   # 4 B read, 2 x 2 B written per element
+    del srcs, dsts
+    torch.cuda.empty_cache()
+
+
+def test_8b_state_with_adam_full_size():
+    wl, t, srcs, dsts, descs = _run("8b_state_adam_tp2pp2_to_tp4pp1")
+    st = wl.stages[0]
+    desc, pa, pb = descs[0]
+    ns, nd = desc.num_shards(pa), desc.num_shards(pb)
+    # parameters
+    F._check_stage_sums(st, desc, srcs[:ns], dsts[:nd], pa, pb, "bf16", "bf16")
+    F._check_stage_sampled(st, srcs[:ns], dsts[:nd], st.src, st.dst, list(range(1, 10)) + [9 * 32 + 1])
+    # the two moments: fp32 on both sides, same (tp, pp)
+    pa32, pb32 = B.Plan(pa.tp, pa.pp, B.FP32), B.Plan(pb.tp, pb.pp, B.FP32)
+    st32 = I.Stage(st.name, st.shape, st.seed, (pa.tp, pa.pp, "fp32"), (pb.tp, pb.pp, "fp32"))
+    d32 = B.ModelDesc(32, 4096, 32, 8, 14336, 128256, B.FP32)
+    for k in range(2):
+        s = srcs[ns * (1 + k):ns * (2 + k)]
+        d = dsts[nd * (1 + k):nd * (2 + k)]
+        F._check_stage_sums(st32, d32, s, d, pa32, pb32, "fp32", "fp32")
+        F._check_stage_sampled(st32, s, d, st32.src, st32.dst, [1, 2, 5, 9, 9 * 32 + 1])
+    rd, wr = t.bytes()
+    assert rd == wr == 5 * (8_030_261_248 * 2 + 65 * 8192 * 3)       # theta bf16 + two fp32 moments = 5x
+    del srcs, dsts, s, d
+    torch.cuda.empty_cache()

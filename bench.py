@@ -34,10 +34,10 @@ DEFAULT_WORKLOAD = "8b_tp1pp1_to_tp4pp2"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic bytes of one nereus_walk launch, from the ncu
-# captures on the 4-layer 8B stand-in summarised in profiles/nereus_walk_bulk__8b_split.md and
-# profiles/nereus_walk_vec__8b_split.md (both kernels: 0.993); traffic grows in
+# captures on the 4-layer 8B stand-ins summarised under profiles/ (bit copy, ring and vector kernel: 0.993;
+# cast ring: 0.9965); traffic grows in
 # proportion to the bytes moved (same tensor classes and piece sizes), so a full launch is scaled by it.
-NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 0.993
+NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = {"copy": 0.993, "cast": 0.9965}
 
 
 def parse_args():
@@ -356,7 +356,7 @@ def run_ours(args):
                    "multi_gpu": "replicas only", "tiles": t.num_tiles()[0], "levels": t.num_tiles()[1]},
         "frac_of_nominal_8TBps": achieved / NOMINAL_HBM_GBS,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": NCU_TRAFFIC_PER_ALGORITHMIC_BYTE * (rd + wr),
+                     "traffic": NCU_TRAFFIC_PER_ALGORITHMIC_BYTE["cast" if rd > wr else "copy"] * (rd + wr),
                      "traffic_note": "ncu capture on the 4-layer stand-in, scaled by bytes moved",
                      "peak_kind": f"of {peak_kind}", "kernel": t.launch_info()["kernel"], "launch": t.launch_info(),
                      "kernel_ms": kernel_ms, "kernel_ms_min": min(per_step)},

@@ -227,7 +227,7 @@ class Transition:
         v, tb, g, th = _i(), _i(), _i(), _i()
         _ck(_lib.nereus_transition_launch_info(self._h, ctypes.byref(v), ctypes.byref(tb), ctypes.byref(g),
                                                ctypes.byref(th)), "nereus_transition_launch_info")
-        return {"kernel": {1: "nereus_walk_vec", 2: "nereus_walk_bulk"}[v.value], "tile_bytes": tb.value,
+        return {"kernel": {1: "nereus_walk_vec", 2: "nereus_walk_ring"}[v.value], "tile_bytes": tb.value,
                 "grid": g.value, "threads": th.value}
 
     def prepare(self):

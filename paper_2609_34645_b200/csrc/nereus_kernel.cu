@@ -14,9 +14,10 @@
 //     limit, until every tile of level k-1 has completed; on giving up it records NEREUS_DEV_TIMEOUT and the
 //     warp leaves.  A warp publishes its completed tiles once per level (one fence, one atomic), not per
 //     tile.  Loads bypass L1 (ld.global.cg) so a level reads what another SM wrote before it.
-//   * second kernel, nereus_walk_bulk, for single-level bit-copy tables: one CTA per SM, a producer warp
+//   * second kernel, nereus_walk_ring, for large tables: one CTA per SM, a producer warp
 //     that claims tiles and issues cp.async.bulk global -> shared copies into a ring of stages, and a
-//     consumer warp that issues cp.async.bulk shared -> global stores; mbarriers track both directions and
+//     consumer warp that issues cp.async.bulk shared -> global stores (cast tables: fifteen consumer warps that
+//     convert from shared memory and store with plain 16-byte stores); mbarriers track both directions and
 //     every wait has an iteration limit.
 #include <cuda_runtime.h>
 
@@ -72,6 +73,13 @@ __device__ __forceinline__ uint32_t claim_tiles(Ctrl* ctrl, unsigned lane, uint3
     if (lane == 0) g = atomicAdd(&ctrl->cursor, n);
     return __shfl_sync(0xffffffffu, g, 0);
 }
+
+// A claim in two halves, so that the atomic's round trip hides behind the work in between: issue it on
+// lane 0, broadcast the answer only when it is needed.
+__device__ __forceinline__ uint32_t claim_issue(Ctrl* ctrl, unsigned lane, uint32_t n) {
+    return lane == 0 ? atomicAdd(&ctrl->cursor, n) : 0u;
+}
+__device__ __forceinline__ uint32_t claim_take(uint32_t issued) { return __shfl_sync(0xffffffffu, issued, 0); }
 
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
     uint32_t v;
@@ -227,30 +235,34 @@ __device__ __forceinline__ char* tile_dst(const WalkParams& p, uint32_t dst_buf,
 // The rect a claimer resolved last: consecutive claims of one warp usually fall into the same rect (a rect
 // has thousands of tiles), so the binary search is skipped while first <= g < next_first.
 struct RectRange {
-    uint32_t index = 0, first = 1, next_first = 0;            // empty range
+    uint32_t first = 1, next_first = 0;                        // empty range
+    uint4    q0, q1, q2, q3;                                   // the rect's 64-byte record
 };
 
 // Resolves tile g: binary search for the rect (largest i with first[i] <= g), then row block x column block.
 // Returns false when the table does not resolve (corrupted).
 template <bool kUseRange>
 __device__ __forceinline__ bool resolve_tile(const WalkParams& p, uint32_t g, RectRange& rr, Tile& t) {
+    uint4 q0, q1, q2, q3;
     if (!kUseRange || g < rr.first || g >= rr.next_first) {
         uint32_t lo = 0, hi = p.n_rects;                       // invariant: first[lo] <= g < first[hi]
         while (hi - lo > 1) {
             const uint32_t mid = (lo + hi) >> 1;
             if (__ldg(p.first + mid) <= g) lo = mid; else hi = mid;
         }
-        rr.index = lo;
+        const RectDev* rp = p.rects + lo;
+        q0 = __ldg(reinterpret_cast<const uint4*>(rp));        // src_off, dst_off
+        q1 = __ldg(reinterpret_cast<const uint4*>(rp) + 1);    // width, src_pitch, dst_pitch
+        q2 = __ldg(reinterpret_cast<const uint4*>(rp) + 2);    // rows, rows_per_tile, tile_w, col_tiles
+        q3 = __ldg(reinterpret_cast<const uint4*>(rp) + 3);    // first_tile, bufs, level|cast, replicas|stride
         if (kUseRange) {
             rr.first = __ldg(p.first + lo);
             rr.next_first = __ldg(p.first + lo + 1);
+            rr.q0 = q0; rr.q1 = q1; rr.q2 = q2; rr.q3 = q3;
         }
+    } else {
+        q0 = rr.q0; q1 = rr.q1; q2 = rr.q2; q3 = rr.q3;
     }
-    const RectDev* rp = p.rects + rr.index;
-    const uint4 q0 = __ldg(reinterpret_cast<const uint4*>(rp));          // src_off, dst_off
-    const uint4 q1 = __ldg(reinterpret_cast<const uint4*>(rp) + 1);      // width, src_pitch, dst_pitch
-    const uint4 q2 = __ldg(reinterpret_cast<const uint4*>(rp) + 2);      // rows, rows_per_tile, tile_w, col_tiles
-    const uint4 q3 = __ldg(reinterpret_cast<const uint4*>(rp) + 3);      // first_tile, bufs, level|cast
     const uint64_t src_off = ((uint64_t)q0.y << 32) | q0.x, dst_off = ((uint64_t)q0.w << 32) | q0.z;
     const uint64_t width   = ((uint64_t)q1.y << 32) | q1.x;
     const uint32_t rows = q2.x, rpt = q2.y, tile_w = q2.z, col_tiles = q2.w;
@@ -292,7 +304,7 @@ __global__ void __launch_bounds__(512, 2) nereus_walk_vec(const __grid_constant_
 
     uint32_t g = claim_tile(ctrl, lane);
     while (g < p.n_tiles) {
-        const uint32_t g_next = claim_tile(ctrl, lane);        // in flight while this tile is copied
+        const uint32_t next_issued = claim_issue(ctrl, lane, 1);   // in flight while this tile is copied
         Tile t;
         if (!resolve_tile<false>(p, g, rr, t)) {
             if (lane == 0) raise_status(ctrl, NEREUS_DEV_BOUNDS, g);
@@ -338,7 +350,7 @@ __global__ void __launch_bounds__(512, 2) nereus_walk_vec(const __grid_constant_
             copy_rect<kUnrollRect>(t.s, D, t.reps, t.nr, t.w >> 4, t.sp, t.dp, lane);
         }
         if (p.n_levels > 1) ++my_done;
-        g = g_next;
+        g = claim_take(next_issued);
     }
     if (my_done) {
         __threadfence();
@@ -352,7 +364,7 @@ __global__ void __launch_bounds__(512, 2) nereus_walk_vec(const __grid_constant_
 // ---------------------------------------------------------------------------------------------------
 //
 // Shared memory: n_stages x stage_bytes of data, then per stage one "full" mbarrier (1 arrival + the
-// bytes the bulk loads deliver), one "empty" mbarrier (32 arrivals: the consumer lanes) and the tile's
+// bytes the bulk loads deliver), one "empty" mbarrier (one arrival per consumer warp) and the tile's
 // destination record.  Data never passes through registers.
 
 struct StageMeta {
@@ -364,9 +376,8 @@ struct StageMeta {
 constexpr uint32_t kStageData = 0, kStageEnd = 1, kStageFlush = 2;
 
 constexpr uint32_t kBulkMaxStages = 28;
-constexpr uint32_t kBulkPiece     = 4096;       // contiguous tiles are issued in pieces of this many bytes
 constexpr uint32_t kClaimBatch    = 4;          // consecutive tiles per claim of the ring's producer
-constexpr uint32_t kBulkLag       = 2;          // stages whose stores may still be reading shared memory
+constexpr uint32_t kCastConsumers = 480;        // cast ring: threads that convert a stage (15 warps)
 constexpr uint32_t kBarrierTries  = 1u << 22;   // try_wait attempts before a wait gives up
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -400,165 +411,265 @@ __device__ __forceinline__ void bulk_store(char* dst, uint32_t src_smem, uint32_
                  ::"l"(dst), "r"(src_smem), "r"(bytes) : "memory");
 }
 
-__global__ void __launch_bounds__(64, 2) nereus_walk_bulk(const __grid_constant__ WalkParams p,
-                                                          const uint32_t stage_bytes, const uint32_t n_stages) {
-    extern __shared__ __align__(128) unsigned char smem[];
-    uint64_t*  full  = reinterpret_cast<uint64_t*>(smem + (size_t)stage_bytes * n_stages);
-    uint64_t*  empty = full + n_stages;
-    StageMeta* meta  = reinterpret_cast<StageMeta*>(empty + n_stages);
-    const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+struct Ring {
+    unsigned char* data;
+    uint64_t*      full;
+    uint64_t*      empty;
+    StageMeta*     meta;
+    uint32_t       stage_bytes, n_stages;
+    uint32_t       piece;          // contiguous tiles are issued as bulk copies of this many bytes
+    uint32_t       lag;            // stages whose stores may still be reading shared memory
+};
+
+// cp.async.bulk.wait_group.read takes an immediate
+__device__ __forceinline__ void wait_store_reads(uint32_t pending) {
+    switch (pending) {
+    case 1:  asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); break;
+    case 2:  asm volatile("cp.async.bulk.wait_group.read 2;" ::: "memory"); break;
+    case 3:  asm volatile("cp.async.bulk.wait_group.read 3;" ::: "memory"); break;
+    case 4:  asm volatile("cp.async.bulk.wait_group.read 4;" ::: "memory"); break;
+    case 5:  asm volatile("cp.async.bulk.wait_group.read 5;" ::: "memory"); break;
+    case 6:  asm volatile("cp.async.bulk.wait_group.read 6;" ::: "memory"); break;
+    case 7:  asm volatile("cp.async.bulk.wait_group.read 7;" ::: "memory"); break;
+    case 8:  asm volatile("cp.async.bulk.wait_group.read 8;" ::: "memory"); break;
+    default: asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); break;
+    }
+}
+
+// Producer warp: claims kClaimBatch consecutive tiles at a time, resolves them and loads them into the ring.
+// kCast: the stage receives the fp32 source bytes (twice the destination bytes).
+template <bool kCast>
+__device__ __forceinline__ void ring_producer(const WalkParams& p, const Ring& R, unsigned lane) {
+    Ctrl* const ctrl = p.ctrl;
+    uint32_t    stage = 0, phase = 0, level = 0;
+    RectRange   rr;
+    uint32_t    g0 = claim_tiles(ctrl, lane, kClaimBatch);
+    bool        running = true;
+    while (running) {
+        const bool     last    = g0 >= p.n_tiles;
+        const uint32_t next_issued = last ? g0 : claim_issue(ctrl, lane, kClaimBatch);   // hidden behind this batch
+        for (uint32_t g = g0; running && g < g0 + kClaimBatch; ++g) {
+            const bool end = g >= p.n_tiles;
+            Tile t;
+            bool ok = true;
+            if (!end) {
+                ok = resolve_tile<true>(p, g, rr, t) && t.cast == (kCast ? 1u : 0u) &&
+                     (((uint64_t)t.nr * t.w) << (kCast ? 1 : 0)) <= R.stage_bytes;
+                if (!ok && lane == 0) raise_status(ctrl, NEREUS_DEV_BOUNDS, g);
+            }
+            // a tile of a higher level: first have the consumer publish this CTA's finished tiles (a flush
+            // stage), only then wait for the level below to be complete everywhere
+            const bool climb = !end && ok && t.level > level;
+            for (int pass = climb ? 0 : 1; running && pass < 2; ++pass) {
+                // the stage is free once the consumer has finished reading its previous contents
+                bool freed = true;
+                if (lane == 0) freed = mbar_wait(smem_addr(R.empty + stage), phase ^ 1);
+                freed = __shfl_sync(0xffffffffu, freed, 0);
+                if (!freed) {
+                    if (lane == 0) raise_status(ctrl, NEREUS_DEV_TIMEOUT, g);
+                    running = false;
+                    break;
+                }
+                const uint32_t base = smem_addr(R.data + (size_t)stage * R.stage_bytes);
+                const uint32_t bar  = smem_addr(R.full + stage);
+                if (pass == 0) {
+                    if (lane == 0) {
+                        R.meta[stage].kind = kStageFlush;
+                        mbar_arrive(bar);
+                    }
+                    if (++stage == R.n_stages) { stage = 0; phase ^= 1; }
+                    // dependency gate, bounded
+                    bool open = true;
+                    if (lane == 0) {
+                        // a cast table counts warp-tiles: every tile is published by each of its consumer warps
+                        const uint32_t need = p.level_end[t.level - 1] * (kCast ? kCastConsumers / 32 : 1u);
+                        uint32_t polls = 0;
+                        while (ld_acquire_u32(&ctrl->done) < need) {
+                            if (++polls > kGatePolls) { open = false; break; }
+                            __nanosleep(200);
+                        }
+                        if (!open) raise_status(ctrl, NEREUS_DEV_TIMEOUT, g);
+                    }
+                    open = __shfl_sync(0xffffffffu, open, 0);
+                    if (!open) { ok = false; }
+                    // what other SMs wrote and published is read below through the async proxy
+                    asm volatile("fence.proxy.async.global;" ::: "memory");
+                    level = t.level;
+                    continue;
+                }
+                if (end || !ok) {
+                    if (lane == 0) {
+                        R.meta[stage].kind = kStageEnd;
+                        mbar_arrive(bar);
+                    }
+                    running = false;
+                    break;
+                }
+                const uint32_t ws = t.w << (kCast ? 1 : 0);                 // source bytes per row piece
+                if (lane == 0) {
+                    StageMeta& m = R.meta[stage];
+                    m.d_off = t.d_off; m.nr = t.nr; m.w = t.w; m.dp = t.dp;
+                    m.dst_buf = (uint16_t)t.dst_buf; m.reps = (uint16_t)t.reps; m.rstride = (uint16_t)t.rstride;
+                    m.kind = kStageData;
+                    mbar_arrive_expect_tx(bar, t.nr * ws);
+                }
+                __syncwarp();
+                if (t.nr == 1) {
+                    for (uint32_t off = lane * R.piece; off < ws; off += 32 * R.piece)
+                        bulk_load(base + off, t.s + off, min(R.piece, ws - off), bar);
+                } else {
+                    for (uint32_t r = lane; r < t.nr; r += 32)
+                        bulk_load(base + r * ws, t.s + (size_t)r * t.sp, ws, bar);
+                }
+                if (++stage == R.n_stages) { stage = 0; phase ^= 1; }
+            }
+        }
+        g0 = last ? g0 : claim_take(next_issued);
+    }
+}
+
+// Consumer warp of the bit-copy ring: stores full stages with bulk copies, hands them back `lag` stages later.
+__device__ __forceinline__ void ring_consumer_copy(const WalkParams& p, const Ring& R, unsigned lane) {
+    Ctrl* const ctrl = p.ctrl;
+    uint32_t    stage = 0, phase = 0, issued = 0, unpublished = 0;
+    while (true) {
+        bool ready = true;
+        if (lane == 0) ready = mbar_wait(smem_addr(R.full + stage), phase);
+        ready = __shfl_sync(0xffffffffu, ready, 0);
+        if (!ready) {
+            if (lane == 0) raise_status(ctrl, NEREUS_DEV_TIMEOUT, 0xFFFFFFFFu);
+            break;
+        }
+        const StageMeta m = R.meta[stage];
+        if (m.kind == kStageEnd) break;
+        if (m.kind == kStageFlush) {
+            // this CTA leaves a level: all its stores must have landed and be visible device-wide before
+            // the tiles are counted as done
+            asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+            asm volatile("fence.proxy.async.global;" ::: "memory");
+            __threadfence();
+            __syncwarp();
+            if (lane == 0 && unpublished) atomicAdd(&ctrl->done, unpublished);
+            unpublished = 0;
+        } else {
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            const uint32_t base = smem_addr(R.data + (size_t)stage * R.stage_bytes);
+            for (uint32_t j = 0; j < m.reps; ++j) {              // one load, `reps` stores
+                char* d = tile_dst(p, m.dst_buf, m.rstride, m.d_off, j);
+                if (m.nr == 1) {
+                    for (uint32_t off = lane * R.piece; off < m.w; off += 32 * R.piece)
+                        bulk_store(d + off, base + off, min(R.piece, m.w - off));
+                } else {
+                    for (uint32_t r = lane; r < m.nr; r += 32)
+                        bulk_store(d + (size_t)r * m.dp, base + r * m.w, m.w);
+                }
+            }
+            ++unpublished;
+        }
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");        // a flush commits an empty group
+        ++issued;
+        if (issued > R.lag) {
+            // all but the `lag` newest groups of this lane have finished reading shared memory
+            wait_store_reads(R.lag);
+            const uint32_t rel = (stage + R.n_stages - R.lag) % R.n_stages;
+            __syncwarp();                                             // every lane's stores have read the stage
+            if (lane == 0) mbar_arrive(smem_addr(R.empty + rel));
+        }
+        if (++stage == R.n_stages) { stage = 0; phase ^= 1; }
+    }
+    // shared memory must outlive the stores that read it; other CTAs may be waiting for this one's tiles
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    if (p.n_levels > 1 && unpublished) {
+        asm volatile("fence.proxy.async.global;" ::: "memory");
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) atomicAdd(&ctrl->done, unpublished);
+    }
+}
+
+
+// Consumer warps of the cast ring: read fp32 from the stage, convert, store bf16 with plain 16-byte stores.
+// The unit is 8 elements: 32 bytes of shared memory in, 16 bytes out.  Each of the warps publishes its
+// own share of a tile, so the completion counter of a cast table counts warp-tiles (15 per tile) and no wait
+// between the warps (which could not be bounded) is needed.  Fifteen warps: a lone warp per scheduler would
+// be bound by the latency of its own dependent instructions.
+__device__ __forceinline__ void ring_consumer_cast(const WalkParams& p, const Ring& R, unsigned ct) {
     Ctrl* const    ctrl = p.ctrl;
+    const unsigned lane = ct & 31;
+    uint32_t       stage = 0, phase = 0, unpublished = 0;
+    while (true) {
+        bool ready = true;
+        if (lane == 0) ready = mbar_wait(smem_addr(R.full + stage), phase);
+        ready = __shfl_sync(0xffffffffu, ready, 0);
+        if (!ready) {
+            if (ct == 0) raise_status(ctrl, NEREUS_DEV_TIMEOUT, 0xFFFFFFFFu);
+            break;
+        }
+        const StageMeta m = R.meta[stage];
+        if (m.kind == kStageEnd) break;
+        if (m.kind == kStageFlush) {
+            __threadfence();
+            __syncwarp();
+            if (lane == 0 && unpublished) atomicAdd(&ctrl->done, unpublished);
+            unpublished = 0;
+        } else {
+            const unsigned char* src = R.data + (size_t)stage * R.stage_bytes;
+            const uint32_t upr = m.w >> 4, nunit = m.nr * upr, ws = m.w << 1;
+#pragma unroll 2
+            for (uint32_t idx = ct; idx < nunit; idx += kCastConsumers) {
+                const uint32_t r = idx / upr, c = idx - r * upr;
+                const uint4 a = *reinterpret_cast<const uint4*>(src + r * ws + c * 32);
+                const uint4 b = *reinterpret_cast<const uint4*>(src + r * ws + c * 32 + 16);
+                uint4 o;
+                o.x = pack_bf16x2(__uint_as_float(a.x), __uint_as_float(a.y));
+                o.y = pack_bf16x2(__uint_as_float(a.z), __uint_as_float(a.w));
+                o.z = pack_bf16x2(__uint_as_float(b.x), __uint_as_float(b.y));
+                o.w = pack_bf16x2(__uint_as_float(b.z), __uint_as_float(b.w));
+                const uint32_t doff = r * m.dp + c * 16;
+                for (uint32_t j = 0; j < m.reps; ++j)
+                    st_stream(tile_dst(p, m.dst_buf, m.rstride, m.d_off, j) + doff, o);
+            }
+            ++unpublished;
+        }
+        __syncwarp();                                            // this warp is done reading the stage
+        if (lane == 0) mbar_arrive(smem_addr(R.empty + stage));
+        if (++stage == R.n_stages) { stage = 0; phase ^= 1; }
+    }
+    if (p.n_levels > 1 && unpublished) {
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) atomicAdd(&ctrl->done, unpublished);
+    }
+}
+
+template <bool kCast>
+__global__ void __launch_bounds__(kCast ? 32 + kCastConsumers : 64, kCast ? 1 : 2)
+nereus_walk_ring(const __grid_constant__ WalkParams p, const uint32_t stage_bytes, const uint32_t n_stages,
+                 const uint32_t piece, const uint32_t lag) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    Ring R;
+    R.data  = smem;
+    R.full  = reinterpret_cast<uint64_t*>(smem + (size_t)stage_bytes * n_stages);
+    R.empty = R.full + n_stages;
+    R.meta  = reinterpret_cast<StageMeta*>(R.empty + n_stages);
+    R.stage_bytes = stage_bytes;
+    R.n_stages = n_stages;
+    R.piece = piece;
+    R.lag = lag;
+    const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
     if (threadIdx.x == 0) {
         for (uint32_t i = 0; i < n_stages; ++i) {
-            mbar_init(smem_addr(full + i), 1);
-            mbar_init(smem_addr(empty + i), 32);
+            mbar_init(smem_addr(R.full + i), 1);
+            mbar_init(smem_addr(R.empty + i), kCast ? kCastConsumers / 32 : 1);     // one arrival per consumer warp
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
 
-    if (warp == 0) {
-        // ---------------- producer: claim kClaimBatch consecutive tiles at a time, resolve, load into the ring
-        uint32_t  stage = 0, phase = 0, level = 0;
-        RectRange rr;
-        uint32_t  g0 = claim_tiles(ctrl, lane, kClaimBatch);
-        bool      running = true;
-        while (running) {
-            const bool     last    = g0 >= p.n_tiles;
-            const uint32_t g0_next = last ? g0 : claim_tiles(ctrl, lane, kClaimBatch);   // hidden behind this batch
-            for (uint32_t g = g0; running && g < g0 + kClaimBatch; ++g) {
-                const bool end = g >= p.n_tiles;
-                Tile t;
-                bool ok = true;
-                if (!end) {
-                    ok = resolve_tile<true>(p, g, rr, t) && t.cast == 0 && (uint64_t)t.nr * t.w <= stage_bytes;
-                    if (!ok && lane == 0) raise_status(ctrl, NEREUS_DEV_BOUNDS, g);
-                }
-                // a tile of a higher level: first have the consumer publish this CTA's finished tiles (a flush
-                // stage), only then wait for the level below to be complete everywhere
-                const bool climb = !end && ok && t.level > level;
-                for (int pass = climb ? 0 : 1; running && pass < 2; ++pass) {
-                    // the stage is free once the consumer's stores of its previous use have read it
-                    bool freed = true;
-                    if (lane == 0) freed = mbar_wait(smem_addr(empty + stage), phase ^ 1);
-                    freed = __shfl_sync(0xffffffffu, freed, 0);
-                    if (!freed) {
-                        if (lane == 0) raise_status(ctrl, NEREUS_DEV_TIMEOUT, g);
-                        running = false;
-                        break;
-                    }
-                    const uint32_t base = smem_addr(smem + (size_t)stage * stage_bytes);
-                    const uint32_t bar  = smem_addr(full + stage);
-                    if (pass == 0) {
-                        if (lane == 0) {
-                            meta[stage].kind = kStageFlush;
-                            mbar_arrive(bar);
-                        }
-                        if (++stage == n_stages) { stage = 0; phase ^= 1; }
-                        // dependency gate, bounded
-                        bool open = true;
-                        if (lane == 0) {
-                            const uint32_t need = p.level_end[t.level - 1];
-                            uint32_t polls = 0;
-                            while (ld_acquire_u32(&ctrl->done) < need) {
-                                if (++polls > kGatePolls) { open = false; break; }
-                                __nanosleep(200);
-                            }
-                            if (!open) raise_status(ctrl, NEREUS_DEV_TIMEOUT, g);
-                        }
-                        open = __shfl_sync(0xffffffffu, open, 0);
-                        if (!open) { ok = false; }
-                        // what other SMs wrote (through the async proxy, published after a proxy fence) is read
-                        // below through the async proxy again
-                        asm volatile("fence.proxy.async.global;" ::: "memory");
-                        level = t.level;
-                        continue;
-                    }
-                    if (end || !ok) {
-                        if (lane == 0) {
-                            meta[stage].kind = kStageEnd;
-                            mbar_arrive(bar);
-                        }
-                        running = false;
-                        break;
-                    }
-                    if (lane == 0) {
-                        meta[stage].d_off = t.d_off; meta[stage].nr = t.nr; meta[stage].w = t.w; meta[stage].dp = t.dp;
-                        meta[stage].dst_buf = (uint16_t)t.dst_buf; meta[stage].reps = (uint16_t)t.reps;
-                        meta[stage].rstride = (uint16_t)t.rstride;
-                        meta[stage].kind = kStageData;
-                        mbar_arrive_expect_tx(bar, t.nr * t.w);
-                    }
-                    __syncwarp();
-                    if (t.nr == 1) {
-                        for (uint32_t off = lane * kBulkPiece; off < t.w; off += 32 * kBulkPiece)
-                            bulk_load(base + off, t.s + off, min(kBulkPiece, t.w - off), bar);
-                    } else {
-                        for (uint32_t r = lane; r < t.nr; r += 32)
-                            bulk_load(base + r * t.w, t.s + (size_t)r * t.sp, t.w, bar);
-                    }
-                    if (++stage == n_stages) { stage = 0; phase ^= 1; }
-                }
-            }
-            g0 = g0_next;
-        }
-    } else {
-        // ---------------- consumer: store full stages, hand them back kBulkLag stages later
-        uint32_t stage = 0, phase = 0, issued = 0, unpublished = 0;
-        while (true) {
-            bool ready = true;
-            if (lane == 0) ready = mbar_wait(smem_addr(full + stage), phase);
-            ready = __shfl_sync(0xffffffffu, ready, 0);
-            if (!ready) {
-                if (lane == 0) raise_status(ctrl, NEREUS_DEV_TIMEOUT, 0xFFFFFFFFu);
-                break;
-            }
-            const StageMeta m = meta[stage];
-            if (m.kind == kStageEnd) break;
-            if (m.kind == kStageFlush) {
-                // this CTA leaves a level: all its stores must have landed and be visible device-wide before
-                // the tiles are counted as done
-                asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-                asm volatile("fence.proxy.async.global;" ::: "memory");
-                __threadfence();
-                __syncwarp();
-                if (lane == 0 && unpublished) atomicAdd(&ctrl->done, unpublished);
-                unpublished = 0;
-            } else {
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                const uint32_t base = smem_addr(smem + (size_t)stage * stage_bytes);
-                for (uint32_t j = 0; j < m.reps; ++j) {              // one load, `reps` stores
-                    char* d = tile_dst(p, m.dst_buf, m.rstride, m.d_off, j);
-                    if (m.nr == 1) {
-                        for (uint32_t off = lane * kBulkPiece; off < m.w; off += 32 * kBulkPiece)
-                            bulk_store(d + off, base + off, min(kBulkPiece, m.w - off));
-                    } else {
-                        for (uint32_t r = lane; r < m.nr; r += 32)
-                            bulk_store(d + (size_t)r * m.dp, base + r * m.w, m.w);
-                    }
-                }
-                ++unpublished;
-            }
-            asm volatile("cp.async.bulk.commit_group;" ::: "memory");        // a flush commits an empty group
-            ++issued;
-            if (issued > kBulkLag) {
-                // all but the kBulkLag newest groups of this lane have finished reading shared memory
-                asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kBulkLag) : "memory");
-                const uint32_t rel = (stage + n_stages - kBulkLag) % n_stages;
-                mbar_arrive(smem_addr(empty + rel));
-            }
-            if (++stage == n_stages) { stage = 0; phase ^= 1; }
-        }
-        // shared memory must outlive the stores that read it; other CTAs may be waiting for this one's tiles
-        asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-        if (p.n_levels > 1 && unpublished) {
-            asm volatile("fence.proxy.async.global;" ::: "memory");
-            __threadfence();
-            __syncwarp();
-            if (lane == 0) atomicAdd(&ctrl->done, unpublished);
-        }
-    }
+    if (warp == 0) ring_producer<kCast>(p, R, lane);
+    else if (kCast) ring_consumer_cast(p, R, threadIdx.x - 32);
+    else ring_consumer_copy(p, R, lane);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -586,15 +697,19 @@ static int env_int(const char* name, int dflt) {
 // Launch shape of one run, from the handle's tuning, the environment and the table.
 struct Launch {
     int      variant = 1;           // 1 vector copy, 2 bulk-copy ring
+    bool     cast = false;          // ring only: the table is all cast
     int      tile_bytes = 0, ctas_per_sm = 0, threads = 0;
     uint32_t n_stages = 0;          // bulk ring
+    uint32_t piece = 16384, lag = 2;
     size_t   smem = 0;
 };
 
-static bool bulk_eligible(const nereus_transition_s& t) {
-    for (const Rect& r : t.rects)
-        if (r.cast) return false;
-    return true;
+// The ring takes tables that are all bit copy or all cast; mixed tables run on the vector kernel.
+static bool ring_eligible(const nereus_transition_s& t, bool& cast) {
+    bool any_cast = false, any_copy = false;
+    for (const Rect& r : t.rects) (r.cast ? any_cast : any_copy) = true;
+    cast = any_cast;
+    return !(any_cast && any_copy);
 }
 
 static int resolve_launch(const nereus_transition_s& t, int sms, Launch& L) {
@@ -602,9 +717,11 @@ static int resolve_launch(const nereus_transition_s& t, int sms, Launch& L) {
     const int asked_tile = t.tuning.tile_bytes ? t.tuning.tile_bytes : env_int("NEREUS_TILE_BYTES", 0);
     // default: the ring for large single-level bit-copy tables (its per-CTA start-up costs more than it gains
     // below a few tens of MB), the vector kernel for everything else
-    if (want == 2)      L.variant = bulk_eligible(t) ? 2 : 1;
+    const bool ring_ok = ring_eligible(t, L.cast);
+    if (want == 2)      L.variant = ring_ok ? 2 : 1;
     else if (want == 1) L.variant = 1;
-    else                L.variant = (bulk_eligible(t) && t.bytes_written >= (64ull << 20) && asked_tile <= 49152) ? 2 : 1;
+    else                L.variant = (ring_ok && t.bytes_written >= (64ull << 20) &&
+                                     asked_tile <= (L.cast ? 24576 : 49152)) ? 2 : 1;
     L.ctas_per_sm = t.tuning.ctas_per_sm ? t.tuning.ctas_per_sm : env_int("NEREUS_CTAS_PER_SM", 2);
     L.threads     = t.tuning.threads     ? t.tuning.threads     : env_int("NEREUS_THREADS", 384);
     L.tile_bytes  = t.tuning.tile_bytes  ? t.tuning.tile_bytes  : env_int("NEREUS_TILE_BYTES", 0);
@@ -614,17 +731,22 @@ static int resolve_launch(const nereus_transition_s& t, int sms, Launch& L) {
     if (L.tile_bytes == 0) {
         // default: 16 KiB per warp tile (32 KiB per ring stage); smaller tiles for small tables, so that every
         // claimer still gets a few tiles
-        L.tile_bytes = L.variant == 2 ? 32768 : 16384;
+        L.tile_bytes = L.variant == 2 ? (L.cast ? 24576 : 32768) : 16384;
         const uint64_t claimers = (uint64_t)sms * L.ctas_per_sm * (L.variant == 2 ? 8 : L.threads / 32);
         while (L.tile_bytes > 1024 && t.bytes_written / L.tile_bytes < 4 * claimers) L.tile_bytes /= 2;
     }
     if (L.tile_bytes < 512 || L.tile_bytes % 512) return NEREUS_ERR_ARG;
     if (L.variant == 2) {
+        if (L.cast) L.ctas_per_sm = 1;
         const size_t budget = (227 * 1024) / L.ctas_per_sm - 1024;          // per CTA
-        if ((size_t)L.tile_bytes > budget / 4) return NEREUS_ERR_ARG;
-        const size_t per_stage = (size_t)L.tile_bytes + 2 * sizeof(uint64_t) + sizeof(StageMeta);
+        const size_t stage_bytes = (size_t)L.tile_bytes << (L.cast ? 1 : 0); // a cast stage holds the fp32 source
+        if (stage_bytes > budget / 4) return NEREUS_ERR_ARG;
+        const size_t per_stage = stage_bytes + 2 * sizeof(uint64_t) + sizeof(StageMeta);
         L.n_stages = (uint32_t)std::min<size_t>(kBulkMaxStages, budget / per_stage);
         L.smem = L.n_stages * per_stage;
+        L.piece = (uint32_t)env_int("NEREUS_RING_PIECE", 16384);
+        L.lag = (uint32_t)env_int("NEREUS_RING_LAG", std::min(3, (int)L.n_stages - 2));
+        if (L.piece < 16 || L.piece % 16 || L.lag < 1 || L.lag > 8 || L.lag + 2 > L.n_stages) return NEREUS_ERR_ARG;
     }
     return NEREUS_OK;
 }
@@ -632,9 +754,15 @@ static int resolve_launch(const nereus_transition_s& t, int sms, Launch& L) {
 static int launch_walk(const Launch& L, int sms, const WalkParams& p, cudaStream_t stream) {
     if (p.n_tiles == 0) return NEREUS_OK;
     if (L.variant == 2) {
-        NEREUS_CUDA(cudaFuncSetAttribute(nereus_walk_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.smem));
         const unsigned grid = std::max(1u, std::min((unsigned)(sms * L.ctas_per_sm), p.n_tiles));
-        nereus_walk_bulk<<<grid, 64, L.smem, stream>>>(p, (uint32_t)L.tile_bytes, L.n_stages);
+        if (L.cast) {
+            NEREUS_CUDA(cudaFuncSetAttribute(nereus_walk_ring<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.smem));
+            nereus_walk_ring<true><<<grid, 32 + kCastConsumers, L.smem, stream>>>(p, (uint32_t)L.tile_bytes * 2, L.n_stages,
+                                                                                  L.piece, L.lag);
+        } else {
+            NEREUS_CUDA(cudaFuncSetAttribute(nereus_walk_ring<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.smem));
+            nereus_walk_ring<false><<<grid, 64, L.smem, stream>>>(p, (uint32_t)L.tile_bytes, L.n_stages, L.piece, L.lag);
+        }
     } else {
         const unsigned warps_per_cta = (unsigned)L.threads / 32;
         unsigned grid = (unsigned)(sms * L.ctas_per_sm);
@@ -761,7 +889,8 @@ int nereus_transition_launch_info(nereus_transition_t t, int* variant, int* tile
     Launch L;
     if (int rc = resolve_launch(*t, sms, L)) return rc;
     if (t->dev.rects) L.tile_bytes = t->dev.tile_bytes;
-    *variant = L.variant; *tile_bytes = L.tile_bytes; *grid = sms * L.ctas_per_sm; *threads = L.threads;
+    *variant = L.variant; *tile_bytes = L.tile_bytes; *grid = sms * L.ctas_per_sm;
+    *threads = L.variant == 2 ? (L.cast ? 32 + (int)kCastConsumers : 64) : L.threads;
     return NEREUS_OK;
 }
 

@@ -90,7 +90,7 @@ def test_8b_extend_two_replicas_full_size():
         assert torch.equal(d, srcs[j % n]), f"replica {j // n} shard {j % n}"
     rd, wr = t.bytes()
     assert wr == 2 * rd == 2 * sum(b.numel() for b in srcs)
-    assert t.launch_info()["kernel"] == "nereus_walk_bulk"
+    assert t.launch_info()["kernel"] == "nereus_walk_ring"
     del srcs, dsts
     torch.cuda.empty_cache()
 

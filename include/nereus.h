@@ -194,11 +194,44 @@ int nereus_transition_prepare(nereus_transition_t t);
  * Errors: ARG (null), ALIGN, ALIAS, CUDA.  Runs of the same handle must not overlap on the device. */
 int nereus_transition_run(nereus_transition_t t, const void* const* src_ptrs, void* const* dst_ptrs,
                           void* cuda_stream);
+/* Environment variables read by run(): NEREUS_TILE_BYTES, NEREUS_CTAS_PER_SM, NEREUS_THREADS, NEREUS_VARIANT
+ * (defaults of the tuning fields), NEREUS_RING_PIECE, NEREUS_RING_LAG (ring internals), and, for tests of the
+ * failure path only, NEREUS_DEBUG_GATE_BIAS: a count added to what every dependency gate waits for, so that
+ * the gate cannot open; the waits then run into their poll limit (about half a second), the run ends with
+ * device status NEREUS_DEV_TIMEOUT and the destinations of the gated levels stay unwritten. */
+
 /* Reads the device status word of the last run (NEREUS_DEV_*).  The caller must have synchronised the
  * stream first; this call copies 4 bytes from the device synchronously. */
 int nereus_transition_status(nereus_transition_t t, int* device_status);
 /* Kernels this handle has launched since it was created (one per run). */
 int nereus_transition_launches(nereus_transition_t t, uint64_t* n);
+
+/* ---- cost side: the transition estimate and the admission gate (Sections 4.3 and 6) ------------------- */
+
+/* L_tran of a compiled transition: the paper estimates the critical-path cost "from bytes, link bandwidth,
+ * and communicator setup" (Section 6); on one GPU the link is HBM and the set-up is the launch.  Levels run
+ * one after another, so seconds = setup_seconds + sum over levels of (bytes read + written) / bandwidth.
+ * gbytes_per_s: the sustained reshard bandwidth (e.g. a value bench.py measured); must be > 0.
+ * Errors: ARG. */
+int nereus_transition_estimate(nereus_transition_t t, double gbytes_per_s, double setup_seconds, double* seconds);
+
+/* The profitability gate, Eq. 2 of Section 4.3: with delta_l = l_step_current - l_step_target (seconds per
+ * step), an executable opportunistic transition is admitted iff delta_l > 0 and
+ * l_tran / delta_l <= gamma * h_x, the payback period in steps against a fraction gamma in [0, 1] of the
+ * horizon h_x (steps until the triggering signal's next threshold crossing; the smallest one when several
+ * signals trigger).  urgent != 0 waives profitability (the urgent path).  gamma = 0 therefore admits only
+ * urgent transitions.  *admit gets 0 or 1, *payback_steps (optional) the ratio, +inf when delta_l <= 0.
+ * Errors: ARG (negative cost, gamma outside [0, 1], negative horizon, null admit). */
+int nereus_admit(double l_tran, double l_step_current, double l_step_target, double gamma, double h_x,
+                 int urgent, int* admit, double* payback_steps);
+
+/* H_x: an exponential moving average of the intervals (in steps) between threshold crossings of one signal,
+ * updated at crossings only; one step before the first interval is observed (Section 4.3).  The paper does
+ * not give the averaging weight; `weight` in (0, 1] is the share of the newest interval (this build's
+ * default reading: 0.5).  The first observed interval replaces the initial value. */
+typedef struct { double h_steps; double weight; int observed; } nereus_horizon_t;
+int nereus_horizon_init(nereus_horizon_t* h, double weight);
+int nereus_horizon_crossing(nereus_horizon_t* h, double interval_steps);
 
 /* ---- execution without allocation --------------------------------------------------------------------- */
 

@@ -58,6 +58,19 @@ class Rect(ctypes.Structure):
                 ("replicas", ctypes.c_int32), ("replica_stride", ctypes.c_int32)]
 
 
+class Horizon(ctypes.Structure):
+    """nereus_horizon_t: the EMA of crossing intervals H_x."""
+    _fields_ = [("h_steps", ctypes.c_double), ("weight", ctypes.c_double), ("observed", ctypes.c_int)]
+
+    def __init__(self, weight: float = 0.5):
+        super().__init__()
+        _ck(_lib.nereus_horizon_init(ctypes.byref(self), weight), "nereus_horizon_init")
+
+    def crossing(self, interval_steps: float) -> float:
+        _ck(_lib.nereus_horizon_crossing(ctypes.byref(self), interval_steps), "nereus_horizon_crossing")
+        return self.h_steps
+
+
 _vp, _i, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
 _P = ctypes.POINTER
 _SIGS = {
@@ -87,6 +100,11 @@ _SIGS = {
     "nereus_transition_status": [_vp, _P(_i)],
     "nereus_transition_launches": [_vp, _P(ctypes.c_uint64)],
     "nereus_last_cuda_error": [],
+    "nereus_transition_estimate": [_vp, ctypes.c_double, ctypes.c_double, _P(ctypes.c_double)],
+    "nereus_admit": [ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_double, _i,
+                     _P(_i), _P(ctypes.c_double)],
+    "nereus_horizon_init": [_P(Horizon), ctypes.c_double],
+    "nereus_horizon_crossing": [_P(Horizon), ctypes.c_double],
     "nereus_transition_run_static": [_vp, _P(_vp), _P(_vp), _vp],
 }
 for _name, _args in _SIGS.items():
@@ -230,6 +248,13 @@ class Transition:
         return {"kernel": {1: "nereus_walk_vec", 2: "nereus_walk_ring"}[v.value], "tile_bytes": tb.value,
                 "grid": g.value, "threads": th.value}
 
+    def estimate(self, gbytes_per_s: float, setup_seconds: float = 0.0) -> float:
+        """L_tran in seconds from the table's bytes, a bandwidth and a set-up time."""
+        out = ctypes.c_double()
+        _ck(_lib.nereus_transition_estimate(self._h, gbytes_per_s, setup_seconds, ctypes.byref(out)),
+            "nereus_transition_estimate")
+        return out.value
+
     def prepare(self):
         _ck(_lib.nereus_transition_prepare(self._h), "nereus_transition_prepare")
 
@@ -292,6 +317,14 @@ class Transition:
             self.close()
         except Exception:
             pass
+
+
+def admit(l_tran, l_step_current, l_step_target, gamma=0.5, h_x=1.0, urgent=False):
+    """Eq. 2: returns (admitted, payback period in steps)."""
+    a, pb = _i(), ctypes.c_double()
+    _ck(_lib.nereus_admit(l_tran, l_step_current, l_step_target, gamma, h_x, int(urgent), ctypes.byref(a),
+                          ctypes.byref(pb)), "nereus_admit")
+    return bool(a.value), pb.value
 
 
 def strerror(code: int) -> str:

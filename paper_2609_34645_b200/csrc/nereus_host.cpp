@@ -492,6 +492,42 @@ int nereus_transition_get_rect(nereus_transition_t t, int index, nereus_rect_t* 
     return NEREUS_OK;
 }
 
+int nereus_transition_estimate(nereus_transition_t t, double gbytes_per_s, double setup_seconds, double* seconds) {
+    if (!t || !seconds || !(gbytes_per_s > 0.0) || !(setup_seconds >= 0.0)) return NEREUS_ERR_ARG;
+    // levels are serial; within a level everything streams at the given bandwidth
+    double bytes = 0.0;
+    for (const Rect& r : t->rects)
+        bytes += (double)(r.rows * (r.width_dst << r.cast)) + (double)(r.rows * r.width_dst) * r.replicas;
+    *seconds = setup_seconds + bytes / (gbytes_per_s * 1e9);
+    return NEREUS_OK;
+}
+
+int nereus_admit(double l_tran, double l_step_current, double l_step_target, double gamma, double h_x, int urgent,
+                 int* admit, double* payback_steps) {
+    if (!admit || !(l_tran >= 0.0) || !(gamma >= 0.0 && gamma <= 1.0) || !(h_x >= 0.0)) return NEREUS_ERR_ARG;
+    const double delta_l = l_step_current - l_step_target;
+    const double inf = 1.0 / 0.0;
+    const double payback = delta_l > 0.0 ? l_tran / delta_l : inf;
+    if (payback_steps) *payback_steps = payback;
+    *admit = urgent ? 1 : (delta_l > 0.0 && payback <= gamma * h_x && gamma > 0.0 ? 1 : 0);
+    return NEREUS_OK;
+}
+
+int nereus_horizon_init(nereus_horizon_t* h, double weight) {
+    if (!h || !(weight > 0.0 && weight <= 1.0)) return NEREUS_ERR_ARG;
+    h->h_steps = 1.0;            // before the first interval is observed
+    h->weight = weight;
+    h->observed = 0;
+    return NEREUS_OK;
+}
+
+int nereus_horizon_crossing(nereus_horizon_t* h, double interval_steps) {
+    if (!h || !(interval_steps >= 0.0) || !(h->weight > 0.0 && h->weight <= 1.0)) return NEREUS_ERR_ARG;
+    h->h_steps = h->observed ? (1.0 - h->weight) * h->h_steps + h->weight * interval_steps : interval_steps;
+    h->observed += 1;
+    return NEREUS_OK;
+}
+
 const char* nereus_strerror(int code) {
     switch (code) {
     case NEREUS_OK:              return "ok";

@@ -916,7 +916,10 @@ int nereus_transition_run(nereus_transition_t t, const void* const* src_ptrs, vo
         WalkParams p;
         p.rects = dv.rects; p.first = dv.first; p.ctrl = dv.ctrl;
         p.n_tiles = dv.n_tiles;
-        for (int k = 0; k < kMaxLevels; ++k) p.level_end[k] = dv.level_end[k];
+        // NEREUS_DEBUG_GATE_BIAS (tests only): raises what a dependency gate waits for, so that it can never
+        // open and the bounded wait must give up with NEREUS_DEV_TIMEOUT
+        const uint32_t gate_bias = (uint32_t)env_int("NEREUS_DEBUG_GATE_BIAS", 0);
+        for (int k = 0; k < kMaxLevels; ++k) p.level_end[k] = dv.level_end[k] + gate_bias;
         fill_params(*t, src_ptrs, dst_ptrs, p);
 
         NEREUS_CUDA(cudaMemsetAsync(dv.ctrl, 0, sizeof(Ctrl), stream));

@@ -355,3 +355,20 @@ def test_state_with_optimizer_tensors():
     rd, wr = t.bytes()
     theta = d.compile(B.Plan(*a), B.Plan(*b)).bytes()[0]
     assert rd == wr == theta * (1 + 2 * 2)            # fp32 moments are twice the bf16 parameters, each
+
+
+def test_buffer_limit_of_one_launch():
+    """One launch addresses at most 448 buffers (its parameter block): a fused table at the limit compiles, one
+    beyond it is refused; so is a single transition with more shards than that."""
+    d = desc_of(I.MICRO)
+    part = d.compile(B.Plan(8, 8), B.Plan(8, 4))                 # 64 + 32 buffers
+    ok = B.Transition.fuse([part] * 4, chained=False)            # 384
+    assert ok.num_buffers() == (256, 128)
+    small = d.compile(B.Plan(8, 4), B.Plan(8, 4))                # 32 + 32
+    assert B.Transition.fuse([part] * 4 + [small], chained=False).num_buffers() == (288, 160)   # 448
+    with pytest.raises(B.NereusError) as e:
+        B.Transition.fuse([part] * 5, chained=False)             # 480
+    assert e.value.code == B.ERR_UNSUPPORTED
+    with pytest.raises(B.NereusError) as e:
+        d.compile_replicated(B.Plan(8, 8), B.Plan(8, 8), 7)      # 64 + 448
+    assert e.value.code == B.ERR_UNSUPPORTED

@@ -133,6 +133,25 @@ def _check_plain_workload(name):
     return rd, wr
 
 
+def test_8b_identity_is_one_16gb_run():
+    """Degenerate transition: equal plans collapse to a single contiguous run of 16 GB (the 8B shape has no
+    padding), far beyond 32-bit byte offsets; the copy must be the identity."""
+    sh = I.LLAMA_8B
+    _need(2 * 16_060_522_496)
+    d = B.ModelDesc(sh.layers, sh.hidden, sh.heads, sh.kv_heads, sh.ffn, sh.vocab, B.BF16)
+    t = d.compile(B.Plan(1, 1), B.Plan(1, 1))
+    assert len(t.rects()) == 1 and t.rects()[0].width_bytes_dst == 16_060_522_496
+    src = I.make_shards(d.shard_sizes(B.Plan(1, 1)), "bf16", 99, "cuda")
+    dst = I.sentinel_shards(d.shard_sizes(B.Plan(1, 1)), "cuda")
+    stream = torch.cuda.current_stream()
+    t.run([src[0].data_ptr()], [dst[0].data_ptr()], stream.cuda_stream)
+    stream.synchronize()
+    assert t.status() == B.DEV_OK
+    assert torch.equal(src[0], dst[0])
+    del src, dst
+    torch.cuda.empty_cache()
+
+
 def test_8b_split_tp1pp1_to_tp4pp2():
     rd, wr = _check_plain_workload("8b_tp1pp1_to_tp4pp2")
     assert rd == wr == 16_062_119_936

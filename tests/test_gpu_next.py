@@ -131,3 +131,27 @@ def test_8b_state_with_adam_full_size():
     assert rd == wr == 5 * (8_030_261_248 * 2 + 65 * 8192 * 3)       # theta bf16 + two fp32 moments = 5x
     del srcs, dsts, s, d
     torch.cuda.empty_cache()
+
+
+def test_transition_estimate_predicts_the_measured_time():
+    """L_tran from bytes and a bandwidth, held against CUDA-event time: with the bandwidth one workload
+    measured (the 4-layer 8B Split), the estimate of another (its Merge back) is within 10% of its time."""
+    def timed(name):
+        wl, t, srcs, dsts, _ = bench.build_workload(name, torch.device("cuda"), dict(
+            tile_bytes=0, ctas_per_sm=0, threads=0, variant=0))
+        stream = torch.cuda.current_stream()
+        sp, dp = [b.data_ptr() for b in srcs], [b.data_ptr() for b in dsts]
+        for _ in range(3):
+            t.run(sp, dp, stream.cuda_stream)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(5):
+            t.run(sp, dp, stream.cuda_stream)
+        b.record(stream)
+        stream.synchronize()
+        return t, a.elapsed_time(b) / 5 / 1e3
+    t1, s1 = timed("8b4l_tp1pp1_to_tp4pp2")
+    gbps = sum(t1.bytes()) / 1e9 / s1
+    t2, s2 = timed("8b4l_tp4pp2_to_tp1pp1")
+    assert t2.estimate(gbps, 0.0) == pytest.approx(s2, rel=0.10)
+    torch.cuda.empty_cache()

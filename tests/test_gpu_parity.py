@@ -196,3 +196,34 @@ def test_run_errors_on_device_pointers():
     assert ch.run_raw(sp, dst.ptrs() + sp) == B.OK
     torch.cuda.synchronize()
     assert ch.status() == B.DEV_OK
+
+
+@pytest.mark.parametrize("variant", [1, 2])
+def test_dependency_wait_gives_up_with_a_status(variant, monkeypatch):
+    """Failure detection without a GPU fault: a gate that nothing will ever open (the debug bias raises its
+    target) makes the bounded wait run out; the kernel returns, the host reads NEREUS_DEV_TIMEOUT, level 0 is
+    complete, level 1 never wrote, and the context stays usable."""
+    sh = I.SMALL
+    d = G.desc_of(sh)
+    a, b = (2, 2), (4, 1)
+    ab, ba = d.compile(B.Plan(*a), B.Plan(*b)), d.compile(B.Plan(*b), B.Plan(*a))
+    t = B.Transition.fuse([ab, ba], chained=True)
+    t.tune(variant=variant)
+    src = G.device_sources(d, B.Plan(*a), "bf16", 8)
+    mid = G.Guarded([t.buffer_bytes(True, j) for j in range(4)])
+    back = G.Guarded([t.buffer_bytes(True, 4 + j) for j in range(4)])
+    stream = torch.cuda.current_stream()
+    monkeypatch.setenv("NEREUS_DEBUG_GATE_BIAS", "1000000")
+    t.run([s.data_ptr() for s in src], mid.ptrs() + back.ptrs(), stream.cuda_stream)
+    stream.synchronize()                                       # returns: the wait is bounded
+    assert t.status() == B.DEV_TIMEOUT
+    want = G.oracle_expected(sh, a, b, "bf16", "bf16", False, [s.cpu().numpy() for s in src])
+    for g, w in zip(mid.bufs, want):
+        assert np.array_equal(g.cpu().numpy(), w)              # level 0 ran to completion
+    for r in back.raw:
+        assert bool((r == G.SENTINEL).all())                   # nothing of level 1 was written
+    monkeypatch.delenv("NEREUS_DEBUG_GATE_BIAS")
+    G.run_transition(t, src, mid.bufs + back.bufs)             # same handle, same context: works again
+    for g, s in zip(back.bufs, src):
+        assert torch.equal(g, s)                               # the round trip restores the source bits
+    assert t.status() == B.DEV_OK

@@ -50,6 +50,9 @@
  *     rows, then its V rows; inside gate/up the rank's gate rows, then its up
  *     rows.  The buffer length is the end of the last tensor rounded up to
  *     256 bytes.  Padding bytes are never read and never written.
+ *   layout variants of a plan (order inside a rank's fused block only):
+ *     grouped QKV: for each kv head of the rank, its q heads, its k head, its v head;
+ *     interleaved gate/up: g0, u0, g1, u1, ... row by row.
  */
 #include <stdint.h>
 #include <stdlib.h>
@@ -68,7 +71,12 @@ typedef struct {
     int value_head;   /* 0: LM head [V, H]; 1: value head [1, H] */
 } oracle_model;
 
-typedef struct { int tp, pp, dtype; } oracle_plan;
+/* layout: bit 0 set = fused QKV stored group by group inside a rank's block (for each of the rank's kv heads: its
+ * q heads, then its k head, then its v head) instead of [all Q; all K; all V]; bit 1 set = gate and up rows
+ * interleaved row by row inside a rank's block (g0, u0, g1, u1, ...) instead of [all gate; all up].  Which
+ * heads and rows a rank holds does not depend on the layout, only their order inside the fused block. */
+enum { ORACLE_QKV_GROUPED = 1, ORACLE_GATE_UP_INTERLEAVED = 2 };
+typedef struct { int tp, pp, dtype, layout; } oracle_plan;
 
 /* kinds of logical tensor */
 enum { K_EMBED, K_LN1, K_WQ, K_WK, K_WV, K_WO, K_LN2, K_WGATE, K_WUP, K_WDOWN, K_LNF, K_HEAD };
@@ -117,7 +125,7 @@ int oracle_logical_shape(const oracle_model* m, int64_t id, int64_t* rows, int64
 }
 
 int oracle_check_plan(const oracle_model* m, oracle_plan p) {
-    if (!m || p.tp < 1 || p.pp < 1) return ORACLE_ERR_ARG;
+    if (!m || p.tp < 1 || p.pp < 1 || (p.layout & ~3)) return ORACLE_ERR_ARG;
     if (m->L < 1 || m->H < 1 || m->nq < 1 || m->nkv < 1 || m->F < 1 || m->V < 1) return ORACLE_ERR_ARG;
     if (m->H % m->nq || m->nq % m->nkv) return ORACLE_ERR_INDIVISIBLE;
     if (p.tp > m->nkv) return ORACLE_ERR_UNSUPPORTED;      /* no KV-head replication */
@@ -156,6 +164,29 @@ static int64_t rank_elems(const oracle_model* m, int kind, int64_t t) {
     return nr * nc;
 }
 
+/* Row of the fused stored block (counted from the block's first row) that holds local row i of the rank's
+ * part of logical tensor `kind`.  Tensors that are stored alone have row i at row i. */
+static int64_t part_rowpos(const oracle_model* m, oracle_plan pl, int kind, int64_t i) {
+    int64_t hd = m->H / m->nq, G = m->nq / m->nkv, t = pl.tp;
+    int64_t qr = m->nq * hd / t, kr = m->nkv * hd / t, fr = m->F / t;
+    if (kind == K_WQ || kind == K_WK || kind == K_WV) {
+        if (pl.layout & ORACLE_QKV_GROUPED) {
+            int64_t head = i / hd, within = i % hd, group_rows = (G + 2) * hd;
+            if (kind == K_WQ) return (head / G) * group_rows + (head % G) * hd + within;
+            if (kind == K_WK) return head * group_rows + G * hd + within;
+            return head * group_rows + (G + 1) * hd + within;
+        }
+        if (kind == K_WQ) return i;
+        if (kind == K_WK) return qr + i;
+        return qr + kr + i;
+    }
+    if (kind == K_WGATE || kind == K_WUP) {
+        if (pl.layout & ORACLE_GATE_UP_INTERLEAVED) return 2 * i + (kind == K_WUP ? 1 : 0);
+        return kind == K_WGATE ? i : fr + i;
+    }
+    return i;
+}
+
 /* Walk the packing order of shard (stage p, any TP rank) and return the byte
  * offset of the first element of logical tensor (kind, layer), or -1 if the
  * stage does not hold it.  *total gets the shard buffer length. */
@@ -173,24 +204,20 @@ static int64_t pack_offset(const oracle_model* m, oracle_plan pl, int64_t p,
         cur = align256(cur);                                    /* ln1 */
         if (hit && want_kind == K_LN1) found = cur;
         cur += rank_elems(m, K_LN1, t) * es;
-        cur = align256(cur);                                    /* fused q;k;v */
-        if (hit && want_kind == K_WQ) found = cur;
-        cur += rank_elems(m, K_WQ, t) * es;
-        if (hit && want_kind == K_WK) found = cur;
-        cur += rank_elems(m, K_WK, t) * es;
-        if (hit && want_kind == K_WV) found = cur;
-        cur += rank_elems(m, K_WV, t) * es;
+        cur = align256(cur);                                    /* fused q;k;v: row 0 of each part */
+        if (hit && (want_kind == K_WQ || want_kind == K_WK || want_kind == K_WV))
+            found = cur + part_rowpos(m, pl, want_kind, 0) * m->H * es;
+        cur += (rank_elems(m, K_WQ, t) + rank_elems(m, K_WK, t) + rank_elems(m, K_WV, t)) * es;
         cur = align256(cur);                                    /* wo */
         if (hit && want_kind == K_WO) found = cur;
         cur += rank_elems(m, K_WO, t) * es;
         cur = align256(cur);                                    /* ln2 */
         if (hit && want_kind == K_LN2) found = cur;
         cur += rank_elems(m, K_LN2, t) * es;
-        cur = align256(cur);                                    /* fused gate;up */
-        if (hit && want_kind == K_WGATE) found = cur;
-        cur += rank_elems(m, K_WGATE, t) * es;
-        if (hit && want_kind == K_WUP) found = cur;
-        cur += rank_elems(m, K_WUP, t) * es;
+        cur = align256(cur);                                    /* fused gate;up: row 0 of each part */
+        if (hit && (want_kind == K_WGATE || want_kind == K_WUP))
+            found = cur + part_rowpos(m, pl, want_kind, 0) * m->H * es;
+        cur += (rank_elems(m, K_WGATE, t) + rank_elems(m, K_WUP, t)) * es;
         cur = align256(cur);                                    /* wdown */
         if (hit && want_kind == K_WDOWN) found = cur;
         cur += rank_elems(m, K_WDOWN, t) * es;
@@ -224,9 +251,10 @@ int oracle_shard_bytes(const oracle_model* m, oracle_plan pl, int64_t shard, int
 
 /* Where shard `shard` of plan `pl` keeps its part of logical tensor `id`:
  * byte offset of the part's first element in the shard buffer, and the part's
- * position [r0, r0+nr) x [c0, c0+nc) in the full tensor.  The part is stored
- * row-major with nc elements per row.  *held = 0 when the shard's stage does
- * not own the tensor. */
+ * position [r0, r0+nr) x [c0, c0+nc) in the full tensor.  Each row of the part
+ * is nc contiguous elements; row i starts oracle_part_row(i) * nc elements
+ * after row 0 (i itself unless the plan's layout interleaves the fused block).
+ * *held = 0 when the shard's stage does not own the tensor. */
 int oracle_locate(const oracle_model* m, oracle_plan pl, int64_t shard, int64_t id,
                   int* held, int64_t* offset, int64_t* r0, int64_t* nr, int64_t* c0, int64_t* nc) {
     int kind; int64_t layer, off;
@@ -241,6 +269,13 @@ int oracle_locate(const oracle_model* m, oracle_plan pl, int64_t shard, int64_t 
     rank_part(m, kind, shard % pl.tp, pl.tp, r0, nr, c0, nc);
     if (!*held) { *nr = 0; *nc = 0; }
     return ORACLE_OK;
+}
+
+/* Distance, in rows of nc elements, from row 0 of a rank's part of logical tensor `id` to its row i. */
+int64_t oracle_part_row(const oracle_model* m, oracle_plan pl, int64_t id, int64_t i) {
+    int kind; int64_t layer;
+    decode_id(m, id, &kind, &layer);
+    return part_rowpos(m, pl, kind, i) - part_rowpos(m, pl, kind, 0);
 }
 
 /* fp32 -> bf16, round to nearest, ties to even, on the bit pattern.
@@ -290,9 +325,11 @@ int oracle_reshard_tensor_parts(const oracle_model* m, oracle_plan sp, oracle_pl
             }
             continue;
         }
-        for (int64_t i = 0; i < nr; ++i)
+        for (int64_t i = 0; i < nr; ++i) {
+            int64_t at = oracle_part_row(m, sp, id, i);                 /* where the plan's layout keeps row i */
             for (int64_t j = 0; j < nc; ++j)
-                memcpy(full + ((r0 + i) * cols + (c0 + j)) * ses, part + (i * nc + j) * ses, (size_t)ses);
+                memcpy(full + ((r0 + i) * cols + (c0 + j)) * ses, part + (at * nc + j) * ses, (size_t)ses);
+        }
         first_replica = 0;
     }
 
@@ -315,9 +352,11 @@ int oracle_reshard_tensor_parts(const oracle_model* m, oracle_plan sp, oracle_pl
         if (!held) continue;
         unsigned char* part = (unsigned char*)dst_parts[d];
         if (!part) { if (cast != full) free(cast); free(full); return ORACLE_ERR_ARG; }
-        for (int64_t i = 0; i < nr; ++i)
+        for (int64_t i = 0; i < nr; ++i) {
+            int64_t at = oracle_part_row(m, dp, id, i);
             for (int64_t j = 0; j < nc; ++j)
-                memcpy(part + (i * nc + j) * des, cast + ((r0 + i) * cols + (c0 + j)) * des, (size_t)des);
+                memcpy(part + (at * nc + j) * des, cast + ((r0 + i) * cols + (c0 + j)) * des, (size_t)des);
+        }
     }
     if (cast != full) free(cast);
     free(full);

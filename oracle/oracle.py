@@ -25,6 +25,8 @@ _LIB = os.path.join(_HERE, "libnereus_oracle.so")
 
 BF16 = 1
 FP32 = 2
+QKV_GROUPED = 1
+GATE_UP_INTERLEAVED = 2
 
 OK = 0
 ERR_ARG = -1
@@ -57,7 +59,7 @@ class _Model(ctypes.Structure):
 
 
 class _Plan(ctypes.Structure):
-    _fields_ = [("tp", ctypes.c_int), ("pp", ctypes.c_int), ("dtype", ctypes.c_int)]
+    _fields_ = [("tp", ctypes.c_int), ("pp", ctypes.c_int), ("dtype", ctypes.c_int), ("layout", ctypes.c_int)]
 
 
 @dataclass(frozen=True)
@@ -81,9 +83,10 @@ class Plan:
     tp: int
     pp: int
     dtype: int = 0  # 0 = the model's dtype
+    layout: int = 0  # QKV_GROUPED | GATE_UP_INTERLEAVED
 
     def c(self) -> _Plan:
-        return _Plan(self.tp, self.pp, self.dtype)
+        return _Plan(self.tp, self.pp, self.dtype, self.layout)
 
 
 _lib = None
@@ -102,6 +105,8 @@ def lib():
         L.oracle_shard_bytes.argtypes = [p(_Model), _Plan, i64, p(i64)]
         L.oracle_locate.argtypes = [p(_Model), _Plan, i64, i64, p(ctypes.c_int), p(i64), p(i64), p(i64),
                                     p(i64), p(i64)]
+        L.oracle_part_row.restype = i64
+        L.oracle_part_row.argtypes = [p(_Model), _Plan, i64, i64]
         L.oracle_rne_bf16.restype = ctypes.c_uint16
         L.oracle_rne_bf16.argtypes = [ctypes.c_uint32]
         L.oracle_rne_bf16_array.restype = None
@@ -172,6 +177,12 @@ def locate(model: Model, plan: Plan, shard: int, tid: int) -> Part:
     _check(lib().oracle_locate(ctypes.byref(m), plan.c(), shard, tid, ctypes.byref(held),
                                *[ctypes.byref(x) for x in v]), "locate")
     return Part(bool(held.value), *[x.value for x in v])
+
+
+def part_row(model: Model, plan: Plan, tid: int, i: int) -> int:
+    """Rows between row 0 and row i of a rank's part of logical tensor tid under the plan's layout."""
+    m = model.c()
+    return int(lib().oracle_part_row(ctypes.byref(m), plan.c(), tid, i))
 
 
 def rne_bf16(u: int) -> int:
@@ -249,7 +260,7 @@ def reshard_state(model: Model, src: Plan, dst: Plan, n_opt: int, src_bufs: list
     out = reshard(model, src, dst, src_bufs[:ns], fill=fill)
     m32 = Model(model.layers, model.hidden, model.heads, model.kv_heads, model.ffn, model.vocab, FP32,
                 model.value_head)
-    s32, d32 = Plan(src.tp, src.pp, FP32), Plan(dst.tp, dst.pp, FP32)
+    s32, d32 = Plan(src.tp, src.pp, FP32, src.layout), Plan(dst.tp, dst.pp, FP32, dst.layout)
     for k in range(n_opt):
         out += reshard(m32, s32, d32, src_bufs[ns * (1 + k):ns * (2 + k)], fill=fill)
     return out

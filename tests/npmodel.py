@@ -61,8 +61,15 @@ def position_coded(sh, es, salt, value_head=False):
     return out
 
 
-def _stored_blocks(sh, tp, pp, p, r, logical, value_head):
-    """The tensors shard (p, r) stores, in packing order, as numpy arrays (np.split formulation)."""
+QKV_GROUPED, GATE_UP_INTERLEAVED = 1, 2
+
+
+def _stored_blocks(sh, tp, pp, p, r, logical, value_head, layout=0):
+    """The tensors shard (p, r) stores, in packing order, as numpy arrays (np.split formulation).  Layout
+    variants reorder rows inside a rank's fused block: grouped QKV = per kv head [its q heads; k; v] (a reshape
+    to [kv_heads, rows per head group, H]); interleaved gate/up = np.stack of the two row sets."""
+    hd = sh.hidden // sh.heads
+    G = sh.heads // sh.kv_heads
     def d0(x):
         return np.split(x, tp, axis=0)[r]
 
@@ -76,10 +83,20 @@ def _stored_blocks(sh, tp, pp, p, r, logical, value_head):
     for l in range(p * lps, (p + 1) * lps):
         g = lambda k: logical[f"{k}.{l}"]
         blocks.append(g("ln1"))
-        blocks.append(np.concatenate([d0(g("wq")), d0(g("wk")), d0(g("wv"))], axis=0))
+        if layout & QKV_GROUPED:
+            q = g("wq").reshape(sh.kv_heads, G * hd, sh.hidden)
+            k = g("wk").reshape(sh.kv_heads, hd, sh.hidden)
+            v = g("wv").reshape(sh.kv_heads, hd, sh.hidden)
+            mine = range(r * sh.kv_heads // tp, (r + 1) * sh.kv_heads // tp)
+            blocks.append(np.concatenate([np.concatenate([q[h], k[h], v[h]], axis=0) for h in mine], axis=0))
+        else:
+            blocks.append(np.concatenate([d0(g("wq")), d0(g("wk")), d0(g("wv"))], axis=0))
         blocks.append(d1(g("wo")))
         blocks.append(g("ln2"))
-        blocks.append(np.concatenate([d0(g("wgate")), d0(g("wup"))], axis=0))
+        if layout & GATE_UP_INTERLEAVED:
+            blocks.append(np.stack([d0(g("wgate")), d0(g("wup"))], axis=1).reshape(-1, sh.hidden))
+        else:
+            blocks.append(np.concatenate([d0(g("wgate")), d0(g("wup"))], axis=0))
         blocks.append(d1(g("wdown")))
     if p == pp - 1:
         blocks.append(logical["ln_f"])
@@ -87,13 +104,13 @@ def _stored_blocks(sh, tp, pp, p, r, logical, value_head):
     return blocks
 
 
-def build_shards(sh, tp, pp, logical, value_head=False, pad=0xA5):
+def build_shards(sh, tp, pp, logical, value_head=False, pad=0xA5, layout=0):
     """Shard byte images (uint8 arrays), index = p * tp + r."""
     out = []
     for p in range(pp):
         for r in range(tp):
             chunks, cur = [], 0
-            for b in _stored_blocks(sh, tp, pp, p, r, logical, value_head):
+            for b in _stored_blocks(sh, tp, pp, p, r, logical, value_head, layout):
                 start = -(-cur // 256) * 256
                 if start > cur:
                     chunks.append(np.full(start - cur, pad, np.uint8))
@@ -107,7 +124,7 @@ def build_shards(sh, tp, pp, logical, value_head=False, pad=0xA5):
     return out
 
 
-def owner(sh, tp, pp, es, name, i, j, value_head=False):
+def owner(sh, tp, pp, es, name, i, j, value_head=False, layout=0):
     """Per-element statement of the contract: every (shard, byte offset) that holds element (i, j) of the
     logical tensor ``name`` (several for replicated tensors)."""
     hd = sh.hidden // sh.heads
@@ -161,6 +178,14 @@ def owner(sh, tp, pp, es, name, i, j, value_head=False):
     start = within_layer(blk)(base)
     if kind in ("ln1", "ln2"):
         return [(p * tp + r, start + j * es) for r in range(tp)]
+    if kind in ("wq", "wk", "wv") and layout & QKV_GROUPED:
+        G = nq // nkv
+        head = i // hd
+        kv = head // G if kind == "wq" else head              # the kv head whose group the row belongs to
+        r = kv // (nkv // tp)
+        row = (kv % (nkv // tp)) * (G + 2) * hd                 # earlier groups of this rank
+        row += {"wq": (head % G) * hd, "wk": G * hd, "wv": (G + 1) * hd}[kind] + i % hd
+        return [(p * tp + r, start + (row * H + j) * es)]
     if kind == "wq":
         r = i // qr
         return [(p * tp + r, start + ((i % qr) * H + j) * es)]
@@ -168,6 +193,9 @@ def owner(sh, tp, pp, es, name, i, j, value_head=False):
         r = i // kr
         skip = qr + (kr if kind == "wv" else 0)
         return [(p * tp + r, start + ((skip + i % kr) * H + j) * es)]
+    if kind in ("wgate", "wup") and layout & GATE_UP_INTERLEAVED:
+        r = i // fr
+        return [(p * tp + r, start + ((2 * (i % fr) + (kind == "wup")) * H + j) * es)]
     if kind in ("wgate", "wup"):
         r = i // fr
         skip = fr if kind == "wup" else 0

@@ -132,6 +132,42 @@ def test_any_plan_pair_against_np_split():
             assert np.array_equal(g, w), (a, b)
 
 
+@pytest.mark.parametrize("sh", [I.TINY, I.MICRO])
+def test_layout_variants_against_np(sh):
+    """Grouped QKV and row-interleaved gate/up on either side: shards built by numpy (reshape to head groups,
+    np.stack of the row sets) for every combination of source and target layout."""
+    m = model_of(sh)
+    logical = npmodel.random_logical(sh, 2, seed=31)
+    pls = [p for p in plans_for(sh) if p in ((1, 1), (2, 1), (2, 2), (4, 2), (8, 1))]
+    for la, lb in itertools.product(range(4), repeat=2):
+        for a, b in itertools.product(pls, repeat=2):
+            src = npmodel.build_shards(sh, a[0], a[1], logical, layout=la)
+            want = npmodel.build_shards(sh, b[0], b[1], logical, layout=lb)
+            got = O.reshard(m, O.Plan(a[0], a[1], 0, la), O.Plan(b[0], b[1], 0, lb), src, fill=0xA5)
+            for g, w in zip(got, want):
+                assert np.array_equal(g, w), (la, lb, a, b)
+
+
+def test_layout_variant_sizes_and_cast():
+    """The layout changes the order inside a rank's block, never what a rank holds: shard sizes are equal; the
+    cast commutes with a layout conversion."""
+    sh = I.SMALL
+    m32 = model_of(sh, O.FP32)
+    for pl in ((2, 2), (4, 1)):
+        for lay in range(4):
+            for s in range(pl[0] * pl[1]):
+                assert O.shard_bytes(m32, O.Plan(pl[0], pl[1], 0, lay), s) == O.shard_bytes(m32, O.Plan(*pl), s)
+    logical = npmodel.random_logical(sh, 4, seed=3)
+    for n in logical:                                           # keep the fp32 payload finite and not NaN
+        logical[n] = (logical[n] & np.uint32(0x3FFFFFFF)) | np.uint32(0x30000000)
+    src = npmodel.build_shards(sh, 2, 2, logical, layout=3)     # Megatron-style training layout, fp32
+    got = O.reshard(m32, O.Plan(2, 2, 0, 3), O.Plan(4, 1, O.BF16, 0), src, fill=0xA5)
+    cast = {n: torch.from_numpy(x.view(np.float32)).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+            for n, x in logical.items()}
+    for g, w in zip(got, npmodel.build_shards(sh, 4, 1, cast, layout=0)):
+        assert np.array_equal(g, w)
+
+
 # ---------------------------------------------------------------- brute-force owner function
 
 @pytest.mark.parametrize("es", [2, 4])
@@ -145,13 +181,13 @@ def test_owner_brute_force(es, vh):
     for salt in (1, 2, 3):
         logical = npmodel.position_coded(sh, es, salt, vh)
         src = npmodel.build_shards(sh, 1, 1, logical, vh)
-        for tp, pp in [(2, 1), (1, 2), (2, 2)]:
-            dst = O.reshard(m, O.Plan(1, 1), O.Plan(tp, pp), src)
+        for tp, pp, lay in [(2, 1, 0), (1, 2, 0), (2, 2, 0), (2, 1, 3), (1, 1, 1), (2, 2, 2)]:
+            dst = O.reshard(m, O.Plan(1, 1), O.Plan(tp, pp, 0, lay), src)
             seen = [np.zeros(d.size, np.uint8) for d in dst]
             for name, x in logical.items():
                 for i in range(x.shape[0]):
                     for j in range(x.shape[1]):
-                        for shard, off in npmodel.owner(sh, tp, pp, es, name, i, j, vh):
+                        for shard, off in npmodel.owner(sh, tp, pp, es, name, i, j, vh, lay):
                             assert dst[shard][off:off + es].view(dt)[0] == x[i, j], (name, i, j, tp, pp)
                             seen[shard][off:off + es] += 1
             for s, mask in enumerate(payload_mask(m, O.Plan(tp, pp))):

@@ -140,7 +140,8 @@ def build_workload(name, device, tune):
         sh = st.shape
         d = B.ModelDesc(sh.layers, sh.hidden, sh.heads, sh.kv_heads, sh.ffn, sh.vocab, B.DTYPES[st.src[2]],
                         st.value_head)
-        pa, pb = B.Plan(st.src[0], st.src[1], B.DTYPES[st.src[2]]), B.Plan(st.dst[0], st.dst[1], B.DTYPES[st.dst[2]])
+        pa = B.Plan(st.src[0], st.src[1], B.DTYPES[st.src[2]], I.layout_of(st.src))
+        pb = B.Plan(st.dst[0], st.dst[1], B.DTYPES[st.dst[2]], I.layout_of(st.dst))
         if st.replicas > 1:
             t = d.compile_replicated(pa, pb, st.replicas)
         elif st.n_opt:
@@ -165,7 +166,7 @@ def build_workload(name, device, tune):
 
         srcs += tied_sources(pa, st.src[2], st.seed)
         for k in range(st.n_opt):                      # optimizer tensors: fp32, same (tp, pp)
-            srcs += tied_sources(B.Plan(pa.tp, pa.pp, B.FP32), "fp32", st.seed * 101 + k)
+            srcs += tied_sources(B.Plan(pa.tp, pa.pp, B.FP32, pa.layout), "fp32", st.seed * 101 + k)
         n_dst = t.num_buffers()[1]
         dsts += I.sentinel_shards([t.buffer_bytes(True, j) for j in range(n_dst)], device)
         parts.append(t)
@@ -202,7 +203,8 @@ def oracle_sample(workload_name, layers, device_srcs=None):
     sh = st.shape
     odt = {"bf16": O.BF16, "fp32": O.FP32}
     m = O.Model(sh.layers, sh.hidden, sh.heads, sh.kv_heads, sh.ffn, sh.vocab, odt[st.src[2]], st.value_head)
-    pa, pb = O.Plan(st.src[0], st.src[1]), O.Plan(st.dst[0], st.dst[1], odt[st.dst[2]])
+    pa = O.Plan(st.src[0], st.src[1], 0, I.layout_of(st.src))
+    pb = O.Plan(st.dst[0], st.dst[1], odt[st.dst[2]], I.layout_of(st.dst))
     layers = max(1, min(layers, sh.layers))
     ses, des = I.element_size(st.src[2]), I.element_size(st.dst[2])
     total_s, total_bytes = 0.0, 0

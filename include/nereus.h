@@ -42,6 +42,7 @@
  *            of the last tensor rounded up to 256 bytes.  Padding bytes are never read and never written.
  *   stored tensor ids (argument tensor_id below): 0 = embed; 1 + 6*l + k for layer l and
  *            k = 0 ln1, 1 qkv, 2 wo, 3 ln2, 4 gate_up, 5 wdown; 1 + 6*L = ln_f; 2 + 6*L = head.
+ *   layout variants (nereus_plan_t.layout) reorder the rows inside qkv and gate_up, see the flags below.
  *   required: tp | nkv, tp | F, tp | V, pp | L, tp <= nkv (no KV-head replication), and every contiguous piece
  *            a transition moves must start on and span a multiple of 16 bytes on both sides (for the cast: 8
  *            elements).
@@ -78,8 +79,17 @@ typedef enum { NEREUS_BF16 = 1, NEREUS_FP32 = 2 } nereus_dtype_t;
 typedef struct nereus_model_desc_s* nereus_model_desc_t;   /* opaque, host */
 typedef struct nereus_transition_s* nereus_transition_t;   /* opaque, host; owns the task table */
 
-/* A (TP, PP) layout.  dtype 0 means "the descriptor's dtype". */
-typedef struct { int tp; int pp; int dtype; } nereus_plan_t;
+/* Order of the rows inside a rank's fused blocks (which heads and rows a rank holds never changes):
+ *   NEREUS_QKV_GROUPED          for each kv head of the rank: its q heads, its k head, its v head (the order
+ *                               Megatron-style trainers keep), instead of [all Q ; all K ; all V]
+ *   NEREUS_GATE_UP_INTERLEAVED  g0, u0, g1, u1, ... row by row (what some fused SwiGLU kernels read), instead
+ *                               of [all gate ; all up]
+ * A transition may convert between layouts, e.g. grouped fp32 training weights to blocked bf16 for generation. */
+#define NEREUS_QKV_GROUPED          1
+#define NEREUS_GATE_UP_INTERLEAVED  2
+
+/* A (TP, PP) layout.  dtype 0 means "the descriptor's dtype"; layout is a mask of the flags above. */
+typedef struct { int tp; int pp; int dtype; int layout; } nereus_plan_t;
 
 /* One rect-copy task of a compiled transition, for inspection and tests.  Buffer indices address the
  * concatenation [src_ptrs..., dst_ptrs...] that nereus_transition_run receives ("unified index").

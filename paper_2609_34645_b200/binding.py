@@ -15,6 +15,8 @@ LIB_PATH = os.path.join(_HERE, "libnereus.so")
 BF16 = 1
 FP32 = 2
 DTYPES = {"bf16": BF16, "fp32": FP32}
+QKV_GROUPED = 1
+GATE_UP_INTERLEAVED = 2
 
 OK = 0
 ERR_ARG, ERR_INDIVISIBLE, ERR_UNSUPPORTED, ERR_ALIAS = -1, -2, -3, -4
@@ -39,14 +41,15 @@ class NereusError(RuntimeError):
 
 
 class Plan(ctypes.Structure):
-    """nereus_plan_t: (tp, pp, dtype); dtype 0 = the descriptor's."""
-    _fields_ = [("tp", ctypes.c_int), ("pp", ctypes.c_int), ("dtype", ctypes.c_int)]
+    """nereus_plan_t: (tp, pp, dtype, layout); dtype 0 = the descriptor's; layout = QKV_GROUPED |
+    GATE_UP_INTERLEAVED."""
+    _fields_ = [("tp", ctypes.c_int), ("pp", ctypes.c_int), ("dtype", ctypes.c_int), ("layout", ctypes.c_int)]
 
-    def __init__(self, tp: int, pp: int, dtype: int = 0):
-        super().__init__(tp, pp, dtype)
+    def __init__(self, tp: int, pp: int, dtype: int = 0, layout: int = 0):
+        super().__init__(tp, pp, dtype, layout)
 
     def __repr__(self):
-        return f"Plan(tp={self.tp}, pp={self.pp}, dtype={self.dtype})"
+        return f"Plan(tp={self.tp}, pp={self.pp}, dtype={self.dtype}, layout={self.layout})"
 
 
 class Rect(ctypes.Structure):

@@ -46,6 +46,7 @@ void build_catalogue(nereus_model_desc_s& d) {
 int check_plan(const nereus_model_desc_s& d, nereus_plan_t p) {
     if (p.tp < 1 || p.pp < 1) return NEREUS_ERR_ARG;
     if (p.dtype != 0 && p.dtype != NEREUS_BF16 && p.dtype != NEREUS_FP32) return NEREUS_ERR_ARG;
+    if (p.layout & ~(NEREUS_QKV_GROUPED | NEREUS_GATE_UP_INTERLEAVED)) return NEREUS_ERR_ARG;
     if (p.tp > d.nkv) return NEREUS_ERR_UNSUPPORTED;
     if (d.nkv % p.tp || d.nq % p.tp || d.F % p.tp || d.V % p.tp || d.L % p.pp) return NEREUS_ERR_INDIVISIBLE;
     return NEREUS_OK;
@@ -91,6 +92,44 @@ void stage_layout(const nereus_model_desc_s& d, nereus_plan_t p, int stage, Stag
 // ---------------------------------------------------------------------------------------------------
 
 namespace {
+
+// One run of consecutive logical rows of one segment of a Rows-cut tensor as a TP rank stores it:
+// logical rows [lo, lo + n) of segment `seg` sit at stored rows at, at + step, at + 2*step, ...
+struct RowPiece {
+    int     seg;
+    int64_t lo, n;
+    int64_t at, step;
+};
+
+// How rank r of t keeps a Rows-cut tensor under a layout.  Blocked: one piece per segment, stacked.
+// Grouped QKV (3 segments, q heads = G per kv head): per kv head of the rank, G*hd rows of Q, hd of K, hd of V.
+// Interleaved gate/up (2 segments): rows alternate, step 2.
+void row_pieces(const nereus_model_desc_s& d, const StoredTensor& x, int layout, int r, int t,
+                std::vector<RowPiece>& out) {
+    out.clear();
+    if (x.nseg == 3 && (layout & NEREUS_QKV_GROUPED)) {
+        const int64_t hd = d.H / d.nq, G = d.nq / d.nkv, per = d.nkv / t, group_rows = (G + 2) * hd;
+        for (int64_t j = 0; j < per; ++j) {
+            const int64_t g = (int64_t)r * per + j;                 // global kv head
+            out.push_back({0, g * G * hd, G * hd, j * group_rows, 1});
+            out.push_back({1, g * hd, hd, j * group_rows + G * hd, 1});
+            out.push_back({2, g * hd, hd, j * group_rows + (G + 1) * hd, 1});
+        }
+        return;
+    }
+    if (x.nseg == 2 && (layout & NEREUS_GATE_UP_INTERLEAVED)) {
+        const int64_t n = x.seg_rows[0] / t;
+        out.push_back({0, (int64_t)r * n, n, 0, 2});
+        out.push_back({1, (int64_t)r * n, n, 1, 2});
+        return;
+    }
+    int64_t base = 0;
+    for (int s = 0; s < x.nseg; ++s) {
+        const int64_t n = x.seg_rows[s] / t;
+        out.push_back({s, (int64_t)r * n, n, base, 1});
+        base += n;
+    }
+}
 
 struct Emitter {
     std::vector<Rect>& out;
@@ -145,6 +184,7 @@ static int compile_one(const nereus_model_desc_s& d, nereus_plan_t sp, nereus_pl
     t.n_levels = 1;
 
     Emitter em{t.rects};
+    std::vector<RowPiece> spieces, dpieces;
     const int ts = sp.tp, td = dp.tp;
     for (int pd = 0; pd < dp.pp; ++pd) {
         for (int rd = 0; rd < td; ++rd) {
@@ -165,22 +205,35 @@ static int compile_one(const nereus_model_desc_s& d, nereus_plan_t sp, nereus_pl
                     r.rows = 1; r.width_dst = (uint64_t)x.seg_rows[0] * x.cols * des;
                     em.emit(r);
                 } else if (x.cut == Cut::Rows) {
-                    // each stacked segment is cut by rows on both sides: intersect row intervals
-                    uint64_t sbase = 0, dbase = 0;       // rows of earlier segments inside the stored block
-                    for (int s = 0; s < x.nseg; ++s) {
-                        const int64_t N = x.seg_rows[s], ns = N / ts, nd = N / td;
-                        const int64_t d0 = rd * nd, d1 = d0 + nd;
-                        for (int rs = 0; rs < ts; ++rs) {
-                            const int64_t s0 = rs * ns, s1 = s0 + ns;
-                            const int64_t lo = std::max(d0, s0), hi = std::min(d1, s1);
-                            if (lo >= hi) continue;
-                            r.src_buf = ps * ts + rs;
-                            r.src_off = soff + (sbase + (uint64_t)(lo - s0)) * x.cols * ses;
-                            r.dst_off = doff + (dbase + (uint64_t)(lo - d0)) * x.cols * des;
-                            r.rows = 1; r.width_dst = (uint64_t)(hi - lo) * x.cols * des;
-                            em.emit(r);
+                    if (ts == td && sp.layout == dp.layout) {
+                        // same cut and same order on both sides: the rank's stored block moves as one run
+                        int64_t brows, bcols;
+                        stored_block(x, td, brows, bcols);
+                        r.src_buf = ps * ts + rd;
+                        r.src_off = soff; r.dst_off = doff;
+                        r.rows = 1; r.width_dst = (uint64_t)brows * bcols * des;
+                        em.emit(r);
+                        continue;
+                    }
+                    // both sides keep runs of logical rows (row pieces): intersect them segment by segment
+                    row_pieces(d, x, dp.layout, rd, td, dpieces);
+                    for (int rs = 0; rs < ts; ++rs) {
+                        row_pieces(d, x, sp.layout, rs, ts, spieces);
+                        for (const RowPiece& q : dpieces) {
+                            for (const RowPiece& s : spieces) {
+                                if (s.seg != q.seg) continue;
+                                const int64_t lo = std::max(q.lo, s.lo), hi = std::min(q.lo + q.n, s.lo + s.n);
+                                if (lo >= hi) continue;
+                                r.src_buf = ps * ts + rs;
+                                r.src_off = soff + (uint64_t)(s.at + (lo - s.lo) * s.step) * x.cols * ses;
+                                r.dst_off = doff + (uint64_t)(q.at + (lo - q.lo) * q.step) * x.cols * des;
+                                r.rows = (uint64_t)(hi - lo);
+                                r.width_dst = (uint64_t)x.cols * des;
+                                r.src_pitch = (uint64_t)s.step * x.cols * ses;
+                                r.dst_pitch = (uint64_t)q.step * x.cols * des;
+                                em.emit(r);       // consecutive rows on both sides collapse to one run
+                            }
                         }
-                        sbase += ns; dbase += nd;
                     }
                 } else {
                     // every row is cut into column pieces on both sides: intersect column intervals
@@ -383,7 +436,7 @@ int nereus_transition_compile_state(nereus_model_desc_t d, nereus_plan_t sp, ner
     nereus_transition_t parts[9] = {nullptr};
     int rc = nereus_transition_compile(d, sp, dp, &parts[0]);
     nereus_plan_t so = sp, dO = dp;
-    so.dtype = NEREUS_FP32; dO.dtype = NEREUS_FP32;                 // omega: fp32 on both sides, same (tp, pp)
+    so.dtype = NEREUS_FP32; dO.dtype = NEREUS_FP32;      // omega: fp32 on both sides, same (tp, pp) and layout
     for (int k = 0; rc == NEREUS_OK && k < n_opt; ++k) rc = nereus_transition_compile(d, so, dO, &parts[1 + k]);
     if (rc == NEREUS_OK) rc = nereus_transition_fuse(parts, 1 + n_opt, 0, out);
     for (int k = 0; k < 9; ++k)

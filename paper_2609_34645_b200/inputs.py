@@ -29,9 +29,18 @@ LLAMA_8B = Shape(32, 4096, 32, 8, 14336, 128256)   # Llama-3-8B-shaped
 DENSE_32B = Shape(64, 5120, 40, 8, 27648, 152064)  # 32B-shaped decoder
 
 
+QKV_GROUPED = 1            # layout flags of a plan: order of the rows inside a rank's fused blocks
+GATE_UP_INTERLEAVED = 2
+
+
+def layout_of(plan: tuple) -> int:
+    return plan[3] if len(plan) > 3 else 0
+
+
 @dataclass(frozen=True)
 class Stage:
-    """One model-stage's transition: (tp, pp, dtype) -> (tp, pp, dtype); dtype is "bf16" or "fp32"."""
+    """One model-stage's transition: (tp, pp, dtype[, layout]) -> (tp, pp, dtype[, layout]); dtype is "bf16" or
+    "fp32", layout a mask of QKV_GROUPED | GATE_UP_INTERLEAVED (0 when absent)."""
     name: str
     shape: Shape
     seed: int
@@ -96,6 +105,11 @@ WORKLOADS["8b_fp32_tp2pp2_to_bf16_tp4pp1_x2"] = Workload("8b_fp32_tp2pp2_to_bf16
 WORKLOADS["8b_state_adam_tp2pp2_to_tp4pp1"] = Workload("8b_state_adam_tp2pp2_to_tp4pp1", (
     Stage("8b_train", LLAMA_8B, 13, (2, 2, "bf16"), (4, 1, "bf16"), n_opt=2),),
     note="parameters (bf16) plus Adam's two fp32 moments, same layout, one table")
+
+WORKLOADS["8b_grouped_fp32_tp2pp2_to_blocked_bf16_tp4pp1"] = Workload(
+    "8b_grouped_fp32_tp2pp2_to_blocked_bf16_tp4pp1", (
+        Stage("8b_master", LLAMA_8B, 14, (2, 2, "fp32", QKV_GROUPED | GATE_UP_INTERLEAVED), (4, 1, "bf16", 0)),),
+    note="weight sync from a trainer's layout (grouped QKV, interleaved gate/up, fp32) to a generation layout")
 
 # scaled-down stand-ins with the same structure, for parity tests the oracle finishes in seconds
 SMALL = Shape(4, 512, 8, 4, 1376, 2048)            # head_dim 64; several tiles and ragged tails

@@ -153,14 +153,14 @@ def test_layout_agrees_with_oracle(sh, vh):
 
 # ---------------------------------------------------------------- the compiler, executed on the host
 
-def check_transition(sh, a, b, sdt="bf16", ddt="bf16", vh=False, seed=0):
+def check_transition(sh, a, b, sdt="bf16", ddt="bf16", vh=False, seed=0, la=0, lb=0):
     odt = {"bf16": O.BF16, "fp32": O.FP32}
     d = desc_of(sh, B.DTYPES[sdt], vh)
     m = omodel_of(sh, odt[sdt], vh)
-    oa, ob = O.Plan(*a), O.Plan(b[0], b[1], odt[ddt])
+    oa, ob = O.Plan(a[0], a[1], 0, la), O.Plan(b[0], b[1], odt[ddt], lb)
     src = random_src(m, oa, seed, sdt)
     want = O.reshard(m, oa, ob, src, fill=0xA5)
-    t = d.compile(B.Plan(*a), B.Plan(b[0], b[1], B.DTYPES[ddt]))
+    t = d.compile(B.Plan(a[0], a[1], 0, la), B.Plan(b[0], b[1], B.DTYPES[ddt], lb))
     n_src, n_dst = t.num_buffers()
     assert (n_src, n_dst) == (len(src), len(want))
     for i, s in enumerate(src):
@@ -200,6 +200,25 @@ def test_micro_plan_pairs_including_paper_example():
 @pytest.mark.parametrize("a,b", [((2, 2), (4, 1)), ((1, 1), (2, 2)), ((4, 4), (1, 1)), ((2, 1), (2, 1))])
 def test_cast_transitions(a, b):
     check_transition(I.SMALL, a, b, "fp32", "bf16", seed=2)
+
+
+@pytest.mark.parametrize("la,lb", [(la, lb) for la in range(4) for lb in range(4) if la or lb])
+def test_layout_variants(la, lb):
+    """Grouped QKV and row-interleaved gate/up on either side, with TP and PP changing at the same time."""
+    check_transition(I.SMALL, (2, 2), (4, 1), seed=la * 4 + lb, la=la, lb=lb)
+    check_transition(I.MICRO, (8, 1), (2, 4), seed=5, la=la, lb=lb)
+    check_transition(I.TINY, (1, 1), (2, 1), "fp32", "bf16", seed=6, la=la, lb=lb)
+
+
+def test_layout_variant_task_shapes():
+    d = desc_of(I.LLAMA_8B, B.FP32)
+    t = d.compile(B.Plan(2, 2, 0, 3), B.Plan(4, 1, B.BF16, 0))
+    rects = t.rects()
+    pitched = {(r.rows, r.width_bytes_dst, r.src_pitch) for r in rects if r.rows > 1 and r.width_bytes_dst == 8192}
+    assert pitched == {(14336 // 4, 8192, 32768)}             # gate / up rows picked out of the interleaved source
+    assert d.plan_check(B.Plan(2, 2, 0, 4)) == B.ERR_ARG       # unknown layout flag
+    same = d.compile(B.Plan(2, 2, 0, 3), B.Plan(2, 2, 0, 3))
+    assert all(r.rows == 1 for r in same.rects())              # same layout on both sides: runs only
 
 
 def test_value_head_and_fp32():

@@ -155,3 +155,63 @@ def test_transition_estimate_predicts_the_measured_time():
     t2, s2 = timed("8b4l_tp4pp2_to_tp1pp1")
     assert t2.estimate(gbps, 0.0) == pytest.approx(s2, rel=0.10)
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("variant", [1, 2])
+@pytest.mark.parametrize("la,lb", [(3, 0), (0, 3), (1, 2), (3, 3)])
+def test_layout_variants_on_the_gpu(la, lb, variant):
+    """Grouped QKV / row-interleaved gate-up on either side, with and without the cast, both kernels."""
+    sh = I.SMALL
+    for sdt, ddt, a, b in [("bf16", "bf16", (2, 2), (4, 1)), ("fp32", "bf16", (4, 1), (2, 2))]:
+        desc = G.desc_of(sh, sdt)
+        pa, pb = B.Plan(a[0], a[1], 0, la), B.Plan(b[0], b[1], B.DTYPES[ddt], lb)
+        t = desc.compile(pa, pb)
+        t.tune(variant=variant, tile_bytes=4096)
+        src = G.device_sources(desc, pa, sdt, 23)
+        dst = G.Guarded([t.buffer_bytes(True, j) for j in range(t.num_buffers()[1])])
+        G.run_transition(t, src, dst.bufs)
+        want = O.reshard(G.omodel_of(sh, sdt), O.Plan(a[0], a[1], 0, la), O.Plan(b[0], b[1], G.ODT[ddt], lb),
+                         [s.cpu().numpy() for s in src], fill=G.SENTINEL)
+        for g, w in zip(dst.bufs, want):
+            assert np.array_equal(g.cpu().numpy(), w)
+        assert dst.guards_intact()
+
+
+def test_8b_trainer_layout_to_generation_layout_full_size():
+    """fp32 weights in a trainer's layout (grouped QKV, interleaved gate/up, TP2PP2) to blocked bf16 TP4PP1:
+    every fused block of the first and last layer and the sums of all tensors against the oracle."""
+    name = "8b_grouped_fp32_tp2pp2_to_blocked_bf16_tp4pp1"
+    wl, t, srcs, dsts, descs = _run(name)
+    st = wl.stages[0]
+    desc, pa, pb = descs[0]
+    F._check_stage_sums(st, desc, srcs, dsts, pa, pb, "fp32", "bf16")
+    # oracle on whole fused blocks (qkv = stored id 1+6l+1, gate_up = 1+6l+4) of two layers, plus wo / wdown
+    sh = st.shape
+    m = O.Model(sh.layers, sh.hidden, sh.heads, sh.kv_heads, sh.ffn, sh.vocab, O.FP32, False)
+    opa, opb = O.Plan(2, 2, 0, 3), O.Plan(4, 1, O.BF16, 0)
+    for l in (0, 31):
+        for tids, sid in (((1 + 9 * l + 1, 1 + 9 * l + 2, 1 + 9 * l + 3), 1 + 6 * l + 1),
+                          ((1 + 9 * l + 6, 1 + 9 * l + 7), 1 + 6 * l + 4)):
+            # host copies of the fused block of every shard that holds it
+            sblk, dblk, dwant = {}, {}, {}
+            for s in range(4):
+                off, rows, cols, _ = desc.tensor_slice(pa, s, sid)
+                if rows:
+                    sblk[s] = (off, srcs[s][off:off + rows * cols * 4].cpu().numpy())
+            for d in range(4):
+                off, rows, cols, _ = desc.tensor_slice(pb, d, sid)
+                dblk[d] = (off, dsts[d][off:off + rows * cols * 2].cpu().numpy())
+                dwant[d] = np.zeros(rows * cols * 2, np.uint8)
+            for tid in tids:
+                sparts, dparts = [], []
+                for s in range(4):
+                    p = O.locate(m, opa, s, tid)
+                    sparts.append(sblk[s][1][p.offset - sblk[s][0]:] if p.held else None)
+                for d in range(4):
+                    p = O.locate(m, opb, d, tid)
+                    dparts.append(dwant[d][p.offset - dblk[d][0]:])
+                O.reshard_tensor_parts(m, opa, opb, tid, sparts, dparts)
+            for d in range(4):
+                assert np.array_equal(dblk[d][1], dwant[d]), (l, sid, d)
+    del srcs, dsts
+    torch.cuda.empty_cache()

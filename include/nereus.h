@@ -243,6 +243,61 @@ typedef struct { double h_steps; double weight; int observed; } nereus_horizon_t
 int nereus_horizon_init(nereus_horizon_t* h, double weight);
 int nereus_horizon_crossing(nereus_horizon_t* h, double interval_steps);
 
+/* ---- transition DAG over EMU primitives (Section 6.1) -------------------------------------------------- */
+
+/* Host-side planner.  Each model-stage M brings its current collection E_M and its target collection E*_M
+ * (units = (tp, pp, GPU list in shard order p*tp + r)); nereus_dag_plan turns every change Delta_M into a
+ * local DAG in the paper's default order Split -> Destroy -> Extend -> Merge and combines the local DAGs
+ * into one global DAG:
+ *   - T_sub = (gcd(tp, tp*), gcd(pp, pp*)), the largest layout both sides split into; Split(EMU, T_sub) makes
+ *     k = tp*pp / |T_sub| replica units on the unit's own GPUs, sub-unit j on GPUs [j*|T_sub|, (j+1)*|T_sub|);
+ *   - the target units' GPUs are cut into slots the same way; a slot that already holds a sub-unit (same
+ *     GPUs, same order) keeps it; every other sub-unit is redundant and gets a Destroy; every other slot is
+ *     filled by an Extend from the lowest-numbered kept sub-unit (else the lowest-numbered one), and a unit
+ *     that an Extend still reads is destroyed only after it; Merge fuses a target unit's slots;
+ *   - resources are bytes of GPU memory: a unit keeps state_bytes / (tp*pp) on each of its GPUs, every GPU
+ *     has gpu_capacity bytes; Split / Extend / Merge need room for what they create, Split / Destroy / Merge
+ *     free what they consume when they complete;
+ *   - the schedule takes ready primitives releasing-before-acquiring, then in stage order generation ->
+ *     inference -> training, then by model-stage and primitive index; because ready primitives run
+ *     concurrently, a primitive that only fits thanks to memory another primitive freed gets a
+ *     resource-dependency edge to it (newest release first); a blocked acquisition selects an executable
+ *     Destroy that frees one of its GPUs and does not depend on it; if there is none the plan is infeasible.
+ * Everything above the first item of each bullet is this build's reading of Section 6.1. */
+typedef struct nereus_dag_s* nereus_dag_t;
+#define NEREUS_GENERATION 0
+#define NEREUS_INFERENCE  1
+#define NEREUS_TRAINING   2
+#define NEREUS_OP_SPLIT   0
+#define NEREUS_OP_DESTROY 1
+#define NEREUS_OP_EXTEND  2
+#define NEREUS_OP_MERGE   3
+#define NEREUS_ERR_INFEASIBLE   -10   /* an acquisition stays blocked: the target plan fails the feasibility check */
+
+typedef struct {
+    int32_t op, stage;                 /* NEREUS_OP_*, model-stage index */
+    int32_t n_src, n_dst;              /* units read / created */
+    int32_t n_deps, n_resource_deps;   /* state edges / resource-dependency edges (primitive indices) */
+    int32_t order;                     /* position in the serial schedule */
+    int32_t level;                     /* longest path from a root: primitives of one level may run together */
+} nereus_prim_t;
+
+int nereus_dag_create(nereus_dag_t* out);
+int nereus_dag_destroy(nereus_dag_t dag);
+/* Adds a model-stage; kind = NEREUS_GENERATION / INFERENCE / TRAINING, state_bytes = one replica's state. */
+int nereus_dag_add_stage(nereus_dag_t dag, int kind, uint64_t state_bytes, int* stage);
+/* Adds a unit to a stage's current (is_target = 0) or target collection; gpus (host) has tp*pp entries. */
+int nereus_dag_add_unit(nereus_dag_t dag, int stage, int is_target, int tp, int pp, const int* gpus);
+/* Plans.  gpu_capacity 0 = unlimited.  Errors: ARG (a stage without units, mixed layouts inside a collection,
+ * a layout T_sub does not divide), NEREUS_ERR_INFEASIBLE. */
+int nereus_dag_plan(nereus_dag_t dag, uint64_t gpu_capacity);
+int nereus_dag_num_units(nereus_dag_t dag, int* n);          /* current units first, then created ones */
+int nereus_dag_unit(nereus_dag_t dag, int unit, int* stage, int* tp, int* pp, int* gpus, int gpus_cap);
+int nereus_dag_num_prims(nereus_dag_t dag, int* n);
+int nereus_dag_prim(nereus_dag_t dag, int prim, nereus_prim_t* out);
+/* Copies the primitive's lists; each pointer may be NULL, else it must hold the matching count. */
+int nereus_dag_prim_lists(nereus_dag_t dag, int prim, int* src, int* dst, int* deps, int* resource_deps);
+
 /* ---- execution without allocation --------------------------------------------------------------------- */
 
 /* The paper has no counterpart of this entry point; it exists for callers that cannot allocate device

@@ -22,6 +22,9 @@ OK = 0
 ERR_ARG, ERR_INDIVISIBLE, ERR_UNSUPPORTED, ERR_ALIAS = -1, -2, -3, -4
 ERR_CUDA, ERR_NOMEM, ERR_MISMATCH, ERR_ALIGN = -5, -6, -7, -8
 ERR_TOO_LARGE = -9
+ERR_INFEASIBLE = -10
+GENERATION, INFERENCE, TRAINING = 0, 1, 2
+OP_SPLIT, OP_DESTROY, OP_EXTEND, OP_MERGE = 0, 1, 2, 3
 STATIC_MAX_RECTS = 4096
 DEV_OK, DEV_BOUNDS, DEV_TIMEOUT = 0, 1, 2
 
@@ -74,6 +77,12 @@ class Horizon(ctypes.Structure):
         return self.h_steps
 
 
+class PrimInfo(ctypes.Structure):
+    """nereus_prim_t."""
+    _fields_ = [(n, ctypes.c_int32) for n in ("op", "stage", "n_src", "n_dst", "n_deps", "n_resource_deps",
+                                              "order", "level")]
+
+
 _vp, _i, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
 _P = ctypes.POINTER
 _SIGS = {
@@ -103,6 +112,16 @@ _SIGS = {
     "nereus_transition_status": [_vp, _P(_i)],
     "nereus_transition_launches": [_vp, _P(ctypes.c_uint64)],
     "nereus_last_cuda_error": [],
+    "nereus_dag_create": [_P(_vp)],
+    "nereus_dag_destroy": [_vp],
+    "nereus_dag_add_stage": [_vp, _i, ctypes.c_uint64, _P(_i)],
+    "nereus_dag_add_unit": [_vp, _i, _i, _i, _i, _P(_i)],
+    "nereus_dag_plan": [_vp, ctypes.c_uint64],
+    "nereus_dag_num_units": [_vp, _P(_i)],
+    "nereus_dag_unit": [_vp, _i, _P(_i), _P(_i), _P(_i), _P(_i), _i],
+    "nereus_dag_num_prims": [_vp, _P(_i)],
+    "nereus_dag_prim": [_vp, _i, _P(PrimInfo)],
+    "nereus_dag_prim_lists": [_vp, _i, _P(_i), _P(_i), _P(_i), _P(_i)],
     "nereus_transition_estimate": [_vp, ctypes.c_double, ctypes.c_double, _P(ctypes.c_double)],
     "nereus_admit": [ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_double, _i,
                      _P(_i), _P(ctypes.c_double)],
@@ -313,6 +332,69 @@ class Transition:
     def close(self):
         if self._h:
             _lib.nereus_transition_destroy(self._h)
+            self._h = _vp()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class Dag:
+    """Transition DAG over EMU primitives (nereus_dag_*)."""
+
+    def __init__(self):
+        self._h = _vp()
+        _ck(_lib.nereus_dag_create(ctypes.byref(self._h)), "nereus_dag_create")
+
+    def add_stage(self, kind: int, state_bytes: int) -> int:
+        s = _i()
+        _ck(_lib.nereus_dag_add_stage(self._h, kind, state_bytes, ctypes.byref(s)), "nereus_dag_add_stage")
+        return s.value
+
+    def add_unit(self, stage: int, is_target: bool, tp: int, pp: int, gpus) -> None:
+        arr = (_i * len(gpus))(*gpus)
+        if len(gpus) != tp * pp:
+            raise ValueError("a unit needs tp*pp GPUs")
+        _ck(_lib.nereus_dag_add_unit(self._h, stage, int(is_target), tp, pp, arr), "nereus_dag_add_unit")
+
+    def plan(self, gpu_capacity: int = 0) -> None:
+        _ck(_lib.nereus_dag_plan(self._h, gpu_capacity), "nereus_dag_plan")
+
+    def units(self) -> list:
+        n = _i()
+        _ck(_lib.nereus_dag_num_units(self._h, ctypes.byref(n)), "nereus_dag_num_units")
+        out = []
+        for u in range(n.value):
+            st, tp, pp = _i(), _i(), _i()
+            _ck(_lib.nereus_dag_unit(self._h, u, ctypes.byref(st), ctypes.byref(tp), ctypes.byref(pp), None, 0),
+                "nereus_dag_unit")
+            g = (_i * (tp.value * pp.value))()
+            _ck(_lib.nereus_dag_unit(self._h, u, ctypes.byref(st), ctypes.byref(tp), ctypes.byref(pp), g, len(g)),
+                "nereus_dag_unit")
+            out.append((st.value, tp.value, pp.value, tuple(g)))
+        return out
+
+    def prims(self) -> list:
+        """[{op, stage, src, dst, deps, resource_deps, order, level}] by primitive index."""
+        n = _i()
+        _ck(_lib.nereus_dag_num_prims(self._h, ctypes.byref(n)), "nereus_dag_num_prims")
+        out = []
+        for k in range(n.value):
+            info = PrimInfo()
+            _ck(_lib.nereus_dag_prim(self._h, k, ctypes.byref(info)), "nereus_dag_prim")
+            a = [(_i * max(1, c))() for c in (info.n_src, info.n_dst, info.n_deps, info.n_resource_deps)]
+            _ck(_lib.nereus_dag_prim_lists(self._h, k, *a), "nereus_dag_prim_lists")
+            out.append({"op": info.op, "stage": info.stage, "src": tuple(a[0][:info.n_src]),
+                        "dst": tuple(a[1][:info.n_dst]), "deps": set(a[2][:info.n_deps]),
+                        "resource_deps": set(a[3][:info.n_resource_deps]), "order": info.order,
+                        "level": info.level})
+        return out
+
+    def close(self):
+        if self._h:
+            _lib.nereus_dag_destroy(self._h)
             self._h = _vp()
 
     def __del__(self):

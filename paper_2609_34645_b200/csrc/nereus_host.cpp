@@ -592,6 +592,7 @@ const char* nereus_strerror(int code) {
     case NEREUS_ERR_NOMEM:       return "out of host memory";
     case NEREUS_ERR_MISMATCH:    return "chained parts do not connect";
     case NEREUS_ERR_ALIGN:       return "a shard pointer is not 16-byte aligned";
+    case NEREUS_ERR_INFEASIBLE:  return "the transition DAG cannot be scheduled: an acquisition stays blocked";
     case NEREUS_ERR_TOO_LARGE:   return "the transition has more tasks than the fixed scratch of run_static holds";
     default:                     return "unknown error";
     }

@@ -80,3 +80,88 @@ def test_infeasible_when_nothing_can_release():
     b = D.StageChange(D.TRAINING, [U(1, 1, 1)], [U(1, 1, 1)])                     # stays: GPU 1 is never freed
     with pytest.raises(D.Infeasible):
         D.plan([a, b], gpu_capacity=1 << 20)
+
+
+# ---------------------------------------------------------------- the library's planner against the oracle
+
+from paper_2609_34645_b200 import binding as B  # noqa: E402
+
+
+def lib_plan(changes, capacity=0):
+    dag = B.Dag()
+    for ch in changes:
+        s = dag.add_stage(ch.kind, ch.state_bytes)
+        for u in ch.current:
+            dag.add_unit(s, False, u.tp, u.pp, list(u.gpus))
+        for u in ch.target:
+            dag.add_unit(s, True, u.tp, u.pp, list(u.gpus))
+    dag.plan(capacity)
+    return dag.units(), dag.prims()
+
+
+def same_as_oracle(changes, capacity=0):
+    try:
+        units, prims, order = D.plan(changes, capacity or 1 << 62)
+    except D.Infeasible:
+        with pytest.raises(B.NereusError) as e:
+            lib_plan(changes, capacity)
+        assert e.value.code == B.ERR_INFEASIBLE
+        return None
+    lunits, lprims = lib_plan(changes, capacity)
+    assert lunits == units
+    assert len(lprims) == len(prims)
+    for i, (a, b) in enumerate(zip(lprims, prims)):
+        assert (a["op"], a["stage"], a["src"], a["dst"]) == (b.op, b.stage, b.src, b.dst), i
+        assert a["deps"] == b.deps and a["resource_deps"] == b.resource_deps, i
+    assert sorted(range(len(prims)), key=lambda i: lprims[i]["order"]) == order
+    for a in lprims:                                   # a level is above every predecessor's
+        for d in a["deps"] | a["resource_deps"]:
+            assert lprims[d]["level"] < a["level"]
+    return lprims
+
+
+def test_library_planner_on_the_paper_examples():
+    S = 32 << 20
+    reward = D.StageChange(D.INFERENCE, [U(4, 8, 33)], [U(8, 2, 33)], S)
+    actor = D.StageChange(D.TRAINING, [U(4, 2, 1)], [U(4, 2, 1), U(4, 2, 49)], S)
+    critic = D.StageChange(D.TRAINING, [U(4, 2, 9)], [U(4, 2, 9), U(4, 2, 57)], S)
+    prims = same_as_oracle([reward, actor, critic])
+    assert [p["op"] for p in prims] == [B.OP_SPLIT, B.OP_DESTROY, B.OP_DESTROY, B.OP_MERGE, B.OP_EXTEND, B.OP_EXTEND]
+    prims = same_as_oracle([reward, actor, critic], S // 8 + S // 16)
+    assert sum(len(p["resource_deps"]) for p in prims) == 2            # the two edges of the figure
+    actor2 = D.StageChange(D.GENERATION, [U(1, 4, 0), U(1, 4, 4)],
+                           [D.Unit(2, 4, tuple(range(0, 4)) + tuple(range(16, 20))),
+                            D.Unit(2, 4, tuple(range(4, 8)) + tuple(range(20, 24)))])
+    critic2 = D.StageChange(D.TRAINING, [U(1, 4, 8), U(1, 4, 12)], [U(1, 4, 8), U(1, 4, 12), U(1, 4, 24), U(1, 4, 28)])
+    same_as_oracle([actor2, critic2])
+    same_as_oracle([D.StageChange(D.INFERENCE, [U(2, 1, 0)], [U(2, 1, 8)])])
+    a = D.StageChange(D.GENERATION, [U(1, 1, 0)], [U(1, 1, 0), U(1, 1, 1)])
+    b = D.StageChange(D.TRAINING, [U(1, 1, 1)], [U(1, 1, 1)])
+    assert same_as_oracle([a, b], 1 << 20) is None                      # infeasible on both sides
+
+
+def test_library_planner_on_random_plan_changes():
+    """Random pools of 32-64 GPUs, 2-5 model-stages, power-of-two layouts, random placements and capacities:
+    the two planners agree on every unit, primitive, edge and on the schedule, or both say infeasible."""
+    rng = random.Random(7)
+    agree = infeasible = 0
+    for trial in range(300):
+        n_gpus = rng.choice([32, 48, 64])
+        changes = []
+        for m in range(rng.randint(2, 5)):
+            def collection():
+                tp, pp = rng.choice([1, 2, 4, 8]), rng.choice([1, 2, 4])
+                dp = rng.randint(1, 3)
+                units = []
+                for _ in range(dp):
+                    first = rng.randrange(0, n_gpus - tp * pp + 1, tp * pp)
+                    units.append(D.Unit(tp, pp, tuple(range(first, first + tp * pp))))
+                return units
+            changes.append(D.StageChange(rng.choice([0, 1, 2]), collection(), collection(),
+                                         rng.choice([8, 16, 70]) << 20))
+        cap = rng.choice([0, 64 << 20, 24 << 20, 12 << 20])
+        if same_as_oracle(changes, cap) is None:
+            infeasible += 1
+        else:
+            agree += 1
+    assert agree > 100 and infeasible > 10

@@ -298,6 +298,22 @@ int nereus_dag_prim(nereus_dag_t dag, int prim, nereus_prim_t* out);
 /* Copies the primitive's lists; each pointer may be NULL, else it must hold the matching count. */
 int nereus_dag_prim_lists(nereus_dag_t dag, int prim, int* src, int* dst, int* deps, int* resource_deps);
 
+/* Lowers a planned DAG to ONE task table that one launch executes (Section 6.2: a primitive is ready only
+ * after its predecessors complete; ready primitives run concurrently): every data-moving primitive becomes the
+ * tasks of a transition between its units' layouts and takes its DAG level as dependency level.
+ *   Split(u -> k units of T_sub)   u's layout -> T_sub, read once, written to the k sub-units
+ *   Extend(s -> n)                 T_sub -> T_sub copy of s into n
+ *   Merge(subs -> v)               T_sub -> v's layout; target shard i is cut from the sub-unit that sits on
+ *                                  the same GPU, i.e. subs[i / |T_sub|] (local slicing of replicated state)
+ *   Destroy                        no device work
+ * descs[m] describes model-stage m (its dtype is the state's dtype; plans use layout 0).  run() then takes as
+ * src_ptrs the shards of the current units, unit by unit in unit order, and as dst_ptrs the shards of every
+ * created unit (sub-units, extended units, target units) in unit order; a destroyed unit's memory may be
+ * reused for a unit created after the last primitive that reads it.
+ * Errors: ARG (not planned), UNSUPPORTED (more than 8 data-moving levels or too many buffers), and whatever
+ * nereus_transition_compile reports for a layout. */
+int nereus_dag_lower(nereus_dag_t dag, const nereus_model_desc_t* descs, int n_descs, nereus_transition_t* out);
+
 /* ---- execution without allocation --------------------------------------------------------------------- */
 
 /* The paper has no counterpart of this entry point; it exists for callers that cannot allocate device

@@ -122,6 +122,7 @@ _SIGS = {
     "nereus_dag_num_prims": [_vp, _P(_i)],
     "nereus_dag_prim": [_vp, _i, _P(PrimInfo)],
     "nereus_dag_prim_lists": [_vp, _i, _P(_i), _P(_i), _P(_i), _P(_i)],
+    "nereus_dag_lower": [_vp, _P(_vp), _i, _P(_vp)],
     "nereus_transition_estimate": [_vp, ctypes.c_double, ctypes.c_double, _P(ctypes.c_double)],
     "nereus_admit": [ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_double, _i,
                      _P(_i), _P(ctypes.c_double)],
@@ -391,6 +392,13 @@ class Dag:
                         "resource_deps": set(a[3][:info.n_resource_deps]), "order": info.order,
                         "level": info.level})
         return out
+
+    def lower(self, descs) -> "Transition":
+        """One task table for the whole DAG; descs[m] is the ModelDesc of model-stage m."""
+        arr = (_vp * len(descs))(*[d._h for d in descs])
+        h = _vp()
+        _ck(_lib.nereus_dag_lower(self._h, arr, len(descs), ctypes.byref(h)), "nereus_dag_lower")
+        return Transition(h)
 
     def close(self):
         if self._h:

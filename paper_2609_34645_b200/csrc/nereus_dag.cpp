@@ -8,36 +8,9 @@
 #include <set>
 #include <vector>
 
-#include "nereus.h"
+#include "nereus_internal.hpp"
 
-namespace {
-
-struct UnitRec {
-    int              stage, tp, pp;
-    std::vector<int> gpus;
-};
-
-struct PrimRec {
-    int              op, stage;
-    std::vector<int> src, dst;
-    std::set<int>    deps, rdeps;
-    int              order = -1, level = 0;
-};
-
-struct StageRec {
-    int                  kind;
-    uint64_t             state_bytes;
-    std::vector<UnitRec> current, target;
-};
-
-}  // namespace
-
-struct nereus_dag_s {
-    std::vector<StageRec> stages;
-    std::vector<UnitRec>  units;
-    std::vector<PrimRec>  prims;
-    bool                  planned = false;
-};
+using namespace nereus;
 
 namespace {
 

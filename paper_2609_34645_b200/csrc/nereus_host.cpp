@@ -545,6 +545,91 @@ int nereus_transition_get_rect(nereus_transition_t t, int index, nereus_rect_t* 
     return NEREUS_OK;
 }
 
+int nereus_dag_lower(nereus_dag_t dag, const nereus_model_desc_t* descs, int n_descs, nereus_transition_t* out) {
+    NEREUS_GUARD_BEGIN
+    if (!dag || !descs || !out || !dag->planned || n_descs != (int)dag->stages.size()) return NEREUS_ERR_ARG;
+    for (int m = 0; m < n_descs; ++m)
+        if (!descs[m]) return NEREUS_ERR_ARG;
+    const int n_units = (int)dag->units.size();
+    // which units are inputs (never created) and where each unit's shards start in the unified buffer list
+    std::vector<int> producer(n_units, -1);
+    for (size_t i = 0; i < dag->prims.size(); ++i)
+        for (int u : dag->prims[i].dst) producer[u] = (int)i;
+    std::vector<int> base(n_units, -1);
+    int n_src = 0, n_all = 0;
+    for (int u = 0; u < n_units; ++u)
+        if (producer[u] < 0) { base[u] = n_src; n_src += dag->units[u].tp * dag->units[u].pp; }
+    n_all = n_src;
+    for (int u = 0; u < n_units; ++u)
+        if (producer[u] >= 0) { base[u] = n_all; n_all += dag->units[u].tp * dag->units[u].pp; }
+    if (n_all > kMaxBuffers) return NEREUS_ERR_UNSUPPORTED;
+
+    // dependency levels of the data-moving primitives, renumbered densely
+    std::vector<int> used_levels;
+    for (const PrimRec& p : dag->prims)
+        if (p.op != NEREUS_OP_DESTROY) used_levels.push_back(p.level);
+    std::sort(used_levels.begin(), used_levels.end());
+    used_levels.erase(std::unique(used_levels.begin(), used_levels.end()), used_levels.end());
+    if ((int)used_levels.size() > kMaxLevels) return NEREUS_ERR_UNSUPPORTED;
+    auto level_of = [&](const PrimRec& p) {
+        return (int)(std::lower_bound(used_levels.begin(), used_levels.end(), p.level) - used_levels.begin());
+    };
+
+    auto* t = new nereus_transition_s();
+    t->src_bytes.assign(n_src, 0);
+    t->src_read_level.assign(n_src, 0);
+    t->dst_bytes.assign(n_all - n_src, 0);
+    t->dst_level.assign(n_all - n_src, 0);
+    t->dst_read_level.assign(n_all - n_src, -1);
+    auto plan_of = [](const UnitRec& u) { return nereus_plan_t{u.tp, u.pp, 0, 0}; };
+    int rc = NEREUS_OK;
+    for (const PrimRec& p : dag->prims) {
+        if (p.op == NEREUS_OP_DESTROY) continue;
+        const nereus_model_desc_s& d = *descs[p.stage];
+        const UnitRec& su = dag->units[p.src[0]];
+        const UnitRec& du = dag->units[p.dst[0]];
+        const int k = p.op == NEREUS_OP_SPLIT ? (int)p.dst.size() : 1;
+        nereus_transition_s part;
+        if ((rc = check_plan(d, plan_of(su))) || (rc = check_plan(d, plan_of(du)))) break;
+        if ((rc = compile_one(d, plan_of(su), plan_of(du), 1, part))) break;
+        const int ns = su.tp * su.pp, nd = du.tp * du.pp, lvl = level_of(p);
+        const int sub = su.tp * su.pp;                 // Merge: GPUs per sub-unit = shards per sub-unit
+        for (int i = 0; i < ns; ++i)
+            for (int u : p.src) {
+                if (producer[u] < 0) {
+                    t->src_bytes[base[u] + i] = part.src_bytes[i];
+                    t->src_read_level[base[u] + i] = std::max(t->src_read_level[base[u] + i], lvl);
+                }
+                else t->dst_read_level[base[u] - n_src + i] = std::max(t->dst_read_level[base[u] - n_src + i], lvl);
+            }
+        for (int u : p.dst)
+            for (int j = 0; j < nd; ++j) {
+                t->dst_bytes[base[u] - n_src + j] = part.dst_bytes[j];
+                t->dst_level[base[u] - n_src + j] = lvl;
+            }
+        for (Rect r : part.rects) {
+            const int shard_s = r.src_buf, shard_d = r.dst_buf - ns;
+            // Merge cuts target shard j from the sub-unit on the same GPU; Split and Extend read their one source
+            const int src_unit = p.op == NEREUS_OP_MERGE ? p.src[shard_d / sub] : p.src[0];
+            r.src_buf = base[src_unit] + shard_s;
+            r.dst_buf = base[p.dst[0]] + shard_d;
+            r.level = lvl;
+            if (k > 1) {
+                // the k sub-units are created one after another, so their buffers are nd apart
+                r.replicas = k;
+                r.replica_stride = nd;
+            }
+            t->rects.push_back(r);
+        }
+    }
+    if (rc) { delete t; return rc; }
+    t->n_levels = std::max<int>(1, (int)used_levels.size());
+    finish(*t);
+    *out = t;
+    return NEREUS_OK;
+    NEREUS_GUARD_END
+}
+
 int nereus_transition_estimate(nereus_transition_t t, double gbytes_per_s, double setup_seconds, double* seconds) {
     if (!t || !seconds || !(gbytes_per_s > 0.0) || !(setup_seconds >= 0.0)) return NEREUS_ERR_ARG;
     // levels are serial; within a level everything streams at the given bandwidth

@@ -129,6 +129,7 @@ struct nereus_transition_s {
     std::vector<nereus::Rect> rects;          // execution order
     std::vector<uint64_t>     src_bytes;      // required length of each source buffer
     std::vector<uint64_t>     dst_bytes;      // ... of each destination buffer
+    std::vector<int>          src_read_level; // last level that reads source buffer i (empty: level 0)
     std::vector<int>          dst_level;      // level that writes destination buffer j
     std::vector<int>          dst_read_level; // level that reads destination j (chained), -1 if none
     int                       n_levels = 1;
@@ -136,6 +137,41 @@ struct nereus_transition_s {
     nereus::Tuning            tuning;
     nereus::DeviceTable       dev;
     uint64_t                  launches = 0;
+};
+
+// ---------------------------------------------------------------------------------------------------
+// Transition DAG over EMU primitives
+// ---------------------------------------------------------------------------------------------------
+
+#include <set>
+
+namespace nereus {
+
+struct UnitRec {
+    int              stage, tp, pp;
+    std::vector<int> gpus;
+};
+
+struct PrimRec {
+    int              op, stage;
+    std::vector<int> src, dst;
+    std::set<int>    deps, rdeps;
+    int              order = -1, level = 0;
+};
+
+struct StageRec {
+    int                  kind;
+    uint64_t             state_bytes;
+    std::vector<UnitRec> current, target;
+};
+
+}  // namespace nereus
+
+struct nereus_dag_s {
+    std::vector<nereus::StageRec> stages;
+    std::vector<nereus::UnitRec>  units;
+    std::vector<nereus::PrimRec>  prims;
+    bool                          planned = false;
 };
 
 namespace nereus {

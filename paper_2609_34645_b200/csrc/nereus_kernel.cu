@@ -837,10 +837,12 @@ static int check_buffers(const nereus_transition_s& t, const void* const* src, v
     }
     for (size_t j = 0; j < nd; ++j) {
         const char* dj = (const char*)dst[j];
-        // a destination may overlap an original source only if it is written after level 0 has read it
-        for (size_t i = 0; i < ns; ++i)
-            if (t.dst_level[j] == 0 && overlap(dj, t.dst_bytes[j], (const char*)src[i], t.src_bytes[i]))
+        // a destination may overlap an original source only if it is written after the source's last reader
+        for (size_t i = 0; i < ns; ++i) {
+            const int last_read = t.src_read_level.empty() ? 0 : t.src_read_level[i];
+            if (t.dst_level[j] <= last_read && overlap(dj, t.dst_bytes[j], (const char*)src[i], t.src_bytes[i]))
                 return NEREUS_ERR_ALIAS;
+        }
         for (size_t k = j + 1; k < nd; ++k) {
             if (!overlap(dj, t.dst_bytes[j], (const char*)dst[k], t.dst_bytes[k])) continue;
             // two destinations may share memory only when the earlier one has been consumed before the

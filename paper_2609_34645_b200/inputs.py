@@ -57,6 +57,10 @@ class Workload:
     stages: tuple
     round_trip: bool = False   # run src->dst, then dst->src back, chained
     note: str = ""
+    # plan change executed through the primitive-level transition DAG instead of one direct transition: per
+    # stage (kind, [(tp, pp, first GPU), ...] current units, [...] target units); kind 0/1/2 = generation /
+    # inference / training
+    dag: tuple = ()
 
 
 WORKLOADS = {
@@ -110,6 +114,12 @@ WORKLOADS["8b_grouped_fp32_tp2pp2_to_blocked_bf16_tp4pp1"] = Workload(
     "8b_grouped_fp32_tp2pp2_to_blocked_bf16_tp4pp1", (
         Stage("8b_master", LLAMA_8B, 14, (2, 2, "fp32", QKV_GROUPED | GATE_UP_INTERLEAVED), (4, 1, "bf16", 0)),),
     note="weight sync from a trainer's layout (grouped QKV, interleaved gate/up, fp32) to a generation layout")
+
+WORKLOADS["8b_dag_tp4pp8_to_tp8pp2"] = Workload("8b_dag_tp4pp8_to_tp8pp2", (
+    Stage("8b_reward", LLAMA_8B, 15, (4, 8, "bf16"), (8, 2, "bf16")),),
+    dag=((1, ((4, 8, 0),), ((8, 2, 0),)),),
+    note="the paper's layout example through its primitives: Split into four (TP4,PP2) replicas, two Destroys, "
+         "Merge of the other two into (TP8,PP2); one launch, two dependency levels")
 
 # scaled-down stand-ins with the same structure, for parity tests the oracle finishes in seconds
 SMALL = Shape(4, 512, 8, 4, 1376, 2048)            # head_dim 64; several tiles and ragged tails

@@ -165,3 +165,76 @@ def test_library_planner_on_random_plan_changes():
         else:
             agree += 1
     assert agree > 100 and infeasible > 10
+
+
+# ---------------------------------------------------------------- lowering the DAG to one task table
+
+import numpy as np  # noqa: E402
+
+from oracle import oracle as O  # noqa: E402
+from paper_2609_34645_b200 import inputs as I  # noqa: E402
+from test_compiler_cpu import desc_of, interpret, omodel_of, payload_mask, random_src  # noqa: E402
+
+
+def lowered(changes, shapes, capacity=0):
+    dag = B.Dag()
+    for ch in changes:
+        s = dag.add_stage(ch.kind, ch.state_bytes)
+        for u in ch.current:
+            dag.add_unit(s, False, u.tp, u.pp, list(u.gpus))
+        for u in ch.target:
+            dag.add_unit(s, True, u.tp, u.pp, list(u.gpus))
+    dag.plan(capacity)
+    descs = [desc_of(sh) for sh in shapes]
+    return dag, dag.lower(descs), descs
+
+
+def test_lowered_paper_example_equals_the_direct_reshard():
+    """(TP4, PP8) -> four (TP4, PP2) replicas -> (TP8, PP2), executed from the lowered table level by level:
+    the replicas equal the oracle's (TP4,PP8)->(TP4,PP2), the target equals its direct (TP4,PP8)->(TP8,PP2)."""
+    sh = I.MICRO
+    ch = D.StageChange(D.INFERENCE, [U(4, 8, 0)], [U(8, 2, 0)])
+    dag, t, descs = lowered([ch], [sh])
+    units, prims = dag.units(), dag.prims()
+    assert [p["op"] for p in prims] == [B.OP_SPLIT, B.OP_DESTROY, B.OP_DESTROY, B.OP_MERGE]
+    n_src, n_dst = t.num_buffers()
+    assert n_src == 32 and n_dst == 4 * 8 + 16
+    assert t.num_tiles()[1] == 2                                  # Split, then Merge
+    m = omodel_of(sh)
+    src = random_src(m, O.Plan(4, 8), 3, "bf16")
+    got = [np.full(t.buffer_bytes(True, j), 0xA5, np.uint8) for j in range(n_dst)]
+    interpret(t.rects(), src, got)
+    sub_want = O.reshard(m, O.Plan(4, 8), O.Plan(4, 2), src, fill=0xA5)
+    for k in range(4):
+        for g, w in zip(got[8 * k:8 * k + 8], sub_want):
+            assert np.array_equal(g, w)
+    for g, w in zip(got[32:], O.reshard(m, O.Plan(4, 8), O.Plan(8, 2), src, fill=0xA5)):
+        assert np.array_equal(g, w)
+    # target shard i is cut from the sub-unit that sits on its GPU: shards 0..7 from replica 0, 8..15 from 1
+    merge = [r for r in t.rects() if r.level == 1]
+    assert {(r.dst_buf - n_src - 32) // 8 for r in merge} == {0, 1}
+    assert all((r.src_buf - n_src) // 8 == (r.dst_buf - n_src - 32) // 8 for r in merge)
+    rd, wr = t.bytes()
+    one = descs[0].compile(B.Plan(4, 8), B.Plan(4, 2)).bytes()
+    assert rd == one[0] + descs[0].compile(B.Plan(4, 2), B.Plan(8, 2)).bytes()[0] and wr > 4 * one[1]
+
+
+def test_lowered_extend_then_merge():
+    """Section 5.1's actor: (TP1, PP4) x2 -> (TP2, PP4) x2 = two Extends and two Merges; both target units hold
+    the same logical state as the two source replicas."""
+    sh = I.MICRO
+    actor = D.StageChange(D.GENERATION, [U(1, 4, 0), U(1, 4, 4)],
+                          [D.Unit(2, 4, tuple(range(0, 4)) + tuple(range(16, 20))),
+                           D.Unit(2, 4, tuple(range(4, 8)) + tuple(range(20, 24)))])
+    dag, t, descs = lowered([actor], [sh])
+    m = omodel_of(sh)
+    one = random_src(m, O.Plan(1, 4), 5, "bf16")
+    src = one + [x.copy() for x in one]                          # DP replicas hold the same logical state
+    n_src, n_dst = t.num_buffers()
+    assert (n_src, n_dst) == (8, 2 * 4 + 2 * 8)
+    got = [np.full(t.buffer_bytes(True, j), 0xA5, np.uint8) for j in range(n_dst)]
+    interpret(t.rects(), src, got)
+    want = O.reshard(m, O.Plan(1, 4), O.Plan(2, 4), one, fill=0xA5)
+    for k in range(2):
+        for g, w in zip(got[8 + 8 * k:16 + 8 * k], want):
+            assert np.array_equal(g, w)

@@ -215,3 +215,51 @@ def test_8b_trainer_layout_to_generation_layout_full_size():
                 assert np.array_equal(dblk[d][1], dwant[d]), (l, sid, d)
     del srcs, dsts
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("variant", [1, 2])
+def test_lowered_dag_runs_in_one_launch(variant):
+    """The paper's (TP4, PP8) -> (TP8, PP2) example planned as Split / Destroy / Merge, lowered to one table with
+    two dependency levels and run in one launch: replicas and target against the oracle."""
+    from oracle import dag as D
+    from test_dag_cpu import U, lowered
+    sh = I.MICRO
+    dag, t, descs = lowered([D.StageChange(D.INFERENCE, [U(4, 8, 0)], [U(8, 2, 0)])], [sh])
+    t.tune(variant=variant, tile_bytes=2048)
+    src = G.device_sources(descs[0], B.Plan(4, 8), "bf16", 3)
+    n_src, n_dst = t.num_buffers()
+    dst = G.Guarded([t.buffer_bytes(True, j) for j in range(n_dst)])
+    G.run_transition(t, src, dst.bufs)
+    assert t.launches() == 1 and t.num_tiles()[1] == 2
+    host = [s.cpu().numpy() for s in src]
+    m = G.omodel_of(sh)
+    sub = O.reshard(m, O.Plan(4, 8), O.Plan(4, 2), host, fill=G.SENTINEL)
+    for k in range(4):
+        for g, w in zip(dst.bufs[8 * k:8 * k + 8], sub):
+            assert np.array_equal(g.cpu().numpy(), w)
+    for g, w in zip(dst.bufs[32:], O.reshard(m, O.Plan(4, 8), O.Plan(8, 2), host, fill=G.SENTINEL)):
+        assert np.array_equal(g.cpu().numpy(), w)
+    assert dst.guards_intact()
+
+
+def test_8b_dag_full_size():
+    name = "8b_dag_tp4pp8_to_tp8pp2"
+    F._need(96 * (1 << 30))
+    wl, t, srcs, dsts, extra = bench.build_workload(name, torch.device("cuda"), dict(
+        tile_bytes=0, ctas_per_sm=0, threads=0, variant=0))
+    stream = torch.cuda.current_stream()
+    t.run([b.data_ptr() for b in srcs], [b.data_ptr() for b in dsts], stream.cuda_stream)
+    stream.synchronize()
+    assert t.status() == B.DEV_OK and t.num_tiles()[1] == 2
+    assert len(srcs) == 32 and len(dsts) == 4 * 8 + 16
+    for k in range(1, 4):                                     # the four replicas are identical
+        for a, b in zip(dsts[0:8], dsts[8 * k:8 * k + 8]):
+            assert torch.equal(a, b)
+    st = wl.stages[0]
+    desc = extra[1][0]
+    F._check_stage_sums(st, desc, srcs, dsts[32:], B.Plan(4, 8), B.Plan(8, 2), "bf16", "bf16")
+    F._check_stage_sums(st, desc, srcs, dsts[:8], B.Plan(4, 8), B.Plan(4, 2), "bf16", "bf16")
+    F._check_stage_sampled(st, srcs, dsts[32:], (4, 8, "bf16"), (8, 2, "bf16"),
+                           list(range(1, 10)) + [0, 9 * 32 + 1, 9 * 32 + 2, 9 * 31 + 5, 9 * 31 + 9])
+    del srcs, dsts
+    torch.cuda.empty_cache()

@@ -48,7 +48,7 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--e2e-steps", type=int, default=2)
-    ap.add_argument("--cpu-layers", type=int, default=6, help="layers in the CPU-oracle sample")
+    ap.add_argument("--cpu-layers", type=int, default=16, help="layers in the CPU-oracle sample (about 1 s each)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--tile-bytes", type=int, default=0)

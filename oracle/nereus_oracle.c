@@ -38,7 +38,8 @@
  *   TP rank r of t holds
  *     embed, LM head [V, H]   rows    [r*V/t, (r+1)*V/t)
  *     wq [nq*hd, H]           rows of q heads  [r*nq/t, (r+1)*nq/t)
- *     wk, wv [nkv*hd, H]      rows of kv heads [r*nkv/t, (r+1)*nkv/t)
+ *     wk, wv [nkv*hd, H]      rows of kv heads [r*nkv/t, (r+1)*nkv/t); when t > nkv (nkv | t) every kv head is
+ *                             replicated on t/nkv ranks: rank r holds head r / (t/nkv), the head its q heads use
  *     wo [H, nq*hd]           columns [r*nq*hd/t, (r+1)*nq*hd/t)
  *     wgate, wup [F, H]       rows    [r*F/t, (r+1)*F/t)
  *     wdown [H, F]            columns [r*F/t, (r+1)*F/t)
@@ -128,9 +129,10 @@ int oracle_check_plan(const oracle_model* m, oracle_plan p) {
     if (!m || p.tp < 1 || p.pp < 1 || (p.layout & ~3)) return ORACLE_ERR_ARG;
     if (m->L < 1 || m->H < 1 || m->nq < 1 || m->nkv < 1 || m->F < 1 || m->V < 1) return ORACLE_ERR_ARG;
     if (m->H % m->nq || m->nq % m->nkv) return ORACLE_ERR_INDIVISIBLE;
-    if (p.tp > m->nkv) return ORACLE_ERR_UNSUPPORTED;      /* no KV-head replication */
-    if (m->nkv % p.tp || m->nq % p.tp || m->F % p.tp || m->V % p.tp || m->L % p.pp)
-        return ORACLE_ERR_INDIVISIBLE;
+    /* tp <= nkv: whole kv heads per rank.  tp > nkv: every kv head is replicated on tp/nkv ranks, which needs
+     * nkv | tp; a rank's q heads must then all belong to its one kv head, which tp | nq gives. */
+    if (p.tp <= m->nkv ? m->nkv % p.tp : p.tp % m->nkv) return ORACLE_ERR_INDIVISIBLE;
+    if (m->nq % p.tp || m->F % p.tp || m->V % p.tp || m->L % p.pp) return ORACLE_ERR_INDIVISIBLE;
     return ORACLE_OK;
 }
 
@@ -142,7 +144,14 @@ static void rank_part(const oracle_model* m, int kind, int64_t r, int64_t t,
     kind_shape(m, kind, &rows, &cols);
     *r0 = 0; *nr = rows; *c0 = 0; *nc = cols;
     switch (kind) {
-    case K_EMBED: case K_WQ: case K_WK: case K_WV: case K_WGATE: case K_WUP:
+    case K_WK: case K_WV:
+        if (t > m->nkv) {                                       /* replicated kv heads: rank r holds the one */
+            int64_t hd = m->H / m->nq;                          /* head its q heads attend to                */
+            *nr = hd; *r0 = (r / (t / m->nkv)) * hd;
+            break;
+        }
+        /* fall through */
+    case K_EMBED: case K_WQ: case K_WGATE: case K_WUP:
         *nr = rows / t; *r0 = r * (rows / t); break;            /* dim-0 (column-parallel) */
     case K_HEAD:
         if (!m->value_head) { *nr = rows / t; *r0 = r * (rows / t); }
@@ -151,10 +160,6 @@ static void rank_part(const oracle_model* m, int kind, int64_t r, int64_t t,
         *nc = cols / t; *c0 = r * (cols / t); break;            /* dim-1 (row-parallel) */
     default: break;                                             /* norms: replicated */
     }
-}
-
-static int kind_replicated(const oracle_model* m, int kind) {
-    return kind == K_LN1 || kind == K_LN2 || kind == K_LNF || (kind == K_HEAD && m->value_head);
 }
 
 /* Elements of `kind` stored by one TP rank of t. */
@@ -167,8 +172,10 @@ static int64_t rank_elems(const oracle_model* m, int kind, int64_t t) {
 /* Row of the fused stored block (counted from the block's first row) that holds local row i of the rank's
  * part of logical tensor `kind`.  Tensors that are stored alone have row i at row i. */
 static int64_t part_rowpos(const oracle_model* m, oracle_plan pl, int kind, int64_t i) {
-    int64_t hd = m->H / m->nq, G = m->nq / m->nkv, t = pl.tp;
-    int64_t qr = m->nq * hd / t, kr = m->nkv * hd / t, fr = m->F / t;
+    int64_t hd = m->H / m->nq, t = pl.tp;
+    int64_t kv_heads = t > m->nkv ? 1 : m->nkv / t;            /* kv heads a rank holds */
+    int64_t G = (m->nq / t) / kv_heads;                        /* q heads per kv head inside a rank */
+    int64_t qr = m->nq * hd / t, kr = kv_heads * hd, fr = m->F / t;
     if (kind == K_WQ || kind == K_WK || kind == K_WV) {
         if (pl.layout & ORACLE_QKV_GROUPED) {
             int64_t head = i / hd, within = i % hd, group_rows = (G + 2) * hd;
@@ -311,26 +318,27 @@ int oracle_reshard_tensor_parts(const oracle_model* m, oracle_plan sp, oracle_pl
     unsigned char* full = (unsigned char*)malloc((size_t)(rows * cols * ses));
     if (!full) return ORACLE_ERR_NOMEM;
 
-    /* 1. GATHER */
-    int first_replica = 1;
+    /* 1. GATHER.  Parts never overlap partly: a part either covers new ground or repeats, exactly, a region an
+     * earlier rank brought (replicated norms and value head; kv heads when tp > kv_heads).  The first copy is
+     * taken, every later copy must be identical: all ranks hold the same logical state. */
+    int64_t seen_r0[64], seen_c0[64]; int n_seen = 0;
     for (int64_t s = 0; s < (int64_t)sp.tp * sp.pp; ++s) {
         oracle_locate(m, sp, s, id, &held, &off, &r0, &nr, &c0, &nc);
         if (!held) continue;
         const unsigned char* part = (const unsigned char*)src_parts[s];
         if (!part) { free(full); return ORACLE_ERR_ARG; }
-        if (kind_replicated(m, kind) && !first_replica) {
-            /* every TP rank of the owning stage holds the same logical state */
-            if (memcmp(full, part, (size_t)(rows * cols * ses)) != 0) {
-                free(full); return ORACLE_ERR_REPLICA_MISMATCH;
-            }
-            continue;
-        }
+        int repeat = 0;
+        for (int q = 0; q < n_seen; ++q) repeat |= (seen_r0[q] == r0 && seen_c0[q] == c0);
         for (int64_t i = 0; i < nr; ++i) {
             int64_t at = oracle_part_row(m, sp, id, i);                 /* where the plan's layout keeps row i */
-            for (int64_t j = 0; j < nc; ++j)
-                memcpy(full + ((r0 + i) * cols + (c0 + j)) * ses, part + (at * nc + j) * ses, (size_t)ses);
+            for (int64_t j = 0; j < nc; ++j) {
+                unsigned char* to = full + ((r0 + i) * cols + (c0 + j)) * ses;
+                const unsigned char* from = part + (at * nc + j) * ses;
+                if (!repeat) memcpy(to, from, (size_t)ses);
+                else if (memcmp(to, from, (size_t)ses) != 0) { free(full); return ORACLE_ERR_REPLICA_MISMATCH; }
+            }
         }
-        first_replica = 0;
+        if (!repeat && n_seen < 64) { seen_r0[n_seen] = r0; seen_c0[n_seen] = c0; ++n_seen; }
     }
 
     /* 2. CAST */

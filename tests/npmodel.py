@@ -69,12 +69,18 @@ def _stored_blocks(sh, tp, pp, p, r, logical, value_head, layout=0):
     variants reorder rows inside a rank's fused block: grouped QKV = per kv head [its q heads; k; v] (a reshape
     to [kv_heads, rows per head group, H]); interleaved gate/up = np.stack of the two row sets."""
     hd = sh.hidden // sh.heads
-    G = sh.heads // sh.kv_heads
+    local_kv = max(1, sh.kv_heads // tp)                  # kv heads a rank holds
+    G = (sh.heads // tp) // local_kv                      # q heads per kv head inside a rank
     def d0(x):
         return np.split(x, tp, axis=0)[r]
 
     def d1(x):
         return np.split(x, tp, axis=1)[r]
+
+    def dkv(x):              # kv heads: cut like any row block, or, past one head per rank, replicated
+        if tp <= sh.kv_heads:
+            return d0(x)
+        return np.split(x, sh.kv_heads, axis=0)[r // (tp // sh.kv_heads)]
 
     lps = sh.layers // pp
     blocks = []
@@ -84,13 +90,13 @@ def _stored_blocks(sh, tp, pp, p, r, logical, value_head, layout=0):
         g = lambda k: logical[f"{k}.{l}"]
         blocks.append(g("ln1"))
         if layout & QKV_GROUPED:
-            q = g("wq").reshape(sh.kv_heads, G * hd, sh.hidden)
-            k = g("wk").reshape(sh.kv_heads, hd, sh.hidden)
-            v = g("wv").reshape(sh.kv_heads, hd, sh.hidden)
-            mine = range(r * sh.kv_heads // tp, (r + 1) * sh.kv_heads // tp)
-            blocks.append(np.concatenate([np.concatenate([q[h], k[h], v[h]], axis=0) for h in mine], axis=0))
+            q = d0(g("wq")).reshape(local_kv, G * hd, sh.hidden)
+            k = dkv(g("wk")).reshape(local_kv, hd, sh.hidden)
+            v = dkv(g("wv")).reshape(local_kv, hd, sh.hidden)
+            blocks.append(np.concatenate([np.concatenate([q[h], k[h], v[h]], axis=0) for h in range(local_kv)],
+                                         axis=0))
         else:
-            blocks.append(np.concatenate([d0(g("wq")), d0(g("wk")), d0(g("wv"))], axis=0))
+            blocks.append(np.concatenate([d0(g("wq")), dkv(g("wk")), dkv(g("wv"))], axis=0))
         blocks.append(d1(g("wo")))
         blocks.append(g("ln2"))
         if layout & GATE_UP_INTERLEAVED:

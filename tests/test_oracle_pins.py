@@ -168,6 +168,30 @@ def test_layout_variant_sizes_and_cast():
         assert np.array_equal(g, w)
 
 
+def test_kv_head_replication_against_np():
+    """tp > kv_heads: every kv head lives on tp/kv_heads ranks (np.split into heads, rank r takes head
+    r // (tp/kv_heads)); q heads, FFN and vocabulary are cut as always.  Both directions and both QKV layouts."""
+    sh = I.Shape(2, 128, 16, 2, 256, 256)                        # 16 q heads, 2 kv heads, head_dim 8
+    m = model_of(sh)
+    logical = npmodel.random_logical(sh, 2, seed=13)
+    pls = [(1, 1), (2, 1), (4, 1), (8, 2), (16, 1)]
+    for la, lb in [(0, 0), (1, 0), (0, 1), (3, 3)]:
+        for a, b in itertools.product(pls, repeat=2):
+            src = npmodel.build_shards(sh, a[0], a[1], logical, layout=la)
+            want = npmodel.build_shards(sh, b[0], b[1], logical, layout=lb)
+            got = O.reshard(m, O.Plan(a[0], a[1], 0, la), O.Plan(b[0], b[1], 0, lb), src, fill=0xA5)
+            for g, w in zip(got, want):
+                assert g.size == w.size and np.array_equal(g, w), (la, lb, a, b)
+    assert O.check_plan(m, O.Plan(3, 1)) == O.ERR_INDIVISIBLE     # neither divides the other
+    assert O.check_plan(m, O.Plan(32, 1)) == O.ERR_INDIVISIBLE    # more ranks than q heads
+    src = npmodel.build_shards(sh, 8, 1, logical)
+    p = O.locate(m, O.Plan(8, 1), 1, 3)                           # wk of layer 0 on rank 1: a copy of rank 0's head
+    src[1][p.offset] ^= 1
+    with pytest.raises(O.OracleError) as e:
+        O.reshard(m, O.Plan(8, 1), O.Plan(1, 1), src)
+    assert e.value.code == O.ERR_REPLICA_MISMATCH
+
+
 # ---------------------------------------------------------------- brute-force owner function
 
 @pytest.mark.parametrize("es", [2, 4])
@@ -388,7 +412,8 @@ def test_cast_commutes_with_reshard():
 
 def test_refusals():
     m = model_of(I.TINY)
-    assert O.check_plan(m, O.Plan(4, 1)) == O.ERR_UNSUPPORTED       # tp > kv_heads
+    assert O.check_plan(m, O.Plan(4, 1)) == O.OK                    # tp > kv_heads: kv heads replicated
+    assert O.check_plan(m, O.Plan(8, 1)) == O.ERR_INDIVISIBLE       # more ranks than q heads
     assert O.check_plan(m, O.Plan(1, 4)) == O.ERR_INDIVISIBLE       # 2 layers over 4 stages
     assert O.check_plan(model_of(I.Shape(2, 256, 4, 2, 689, 1024)), O.Plan(2, 1)) == O.ERR_INDIVISIBLE
     assert O.check_plan(m, O.Plan(0, 1)) == O.ERR_ARG

@@ -43,7 +43,9 @@
  *   stored tensor ids (argument tensor_id below): 0 = embed; 1 + 6*l + k for layer l and
  *            k = 0 ln1, 1 qkv, 2 wo, 3 ln2, 4 gate_up, 5 wdown; 1 + 6*L = ln_f; 2 + 6*L = head.
  *   layout variants (nereus_plan_t.layout) reorder the rows inside qkv and gate_up, see the flags below.
- *   required: tp | nkv, tp | F, tp | V, pp | L, tp <= nkv (no KV-head replication), and every contiguous piece
+ *   tp > nkv (nkv | tp): every kv head is replicated on tp/nkv consecutive ranks; rank r stores head
+ *            r / (tp/nkv), the one its q heads attend to; as a source only the first copy of a head is read.
+ *   required: tp | nkv or nkv | tp, tp | nq, tp | F, tp | V, pp | L, and every contiguous piece
  *            a transition moves must start on and span a multiple of 16 bytes on both sides (for the cast: 8
  *            elements).
  */
@@ -60,7 +62,7 @@ extern "C" {
 #define NEREUS_OK                 0
 #define NEREUS_ERR_ARG           -1   /* null pointer, negative or zero size, index out of range          */
 #define NEREUS_ERR_INDIVISIBLE   -2   /* a divisibility or 16-byte rule of the layout contract fails       */
-#define NEREUS_ERR_UNSUPPORTED   -3   /* dtype pair other than same->same or fp32->bf16; tp > kv_heads;    */
+#define NEREUS_ERR_UNSUPPORTED   -3   /* dtype pair other than same->same or fp32->bf16;                   */
                                       /* more buffers than one launch can address                          */
 #define NEREUS_ERR_ALIAS         -4   /* a destination buffer overlaps a source or another destination     */
 #define NEREUS_ERR_CUDA          -5   /* a CUDA call failed; see nereus_last_cuda_error                    */

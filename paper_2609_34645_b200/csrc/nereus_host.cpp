@@ -17,13 +17,13 @@ namespace nereus {
 // ---------------------------------------------------------------------------------------------------
 
 static StoredTensor whole(int64_t rows, int64_t cols, int layer) {
-    return StoredTensor{Cut::Whole, 1, {rows, 0, 0}, cols, layer};
+    return StoredTensor{Cut::Whole, 1, {rows, 0, 0}, {0, 0, 0}, cols, layer};
 }
 static StoredTensor by_rows(int nseg, int64_t r0, int64_t r1, int64_t r2, int64_t cols, int layer) {
-    return StoredTensor{Cut::Rows, nseg, {r0, r1, r2}, cols, layer};
+    return StoredTensor{Cut::Rows, nseg, {r0, r1, r2}, {0, 0, 0}, cols, layer};
 }
 static StoredTensor by_cols(int64_t rows, int64_t cols, int layer) {
-    return StoredTensor{Cut::Cols, 1, {rows, 0, 0}, cols, layer};
+    return StoredTensor{Cut::Cols, 1, {rows, 0, 0}, {0, 0, 0}, cols, layer};
 }
 
 void build_catalogue(nereus_model_desc_s& d) {
@@ -34,6 +34,7 @@ void build_catalogue(nereus_model_desc_s& d) {
     for (int l = 0; l < d.L; ++l) {
         d.catalogue.push_back(whole(1, d.H, l));                                             // ln1
         d.catalogue.push_back(by_rows(3, d.nq * hd, d.nkv * hd, d.nkv * hd, d.H, l));        // q;k;v
+        d.catalogue.back().seg_unit[1] = d.catalogue.back().seg_unit[2] = hd;                // kv heads stay whole
         d.catalogue.push_back(by_cols(d.H, d.nq * hd, l));                                   // wo
         d.catalogue.push_back(whole(1, d.H, l));                                             // ln2
         d.catalogue.push_back(by_rows(2, d.F, d.F, 0, d.H, l));                              // gate;up
@@ -47,8 +48,9 @@ int check_plan(const nereus_model_desc_s& d, nereus_plan_t p) {
     if (p.tp < 1 || p.pp < 1) return NEREUS_ERR_ARG;
     if (p.dtype != 0 && p.dtype != NEREUS_BF16 && p.dtype != NEREUS_FP32) return NEREUS_ERR_ARG;
     if (p.layout & ~(NEREUS_QKV_GROUPED | NEREUS_GATE_UP_INTERLEAVED)) return NEREUS_ERR_ARG;
-    if (p.tp > d.nkv) return NEREUS_ERR_UNSUPPORTED;
-    if (d.nkv % p.tp || d.nq % p.tp || d.F % p.tp || d.V % p.tp || d.L % p.pp) return NEREUS_ERR_INDIVISIBLE;
+    // tp <= nkv: whole kv heads per rank; tp > nkv: each kv head replicated on tp/nkv ranks (needs nkv | tp)
+    if (p.tp <= d.nkv ? d.nkv % p.tp : p.tp % d.nkv) return NEREUS_ERR_INDIVISIBLE;
+    if (d.nq % p.tp || d.F % p.tp || d.V % p.tp || d.L % p.pp) return NEREUS_ERR_INDIVISIBLE;
     return NEREUS_OK;
 }
 
@@ -65,10 +67,20 @@ void stored_block(const StoredTensor& t, int tp, int64_t& rows, int64_t& cols) {
     case Cut::Cols:  rows = t.seg_rows[0]; cols = t.cols / tp; break;
     case Cut::Rows:
         rows = 0;
-        for (int s = 0; s < t.nseg; ++s) rows += t.seg_rows[s] / tp;
+        for (int s = 0; s < t.nseg; ++s) rows += std::max(t.seg_rows[s] / tp, t.seg_unit[s]);
         cols = t.cols;
         break;
     }
+}
+
+void segment_share(const StoredTensor& t, int s, int r, int tp, int64_t& lo, int64_t& n, bool& primary) {
+    const int64_t even = t.seg_rows[s] / tp;
+    if (even >= t.seg_unit[s]) { lo = r * even; n = even; primary = true; return; }
+    // fewer rows than one unit per rank: units are replicated, `copies` consecutive ranks hold the same unit
+    const int64_t copies = (int64_t)tp * t.seg_unit[s] / t.seg_rows[s];
+    lo = (r / copies) * t.seg_unit[s];
+    n = t.seg_unit[s];
+    primary = r % copies == 0;
 }
 
 void stage_layout(const nereus_model_desc_s& d, nereus_plan_t p, int stage, StageLayout& out) {
@@ -95,39 +107,42 @@ namespace {
 
 // One run of consecutive logical rows of one segment of a Rows-cut tensor as a TP rank stores it:
 // logical rows [lo, lo + n) of segment `seg` sit at stored rows at, at + step, at + 2*step, ...
+// primary = false on the later copies of rows that several ranks hold (replicated kv heads): as a source
+// only the first copy is read.
 struct RowPiece {
     int     seg;
     int64_t lo, n;
     int64_t at, step;
+    bool    primary;
 };
 
 // How rank r of t keeps a Rows-cut tensor under a layout.  Blocked: one piece per segment, stacked.
-// Grouped QKV (3 segments, q heads = G per kv head): per kv head of the rank, G*hd rows of Q, hd of K, hd of V.
+// Grouped QKV (3 segments): per kv head of the rank, its q heads, then its K rows, then its V rows.
 // Interleaved gate/up (2 segments): rows alternate, step 2.
 void row_pieces(const nereus_model_desc_s& d, const StoredTensor& x, int layout, int r, int t,
                 std::vector<RowPiece>& out) {
     out.clear();
+    int64_t lo[3], n[3]; bool primary[3];
+    for (int s = 0; s < x.nseg; ++s) segment_share(x, s, r, t, lo[s], n[s], primary[s]);
     if (x.nseg == 3 && (layout & NEREUS_QKV_GROUPED)) {
-        const int64_t hd = d.H / d.nq, G = d.nq / d.nkv, per = d.nkv / t, group_rows = (G + 2) * hd;
-        for (int64_t j = 0; j < per; ++j) {
-            const int64_t g = (int64_t)r * per + j;                 // global kv head
-            out.push_back({0, g * G * hd, G * hd, j * group_rows, 1});
-            out.push_back({1, g * hd, hd, j * group_rows + G * hd, 1});
-            out.push_back({2, g * hd, hd, j * group_rows + (G + 1) * hd, 1});
+        const int64_t hd = d.H / d.nq, heads = n[1] / hd;          // kv heads this rank holds
+        const int64_t q_rows = n[0] / heads, group_rows = q_rows + 2 * hd;
+        for (int64_t j = 0; j < heads; ++j) {
+            out.push_back({0, lo[0] + j * q_rows, q_rows, j * group_rows, 1, primary[0]});
+            out.push_back({1, lo[1] + j * hd, hd, j * group_rows + q_rows, 1, primary[1]});
+            out.push_back({2, lo[2] + j * hd, hd, j * group_rows + q_rows + hd, 1, primary[2]});
         }
         return;
     }
     if (x.nseg == 2 && (layout & NEREUS_GATE_UP_INTERLEAVED)) {
-        const int64_t n = x.seg_rows[0] / t;
-        out.push_back({0, (int64_t)r * n, n, 0, 2});
-        out.push_back({1, (int64_t)r * n, n, 1, 2});
+        out.push_back({0, lo[0], n[0], 0, 2, primary[0]});
+        out.push_back({1, lo[1], n[1], 1, 2, primary[1]});
         return;
     }
     int64_t base = 0;
     for (int s = 0; s < x.nseg; ++s) {
-        const int64_t n = x.seg_rows[s] / t;
-        out.push_back({s, (int64_t)r * n, n, base, 1});
-        base += n;
+        out.push_back({s, lo[s], n[s], base, 1, primary[s]});
+        base += n[s];
     }
 }
 
@@ -221,7 +236,7 @@ static int compile_one(const nereus_model_desc_s& d, nereus_plan_t sp, nereus_pl
                         row_pieces(d, x, sp.layout, rs, ts, spieces);
                         for (const RowPiece& q : dpieces) {
                             for (const RowPiece& s : spieces) {
-                                if (s.seg != q.seg) continue;
+                                if (s.seg != q.seg || !s.primary) continue;
                                 const int64_t lo = std::max(q.lo, s.lo), hi = std::min(q.lo + q.n, s.lo + s.n);
                                 if (lo >= hi) continue;
                                 r.src_buf = ps * ts + rs;

@@ -25,6 +25,8 @@ struct StoredTensor {
     Cut     cut;
     int     nseg;        // Rows: number of stacked segments (1, 2 or 3); otherwise 1
     int64_t seg_rows[3]; // Rows: logical rows of each segment; Whole/Cols: seg_rows[0] = rows
+    int64_t seg_unit[3]; // Rows: smallest block of rows a rank may hold (head_dim for K and V, else 0): when a
+                         //       rank's share would be smaller, the block is replicated over ranks instead
     int64_t cols;        // logical columns (the contiguous dimension)
     int     layer;       // owning layer, -1 embed (first stage), -2 final norm / head (last stage)
 };
@@ -59,6 +61,9 @@ int  owning_stage(const nereus_model_desc_s& d, int id, int pp);
 void stage_layout(const nereus_model_desc_s& d, nereus_plan_t p, int stage, StageLayout& out);
 // Rows x cols (elements) of the block one TP rank of `tp` stores for tensor `t`.
 void stored_block(const StoredTensor& t, int tp, int64_t& rows, int64_t& cols);
+// Segment s of a Rows-cut tensor on rank r of t: first logical row, row count, and whether r is the first
+// rank holding these rows (false on the later copies of a replicated block).
+void segment_share(const StoredTensor& t, int s, int r, int tp, int64_t& lo, int64_t& n, bool& primary);
 
 // ---------------------------------------------------------------------------------------------------
 // Task table

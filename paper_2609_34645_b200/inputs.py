@@ -121,6 +121,10 @@ WORKLOADS["8b_dag_tp4pp8_to_tp8pp2"] = Workload("8b_dag_tp4pp8_to_tp8pp2", (
     note="the paper's layout example through its primitives: Split into four (TP4,PP2) replicas, two Destroys, "
          "Merge of the other two into (TP8,PP2); one launch, two dependency levels")
 
+WORKLOADS["8b_tp4pp1_to_tp16pp1"] = Workload("8b_tp4pp1_to_tp16pp1", (
+    Stage("8b_generation", LLAMA_8B, 16, (4, 1, "bf16"), (16, 1, "bf16")),),
+    note="TP beyond the 8 kv heads: every kv head replicated on two ranks")
+
 # scaled-down stand-ins with the same structure, for parity tests the oracle finishes in seconds
 SMALL = Shape(4, 512, 8, 4, 1376, 2048)            # head_dim 64; several tiles and ragged tails
 MICRO = Shape(8, 64, 8, 8, 128, 128)               # head_dim 8; brute-force sized, TP up to 8, PP up to 8

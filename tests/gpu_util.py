@@ -47,6 +47,24 @@ def device_sources(desc, plan, dtype, seed, device="cuda"):
     return bufs
 
 
+def device_sources_by_oracle(sh, plan, dtype, seed, value_head=False, device="cuda"):
+    """Same, with the copies found through the oracle's layout: every region that several shards hold (norms,
+    value head, kv heads when tp > kv_heads) is tied.  plan = oracle Plan."""
+    m = omodel_of(sh, dtype, value_head)
+    n = O.num_shards(m, plan)
+    bufs = I.make_shards([O.shard_bytes(m, plan, s) for s in range(n)], dtype, seed, device)
+    groups = []
+    for t in range(O.num_logical(m)):
+        same = {}
+        for s in range(n):
+            p = O.locate(m, plan, s, t)
+            if p.held:
+                same.setdefault((p.r0, p.c0, p.nr, p.nc), []).append((s, p.offset, p.nr * p.nc * O.es(m, plan)))
+        groups += [g for g in same.values() if len(g) > 1]
+    I.tie_replicas(bufs, groups)
+    return bufs
+
+
 class Guarded:
     """Destination buffers with a guard zone on both sides, all pre-filled with a sentinel byte."""
 

@@ -29,11 +29,12 @@ def random_src(m, plan, seed, dtype):
     bufs = I.make_shards(sizes, dtype, seed)
     groups = []
     for t in range(O.num_logical(m)):
-        rows, cols = O.logical_shape(m, t)
-        held = [(s, O.locate(m, plan, s, t)) for s in range(len(sizes))]
-        held = [(s, p) for s, p in held if p.held]
-        if len(held) > 1 and all(p.nr * p.nc == rows * cols for _, p in held):
-            groups.append([(s, p.offset, p.nr * p.nc * O.es(m, plan)) for s, p in held])
+        same = {}                                    # parts that cover the same region are copies of each other
+        for s in range(len(sizes)):
+            p = O.locate(m, plan, s, t)
+            if p.held:
+                same.setdefault((p.r0, p.c0, p.nr, p.nc), []).append((s, p.offset, p.nr * p.nc * O.es(m, plan)))
+        groups += [g for g in same.values() if len(g) > 1]
     I.tie_replicas(bufs, groups)
     return [b.numpy() for b in bufs]
 
@@ -89,7 +90,8 @@ def test_library_exports_every_declared_symbol():
 
 def test_argument_errors():
     d = desc_of(I.TINY)
-    assert d.plan_check(B.Plan(4, 1)) == B.ERR_UNSUPPORTED
+    assert d.plan_check(B.Plan(4, 1)) == B.OK                      # tp > kv_heads: kv heads are replicated
+    assert d.plan_check(B.Plan(8, 1)) == B.ERR_INDIVISIBLE         # more ranks than q heads
     assert d.plan_check(B.Plan(1, 4)) == B.ERR_INDIVISIBLE
     assert d.plan_check(B.Plan(0, 1)) == B.ERR_ARG
     assert d.plan_check(B.Plan(1, 1, 7)) == B.ERR_ARG
@@ -219,6 +221,19 @@ def test_layout_variant_task_shapes():
     assert d.plan_check(B.Plan(2, 2, 0, 4)) == B.ERR_ARG       # unknown layout flag
     same = d.compile(B.Plan(2, 2, 0, 3), B.Plan(2, 2, 0, 3))
     assert all(r.rows == 1 for r in same.rects())              # same layout on both sides: runs only
+
+
+GQA16 = I.Shape(2, 128, 16, 2, 256, 256)          # 16 q heads, 2 kv heads, head_dim 8: room for tp up to 16
+
+
+@pytest.mark.parametrize("a,b", [((1, 1), (8, 1)), ((8, 2), (2, 1)), ((16, 1), (4, 2)), ((4, 1), (16, 1)),
+                                 ((8, 1), (8, 2)), ((2, 2), (16, 1))])
+def test_kv_head_replication(a, b):
+    """tp > kv_heads on either side: replicated kv heads are written to every rank that needs them and read
+    from the first rank that has them; with the cast and with grouped QKV as well."""
+    check_transition(GQA16, a, b, seed=1)
+    check_transition(GQA16, a, b, "fp32", "bf16", seed=2, la=1, lb=0)
+    check_transition(GQA16, a, b, seed=3, la=3, lb=3)
 
 
 def test_value_head_and_fp32():

@@ -263,3 +263,44 @@ def test_8b_dag_full_size():
                            list(range(1, 10)) + [0, 9 * 32 + 1, 9 * 32 + 2, 9 * 31 + 5, 9 * 31 + 9])
     del srcs, dsts
     torch.cuda.empty_cache()
+
+
+GQA16 = I.Shape(2, 128, 16, 2, 256, 256)          # 16 q heads, 2 kv heads, head_dim 8
+
+
+@pytest.mark.parametrize("variant", [1, 2])
+@pytest.mark.parametrize("a,b", [((1, 1), (8, 1)), ((8, 2), (2, 1)), ((16, 1), (4, 2)), ((4, 1), (16, 1))])
+def test_kv_head_replication_on_the_gpu(a, b, variant):
+    """tp > kv_heads on either side, bit copy and cast, both kernels."""
+    for sdt, ddt, la, lb in [("bf16", "bf16", 0, 0), ("fp32", "bf16", 1, 0)]:
+        desc = G.desc_of(GQA16, sdt)
+        pa, pb = B.Plan(a[0], a[1], 0, la), B.Plan(b[0], b[1], B.DTYPES[ddt], lb)
+        t = desc.compile(pa, pb)
+        t.tune(variant=variant, tile_bytes=1024)
+        src = G.device_sources_by_oracle(GQA16, O.Plan(a[0], a[1], 0, la), sdt, 29)
+        dst = G.Guarded([t.buffer_bytes(True, j) for j in range(t.num_buffers()[1])])
+        G.run_transition(t, src, dst.bufs)
+        want = O.reshard(G.omodel_of(GQA16, sdt), O.Plan(a[0], a[1], 0, la), O.Plan(b[0], b[1], G.ODT[ddt], lb),
+                         [s.cpu().numpy() for s in src], fill=G.SENTINEL)
+        for g, w in zip(dst.bufs, want):
+            assert np.array_equal(g.cpu().numpy(), w)
+        assert dst.guards_intact()
+
+
+def test_8b_tp16_beyond_the_kv_heads_full_size():
+    wl, t, srcs, dsts, descs = _run("8b_tp4pp1_to_tp16pp1")
+    st = wl.stages[0]
+    desc, pa, pb = descs[0]
+    F._check_stage_sampled(st, srcs, dsts, st.src, st.dst, list(range(1, 10)) + [0, 9 * 32 + 1, 9 * 32 + 2, 9 * 17 + 3])
+    # kv heads: ranks 2g and 2g+1 hold the same K and V rows of every layer
+    for tid in (1 + 6 * 0 + 1, 1 + 6 * 31 + 1):
+        off, rows, cols, _ = desc.tensor_slice(pb, 0, tid)
+        q_rows = 32 * 128 // 16
+        for r in range(0, 16, 2):
+            a = dsts[r][off + q_rows * cols * 2: off + rows * cols * 2]
+            b = dsts[r + 1][off + q_rows * cols * 2: off + rows * cols * 2]
+            assert torch.equal(a, b)
+    rd, wr = t.bytes()
+    assert rd == wr > 8_030_261_248 * 2 + 16 * 65 * 8192         # replicated kv heads move once per holder
+    del srcs, dsts
+    torch.cuda.empty_cache()

@@ -243,11 +243,12 @@ def _random_src(m, plan, seed, dtype):
     bufs = I.make_shards(sizes, dtype, seed)
     groups = []
     for t in range(O.num_logical(m)):
-        rows, cols = O.logical_shape(m, t)
-        held = [(s, O.locate(m, plan, s, t)) for s in range(len(sizes))]
-        held = [(s, p) for s, p in held if p.held]
-        if len(held) > 1 and all(p.nr * p.nc == rows * cols for _, p in held):
-            groups.append([(s, p.offset, p.nr * p.nc * O.es(m, plan)) for s, p in held])
+        same = {}                                    # parts that cover the same region are copies of each other
+        for s in range(len(sizes)):
+            p = O.locate(m, plan, s, t)
+            if p.held:
+                same.setdefault((p.r0, p.c0, p.nr, p.nc), []).append((s, p.offset, p.nr * p.nc * O.es(m, plan)))
+        groups += [g for g in same.values() if len(g) > 1]
     I.tie_replicas(bufs, groups)
     return [b.numpy() for b in bufs]
 

@@ -458,7 +458,7 @@ def run_e2e(args, t, srcs, dsts, sp, dp, stream, algo_bytes, world, device):
     import torch.distributed as dist
 
     need = sum(b.numel() for b in srcs) + sum(b.numel() for b in dsts)
-    budget = host_memory_budget()
+    budget = host_memory_budget() // max(1, world)      # every rank of the node pins its own copy
     if need > 0.5 * budget:
         return {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
                 "note": f"skipped: {need / 1e9:.1f} GB of pinned host memory needed, {budget / 1e9:.1f} GB available"}

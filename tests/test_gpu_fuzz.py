@@ -1,0 +1,68 @@
+"""Seeded random transitions on the GPU against the oracle: shapes, plans, layouts, dtypes, replica counts,
+kernels and tile sizes drawn together, so that combinations no hand-written case lists are exercised."""
+import random
+
+import numpy as np
+import pytest
+
+import gpu_util as G
+from oracle import oracle as O
+from paper_2609_34645_b200 import binding as B
+from paper_2609_34645_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+SHAPES = [I.SMALL, I.MICRO, I.TINY, I.Shape(2, 128, 16, 2, 256, 256), I.Shape(3, 192, 6, 3, 384, 768)]
+
+
+def valid_plans(sh):
+    out = []
+    for tp in (1, 2, 3, 4, 6, 8, 16):
+        for pp in (1, 2, 3, 4, 8):
+            kv_ok = sh.kv_heads % tp == 0 if tp <= sh.kv_heads else tp % sh.kv_heads == 0
+            if kv_ok and sh.heads % tp == 0 and sh.ffn % tp == 0 and sh.vocab % tp == 0 and sh.layers % pp == 0:
+                out.append((tp, pp))
+    return out
+
+
+def draw(rng):
+    sh = rng.choice(SHAPES)
+    a, b = rng.choice(valid_plans(sh)), rng.choice(valid_plans(sh))
+    sdt = rng.choice(["bf16", "bf16", "fp32"])
+    ddt = "bf16" if sdt == "bf16" else rng.choice(["fp32", "bf16"])
+    return dict(sh=sh, a=a, b=b, sdt=sdt, ddt=ddt, la=rng.randrange(4), lb=rng.randrange(4),
+                vh=rng.random() < 0.25, k=rng.choice([1, 1, 1, 2, 3]), variant=rng.choice([1, 2]),
+                tile=rng.choice([512, 1024, 4096, 16384]))
+
+
+@pytest.mark.parametrize("chunk", range(6))
+def test_random_transitions(chunk):
+    rng = random.Random(1000 + chunk)
+    ran = 0
+    for _ in range(14):
+        c = draw(rng)
+        sh = c["sh"]
+        desc = G.desc_of(sh, c["sdt"], c["vh"])
+        pa = B.Plan(c["a"][0], c["a"][1], 0, c["la"])
+        pb = B.Plan(c["b"][0], c["b"][1], B.DTYPES[c["ddt"]], c["lb"])
+        if c["variant"] == 2 and c["sdt"] != c["ddt"] and c["tile"] > 16384:
+            continue
+        try:
+            t = desc.compile_replicated(pa, pb, c["k"])
+        except B.NereusError as e:
+            # pieces that are not multiples of 16 bytes are refused at compile time, never mis-copied
+            assert e.code == B.ERR_INDIVISIBLE, c
+            continue
+        t.tune(tile_bytes=c["tile"], variant=c["variant"])
+        oa = O.Plan(c["a"][0], c["a"][1], 0, c["la"])
+        ob = O.Plan(c["b"][0], c["b"][1], G.ODT[c["ddt"]], c["lb"])
+        src = G.device_sources_by_oracle(sh, oa, c["sdt"], 77 + ran, c["vh"])
+        dst = G.Guarded([t.buffer_bytes(True, j) for j in range(t.num_buffers()[1])])
+        G.run_transition(t, src, dst.bufs)
+        want = O.reshard_replicated(G.omodel_of(sh, c["sdt"], c["vh"]), oa, ob, c["k"],
+                                    [s.cpu().numpy() for s in src], fill=G.SENTINEL)
+        for j, (g, w) in enumerate(zip(dst.bufs, want)):
+            assert np.array_equal(g.cpu().numpy(), w), (c, j)
+        assert dst.guards_intact(), c
+        ran += 1
+    assert ran >= 6

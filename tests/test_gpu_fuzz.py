@@ -12,7 +12,8 @@ from paper_2609_34645_b200 import inputs as I
 
 pytestmark = pytest.mark.gpu
 
-SHAPES = [I.SMALL, I.MICRO, I.TINY, I.Shape(2, 128, 16, 2, 256, 256), I.Shape(3, 192, 6, 3, 384, 768)]
+SHAPES = [I.SMALL, I.MICRO, I.TINY, I.Shape(2, 128, 16, 2, 256, 256), I.Shape(3, 192, 6, 3, 384, 768),
+          I.Shape(3, 192, 6, 6, 384, 768)]              # 6 kv heads: TP 2 and 3 do not nest
 
 
 def valid_plans(sh):

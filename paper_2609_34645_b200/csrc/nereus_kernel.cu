@@ -371,7 +371,7 @@ struct StageMeta {
     uint64_t d_off;
     uint32_t nr, w, dp;
     uint32_t kind;          // kStageData, kStageEnd or kStageFlush
-    uint16_t dst_buf, reps, rstride, pad_;
+    uint16_t dst_buf, reps, rstride, cast;
 };
 constexpr uint32_t kStageData = 0, kStageEnd = 1, kStageFlush = 2;
 
@@ -453,8 +453,9 @@ __device__ __forceinline__ void ring_producer(const WalkParams& p, const Ring& R
             Tile t;
             bool ok = true;
             if (!end) {
-                ok = resolve_tile<true>(p, g, rr, t) && t.cast == (kCast ? 1u : 0u) &&
-                     (((uint64_t)t.nr * t.w) << (kCast ? 1 : 0)) <= R.stage_bytes;
+                // the converting ring (kCast) takes both kinds of tile, the bit-copy ring only its own
+                ok = resolve_tile<true>(p, g, rr, t) && (kCast || t.cast == 0) &&
+                     (((uint64_t)t.nr * t.w) << t.cast) <= R.stage_bytes;
                 if (!ok && lane == 0) raise_status(ctrl, NEREUS_DEV_BOUNDS, g);
             }
             // a tile of a higher level: first have the consumer publish this CTA's finished tiles (a flush
@@ -505,11 +506,12 @@ __device__ __forceinline__ void ring_producer(const WalkParams& p, const Ring& R
                     running = false;
                     break;
                 }
-                const uint32_t ws = t.w << (kCast ? 1 : 0);                 // source bytes per row piece
+                const uint32_t ws = t.w << t.cast;                          // source bytes per row piece
                 if (lane == 0) {
                     StageMeta& m = R.meta[stage];
                     m.d_off = t.d_off; m.nr = t.nr; m.w = t.w; m.dp = t.dp;
                     m.dst_buf = (uint16_t)t.dst_buf; m.reps = (uint16_t)t.reps; m.rstride = (uint16_t)t.rstride;
+                    m.cast = (uint16_t)t.cast;
                     m.kind = kStageData;
                     mbar_arrive_expect_tx(bar, t.nr * ws);
                 }
@@ -588,7 +590,8 @@ __device__ __forceinline__ void ring_consumer_copy(const WalkParams& p, const Ri
 }
 
 
-// Consumer warps of the cast ring: read fp32 from the stage, convert, store bf16 with plain 16-byte stores.
+// Consumer warps of the converting ring: read fp32 from the stage, convert, store bf16 with plain 16-byte stores
+// (bit-copy tiles of a mixed table: 16 bytes in, 16 bytes out).
 // The unit is 8 elements: 32 bytes of shared memory in, 16 bytes out.  Each of the warps publishes its
 // own share of a tile, so the completion counter of a cast table counts warp-tiles (15 per tile) and no wait
 // between the warps (which could not be bounded) is needed.  Fifteen warps: a lone warp per scheduler would
@@ -612,6 +615,19 @@ __device__ __forceinline__ void ring_consumer_cast(const WalkParams& p, const Ri
             __syncwarp();
             if (lane == 0 && unpublished) atomicAdd(&ctrl->done, unpublished);
             unpublished = 0;
+        } else if (!m.cast) {
+            // a bit-copy tile of a mixed table: 16 bytes per lane straight from the stage
+            const unsigned char* src = R.data + (size_t)stage * R.stage_bytes;
+            const uint32_t vpr = m.w >> 4, nvec = m.nr * vpr;
+#pragma unroll 2
+            for (uint32_t idx = ct; idx < nvec; idx += kCastConsumers) {
+                const uint32_t r = idx / vpr, c = idx - r * vpr;
+                const uint4 v = *reinterpret_cast<const uint4*>(src + r * m.w + c * 16);
+                const uint32_t doff = r * m.dp + c * 16;
+                for (uint32_t j = 0; j < m.reps; ++j)
+                    st_stream(tile_dst(p, m.dst_buf, m.rstride, m.d_off, j) + doff, v);
+            }
+            ++unpublished;
         } else {
             const unsigned char* src = R.data + (size_t)stage * R.stage_bytes;
             const uint32_t upr = m.w >> 4, nunit = m.nr * upr, ws = m.w << 1;
@@ -704,12 +720,12 @@ struct Launch {
     size_t   smem = 0;
 };
 
-// The ring takes tables that are all bit copy or all cast; mixed tables run on the vector kernel.
+// The ring takes every table: all bit copy on the bulk-store consumer, anything with a cast in it on the
+// converting consumers (which copy the bit-copy tiles of a mixed table from shared memory as well).
 static bool ring_eligible(const nereus_transition_s& t, bool& cast) {
-    bool any_cast = false, any_copy = false;
-    for (const Rect& r : t.rects) (r.cast ? any_cast : any_copy) = true;
-    cast = any_cast;
-    return !(any_cast && any_copy);
+    cast = false;
+    for (const Rect& r : t.rects) cast = cast || r.cast;
+    return true;
 }
 
 static int resolve_launch(const nereus_transition_s& t, int sms, Launch& L) {

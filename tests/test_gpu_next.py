@@ -304,3 +304,26 @@ def test_8b_tp16_beyond_the_kv_heads_full_size():
     assert rd == wr > 8_030_261_248 * 2 + 16 * 65 * 8192         # replicated kv heads move once per holder
     del srcs, dsts
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("variant", [1, 2])
+def test_mixed_cast_and_copy_table(variant):
+    """One table with cast tiles (fp32 parameters -> bf16) and bit-copy tiles (fp32 optimizer moments): the
+    converting ring serves both kinds."""
+    sh = I.SMALL
+    desc = G.desc_of(sh, "fp32")
+    a, b = (2, 2), (4, 1)
+    pa, pb = B.Plan(a[0], a[1], B.FP32), B.Plan(b[0], b[1], B.BF16)
+    t = desc.compile_state(pa, pb, 2)
+    assert {r.cast for r in t.rects()} == {0, 1}
+    t.tune(variant=variant, tile_bytes=4096)
+    assert t.launch_info()["kernel"] == ("nereus_walk_ring" if variant == 2 else "nereus_walk_vec")
+    src = G.device_sources(desc, pa, "fp32", 1) + G.device_sources(desc, pa, "fp32", 2) + \
+        G.device_sources(desc, pa, "fp32", 3)
+    dst = G.Guarded([t.buffer_bytes(True, j) for j in range(t.num_buffers()[1])])
+    G.run_transition(t, src, dst.bufs)
+    want = O.reshard_state(G.omodel_of(sh, "fp32"), O.Plan(*a), O.Plan(b[0], b[1], O.BF16), 2,
+                           [s.cpu().numpy() for s in src], fill=G.SENTINEL)
+    for g, w in zip(dst.bufs, want):
+        assert np.array_equal(g.cpu().numpy(), w)
+    assert dst.guards_intact()

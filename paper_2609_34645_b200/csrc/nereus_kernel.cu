@@ -376,7 +376,6 @@ struct StageMeta {
 constexpr uint32_t kStageData = 0, kStageEnd = 1, kStageFlush = 2;
 
 constexpr uint32_t kBulkMaxStages = 28;
-constexpr uint32_t kClaimBatch    = 4;          // consecutive tiles per claim of the ring's producer
 constexpr uint32_t kCastConsumers = 480;        // cast ring: threads that convert a stage (15 warps)
 constexpr uint32_t kBarrierTries  = 1u << 22;   // try_wait attempts before a wait gives up
 
@@ -419,6 +418,7 @@ struct Ring {
     uint32_t       stage_bytes, n_stages;
     uint32_t       piece;          // contiguous tiles are issued as bulk copies of this many bytes
     uint32_t       lag;            // stages whose stores may still be reading shared memory
+    uint32_t       claim;          // consecutive tiles the producer takes per atomic
 };
 
 // cp.async.bulk.wait_group.read takes an immediate
@@ -436,19 +436,19 @@ __device__ __forceinline__ void wait_store_reads(uint32_t pending) {
     }
 }
 
-// Producer warp: claims kClaimBatch consecutive tiles at a time, resolves them and loads them into the ring.
+// Producer warp: claims R.claim consecutive tiles at a time, resolves them and loads them into the ring.
 // kCast: the stage receives the fp32 source bytes (twice the destination bytes).
 template <bool kCast>
 __device__ __forceinline__ void ring_producer(const WalkParams& p, const Ring& R, unsigned lane) {
     Ctrl* const ctrl = p.ctrl;
     uint32_t    stage = 0, phase = 0, level = 0;
     RectRange   rr;
-    uint32_t    g0 = claim_tiles(ctrl, lane, kClaimBatch);
+    uint32_t    g0 = claim_tiles(ctrl, lane, R.claim);
     bool        running = true;
     while (running) {
         const bool     last    = g0 >= p.n_tiles;
-        const uint32_t next_issued = last ? g0 : claim_issue(ctrl, lane, kClaimBatch);   // hidden behind this batch
-        for (uint32_t g = g0; running && g < g0 + kClaimBatch; ++g) {
+        const uint32_t next_issued = last ? g0 : claim_issue(ctrl, lane, R.claim);   // hidden behind this batch
+        for (uint32_t g = g0; running && g < g0 + R.claim; ++g) {
             const bool end = g >= p.n_tiles;
             Tile t;
             bool ok = true;
@@ -661,7 +661,7 @@ __device__ __forceinline__ void ring_consumer_cast(const WalkParams& p, const Ri
 template <bool kCast>
 __global__ void __launch_bounds__(kCast ? 32 + kCastConsumers : 64, kCast ? 1 : 2)
 nereus_walk_ring(const __grid_constant__ WalkParams p, const uint32_t stage_bytes, const uint32_t n_stages,
-                 const uint32_t piece, const uint32_t lag) {
+                 const uint32_t piece, const uint32_t lag, const uint32_t claim) {
     extern __shared__ __align__(128) unsigned char smem[];
     Ring R;
     R.data  = smem;
@@ -672,6 +672,7 @@ nereus_walk_ring(const __grid_constant__ WalkParams p, const uint32_t stage_byte
     R.n_stages = n_stages;
     R.piece = piece;
     R.lag = lag;
+    R.claim = claim;
     const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
     if (threadIdx.x == 0) {
@@ -716,7 +717,7 @@ struct Launch {
     bool     cast = false;          // ring only: the table is all cast
     int      tile_bytes = 0, ctas_per_sm = 0, threads = 0;
     uint32_t n_stages = 0;          // bulk ring
-    uint32_t piece = 16384, lag = 2;
+    uint32_t piece = 16384, lag = 2, claim = 4;
     size_t   smem = 0;
 };
 
@@ -762,6 +763,8 @@ static int resolve_launch(const nereus_transition_s& t, int sms, Launch& L) {
         L.smem = L.n_stages * per_stage;
         L.piece = (uint32_t)env_int("NEREUS_RING_PIECE", 16384);
         L.lag = (uint32_t)env_int("NEREUS_RING_LAG", std::min(3, (int)L.n_stages - 2));
+        L.claim = (uint32_t)env_int("NEREUS_RING_CLAIM", 4);
+        if (L.claim < 1 || L.claim > 64) return NEREUS_ERR_ARG;
         if (L.piece < 16 || L.piece % 16 || L.lag < 1 || L.lag > 8 || L.lag + 2 > L.n_stages) return NEREUS_ERR_ARG;
     }
     return NEREUS_OK;
@@ -774,10 +777,10 @@ static int launch_walk(const Launch& L, int sms, const WalkParams& p, cudaStream
         if (L.cast) {
             NEREUS_CUDA(cudaFuncSetAttribute(nereus_walk_ring<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.smem));
             nereus_walk_ring<true><<<grid, 32 + kCastConsumers, L.smem, stream>>>(p, (uint32_t)L.tile_bytes * 2, L.n_stages,
-                                                                                  L.piece, L.lag);
+                                                                                  L.piece, L.lag, L.claim);
         } else {
             NEREUS_CUDA(cudaFuncSetAttribute(nereus_walk_ring<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.smem));
-            nereus_walk_ring<false><<<grid, 64, L.smem, stream>>>(p, (uint32_t)L.tile_bytes, L.n_stages, L.piece, L.lag);
+            nereus_walk_ring<false><<<grid, 64, L.smem, stream>>>(p, (uint32_t)L.tile_bytes, L.n_stages, L.piece, L.lag, L.claim);
         }
     } else {
         const unsigned warps_per_cta = (unsigned)L.threads / 32;

@@ -108,6 +108,7 @@ struct Ctrl {
 
 constexpr int kMaxBuffers = 448;      // pointers carried in the kernel's parameter block
 constexpr int kMaxLevels  = 8;
+constexpr int kCtrlSlots  = 64;
 constexpr int kMaxReplicas = 16;
 
 struct Tuning {
@@ -121,7 +122,8 @@ struct DeviceTable {                  // one per prepare()
     int       device    = -1;
     RectDev*  rects     = nullptr;
     uint32_t* first     = nullptr;    // n_rects + 1 tile prefix
-    Ctrl*     ctrl      = nullptr;
+    Ctrl*     ctrl      = nullptr;    // kCtrlSlots control blocks, used round robin: one memset per cycle
+    uint32_t  runs      = 0;          // runs launched on this device copy
     uint32_t  n_tiles   = 0;
     uint32_t  level_end[kMaxLevels] = {0};   // tiles up to and including each level
     int       sm_count  = 0;

@@ -56,6 +56,7 @@ static_assert(sizeof(WalkParams) <= 4000, "kernel parameter block too large");
 constexpr int      kUnrollRun   = 8;            // 16-byte loads in flight per lane, contiguous runs
 constexpr int      kUnrollRect  = 6;            // ... pitched rects (their index math needs registers)
 constexpr int      kUnrollCast  = 8;            // ... the cast
+constexpr uint32_t kPrefixCache = 2047;         // rects whose tile prefix the vector kernel keeps in shared memory
 constexpr uint32_t kGatePolls   = 1u << 21;     // x ~200 ns sleep: gives up after roughly half a second
 
 // ---------------------------------------------------------------------------------------------------
@@ -241,14 +242,16 @@ struct RectRange {
 
 // Resolves tile g: binary search for the rect (largest i with first[i] <= g), then row block x column block.
 // Returns false when the table does not resolve (corrupted).
-template <bool kUseRange>
-__device__ __forceinline__ bool resolve_tile(const WalkParams& p, uint32_t g, RectRange& rr, Tile& t) {
+// `first_at(i)` reads entry i of the tile-prefix array (from global memory, or from a shared-memory copy).
+template <bool kUseRange, class FirstAt>
+__device__ __forceinline__ bool resolve_tile(const WalkParams& p, uint32_t g, RectRange& rr, Tile& t,
+                                             FirstAt first_at) {
     uint4 q0, q1, q2, q3;
     if (!kUseRange || g < rr.first || g >= rr.next_first) {
         uint32_t lo = 0, hi = p.n_rects;                       // invariant: first[lo] <= g < first[hi]
         while (hi - lo > 1) {
             const uint32_t mid = (lo + hi) >> 1;
-            if (__ldg(p.first + mid) <= g) lo = mid; else hi = mid;
+            if (first_at(mid) <= g) lo = mid; else hi = mid;
         }
         const RectDev* rp = p.rects + lo;
         q0 = __ldg(reinterpret_cast<const uint4*>(rp));        // src_off, dst_off
@@ -256,8 +259,8 @@ __device__ __forceinline__ bool resolve_tile(const WalkParams& p, uint32_t g, Re
         q2 = __ldg(reinterpret_cast<const uint4*>(rp) + 2);    // rows, rows_per_tile, tile_w, col_tiles
         q3 = __ldg(reinterpret_cast<const uint4*>(rp) + 3);    // first_tile, bufs, level|cast, replicas|stride
         if (kUseRange) {
-            rr.first = __ldg(p.first + lo);
-            rr.next_first = __ldg(p.first + lo + 1);
+            rr.first = first_at(lo);
+            rr.next_first = first_at(lo + 1);
             rr.q0 = q0; rr.q1 = q1; rr.q2 = q2; rr.q3 = q3;
         }
     } else {
@@ -302,11 +305,21 @@ __global__ void __launch_bounds__(512, 2) nereus_walk_vec(const __grid_constant_
     uint32_t       open_level = 0;                             // highest level whose gate this warp has passed
     RectRange      rr;
 
+    // small tables: the tile prefix is copied to shared memory once per CTA, so that resolving a tile costs
+    // one trip to memory (the rect record) instead of a chain of dependent ones
+    __shared__ uint32_t s_first[kPrefixCache + 1];
+    const bool cached = p.n_rects <= kPrefixCache;
+    if (cached)
+        for (uint32_t i = threadIdx.x; i <= p.n_rects; i += blockDim.x) s_first[i] = __ldg(p.first + i);
+    __syncthreads();
+    const uint32_t* const sf = s_first;
+    auto first_at = [&p, cached, sf](uint32_t i) { return cached ? sf[i] : __ldg(p.first + i); };
+
     uint32_t g = claim_tile(ctrl, lane);
     while (g < p.n_tiles) {
         const uint32_t next_issued = claim_issue(ctrl, lane, 1);   // in flight while this tile is copied
         Tile t;
-        if (!resolve_tile<false>(p, g, rr, t)) {
+        if (!resolve_tile<false>(p, g, rr, t, first_at)) {
             if (lane == 0) raise_status(ctrl, NEREUS_DEV_BOUNDS, g);
             return;
         }
@@ -454,7 +467,8 @@ __device__ __forceinline__ void ring_producer(const WalkParams& p, const Ring& R
             bool ok = true;
             if (!end) {
                 // the converting ring (kCast) takes both kinds of tile, the bit-copy ring only its own
-                ok = resolve_tile<true>(p, g, rr, t) && (kCast || t.cast == 0) &&
+                ok = resolve_tile<true>(p, g, rr, t, [&p](uint32_t i) { return __ldg(p.first + i); }) &&
+                     (kCast || t.cast == 0) &&
                      (((uint64_t)t.nr * t.w) << t.cast) <= R.stage_bytes;
                 if (!ok && lane == 0) raise_status(ctrl, NEREUS_DEV_BOUNDS, g);
             }
@@ -746,11 +760,11 @@ static int resolve_launch(const nereus_transition_s& t, int sms, Launch& L) {
     if (L.ctas_per_sm < 1 || L.ctas_per_sm > 2 || L.threads < 32 || L.threads > 512 || L.threads % 32)
         return NEREUS_ERR_ARG;
     if (L.tile_bytes == 0) {
-        // default: 16 KiB per warp tile (32 KiB per ring stage); smaller tiles for small tables, so that every
-        // claimer still gets a few tiles
+        // default: 16 KiB per warp tile (32 KiB per ring stage); smaller tiles for small tables, until at least
+        // every other claimer gets a tile
         L.tile_bytes = L.variant == 2 ? (L.cast ? 24576 : 32768) : 16384;
         const uint64_t claimers = (uint64_t)sms * L.ctas_per_sm * (L.variant == 2 ? 8 : L.threads / 32);
-        while (L.tile_bytes > 1024 && t.bytes_written / L.tile_bytes < 4 * claimers) L.tile_bytes /= 2;
+        while (L.tile_bytes > 1024 && t.bytes_written / L.tile_bytes < claimers / 2) L.tile_bytes /= 2;
     }
     if (L.tile_bytes < 512 || L.tile_bytes % 512) return NEREUS_ERR_ARG;
     if (L.variant == 2) {
@@ -818,13 +832,14 @@ static int prepare(nereus_transition_s& t) {
     const size_t rects_b = round_up(rects.size() * sizeof(RectDev), 256);
     const size_t first_b = round_up(first.size() * sizeof(uint32_t), 256);
     char* base = nullptr;
-    NEREUS_CUDA(cudaMalloc(&base, rects_b + first_b + 256));
+    const size_t ctrl_b = round_up(sizeof(Ctrl) * kCtrlSlots, 256);
+    NEREUS_CUDA(cudaMalloc(&base, rects_b + first_b + ctrl_b));
     dv.rects = reinterpret_cast<RectDev*>(base);
     dv.first = reinterpret_cast<uint32_t*>(base + rects_b);
     dv.ctrl  = reinterpret_cast<Ctrl*>(base + rects_b + first_b);
     cudaError_t e = cudaMemcpy(dv.rects, rects.data(), rects.size() * sizeof(RectDev), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(dv.first, first.data(), first.size() * sizeof(uint32_t), cudaMemcpyHostToDevice);
-    if (e == cudaSuccess) e = cudaMemset(dv.ctrl, 0, 256);
+    if (e == cudaSuccess) e = cudaMemset(dv.ctrl, 0, ctrl_b);
     if (e != cudaSuccess) { cudaFree(base); set_cuda_error((int)e); (void)cudaGetLastError(); return NEREUS_ERR_CUDA; }
     t.dev = dv;
     return NEREUS_OK;
@@ -935,7 +950,11 @@ int nereus_transition_run(nereus_transition_t t, const void* const* src_ptrs, vo
         if (int rc = resolve_launch(*t, dv.sm_count, L)) return rc;
         L.tile_bytes = dv.tile_bytes;
         WalkParams p;
-        p.rects = dv.rects; p.first = dv.first; p.ctrl = dv.ctrl;
+        // control words: a fresh (zeroed) block per run; the blocks are zeroed together once per cycle
+        const uint32_t slot = t->dev.runs % kCtrlSlots;
+        if (slot == 0 && t->dev.runs != 0)
+            NEREUS_CUDA(cudaMemsetAsync(dv.ctrl, 0, sizeof(Ctrl) * kCtrlSlots, stream));
+        p.rects = dv.rects; p.first = dv.first; p.ctrl = dv.ctrl + slot;
         p.n_tiles = dv.n_tiles;
         // NEREUS_DEBUG_GATE_BIAS (tests only): raises what a dependency gate waits for, so that it can never
         // open and the bounded wait must give up with NEREUS_DEV_TIMEOUT
@@ -943,8 +962,8 @@ int nereus_transition_run(nereus_transition_t t, const void* const* src_ptrs, vo
         for (int k = 0; k < kMaxLevels; ++k) p.level_end[k] = dv.level_end[k] + gate_bias;
         fill_params(*t, src_ptrs, dst_ptrs, p);
 
-        NEREUS_CUDA(cudaMemsetAsync(dv.ctrl, 0, sizeof(Ctrl), stream));
         if (int rc = launch_walk(L, dv.sm_count, p, stream)) return rc;
+        t->dev.runs += 1;
         if (dv.n_tiles > 0) t->launches += 1;
         return NEREUS_OK;
     } catch (const std::bad_alloc&) { return NEREUS_ERR_NOMEM; }
@@ -954,7 +973,8 @@ int nereus_transition_status(nereus_transition_t t, int* device_status) {
     if (!t || !device_status) return NEREUS_ERR_ARG;
     if (!t->dev.rects) { *device_status = NEREUS_DEV_OK; return NEREUS_OK; }
     Ctrl c;
-    NEREUS_CUDA(cudaMemcpy(&c, t->dev.ctrl, sizeof(Ctrl), cudaMemcpyDeviceToHost));
+    if (t->dev.runs == 0) { *device_status = NEREUS_DEV_OK; return NEREUS_OK; }
+    NEREUS_CUDA(cudaMemcpy(&c, t->dev.ctrl + (t->dev.runs - 1) % kCtrlSlots, sizeof(Ctrl), cudaMemcpyDeviceToHost));
     *device_status = (int)c.status;
     return NEREUS_OK;
 }

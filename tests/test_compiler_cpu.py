@@ -415,3 +415,30 @@ def test_buffer_limit_of_one_launch():
     with pytest.raises(B.NereusError) as e:
         d.compile_replicated(B.Plan(8, 8), B.Plan(8, 8), 7)      # 64 + 448
     assert e.value.code == B.ERR_UNSUPPORTED
+
+
+def test_header_is_plain_c_and_the_library_links_from_c(tmp_path):
+    """The boundary is a C ABI: nereus.h compiles as C99, and a C program that calls a few entry points links
+    against the library and runs (host-only calls, no GPU needed)."""
+    import subprocess
+    src = tmp_path / "use_nereus.c"
+    src.write_text(r'''
+#include <stdio.h>
+#include "nereus.h"
+int main(void) {
+    nereus_model_desc_t d; nereus_transition_t t; size_t rd, wr; int n;
+    nereus_plan_t a = {2, 1, 0, 0}, b = {1, 1, 0, 0};
+    if (nereus_model_desc(2, 256, 4, 2, 688, 1024, NEREUS_BF16, &d)) return 1;
+    if (nereus_transition_compile(d, a, b, &t)) return 2;
+    if (nereus_transition_bytes(t, &rd, &wr) || nereus_transition_num_rects(t, &n)) return 3;
+    printf("%zu %zu %d %s\n", rd, wr, n, nereus_strerror(NEREUS_ERR_ALIAS));
+    nereus_transition_destroy(t); nereus_model_desc_destroy(d);
+    return 0;
+}
+''')
+    exe = tmp_path / "use_nereus"
+    libdir = os.path.dirname(B.LIB_PATH)
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), str(src),
+                           "-o", str(exe), "-L", libdir, "-lnereus", f"-Wl,-rpath,{libdir}"])
+    out = subprocess.check_output([str(exe)], text=True).split()
+    assert out[0] == out[1] == str(1_975_552 * 2) and int(out[2]) > 0

@@ -5,7 +5,7 @@
  * paper) are carried from a source (TP, PP) layout to a target (TP, PP) layout on ONE GPU, every virtual
  * TP/PP rank's shard being a separate device buffer.  This is the local layout change that the paper's Split
  * and Merge primitives perform next to their collectives (Section 6.2, "DAG Execution and Safety" and
- * "Resharding--transport interplay"); it changes placement and sharding and never the logical state
+ * "Resharding--transport interplay"); it re-cuts and moves the state and leaves the logical state untouched
  * (Section 6.2, "Preserving training semantics").  An optional fp32 -> bf16 round-to-nearest-even cast is
  * fused into the move for the training -> generation weight sync between the actor's two model-stages
  * (Section 5, EMU definition).
@@ -139,7 +139,7 @@ int nereus_plan_tensor_slice(nereus_model_desc_t desc, nereus_plan_t plan, int s
 
 /* Compiles src -> dst for one model-stage into rect-copy tasks by intersecting every destination slice
  * with the source slices directly (no intermediate layout).  Host work only.
- * Errors: ARG, INDIVISIBLE, UNSUPPORTED (dtype pair; tp > kv_heads), NOMEM. */
+ * Errors: ARG, INDIVISIBLE, UNSUPPORTED (dtype pair, too many buffers), NOMEM. */
 int nereus_transition_compile(nereus_model_desc_t desc, nereus_plan_t src, nereus_plan_t dst,
                               nereus_transition_t* out);
 /* Same, with `replicas` identical destination units (1..16): every source byte is read once and written
@@ -150,14 +150,14 @@ int nereus_transition_compile(nereus_model_desc_t desc, nereus_plan_t src, nereu
 int nereus_transition_compile_replicated(nereus_model_desc_t desc, nereus_plan_t src, nereus_plan_t dst,
                                          int replicas, nereus_transition_t* out);
 /* The EMU's full state (theta, omega) in one table: the parameters src -> dst as above, plus `n_opt`
- * optimizer tensors per parameter (Adam: 2), held in fp32 and following the same layout (Section 5: "optimizer
- * shards omega follow the same layout").  run() takes, on either side, the parameter shards followed by the
+ * optimizer tensors per parameter (Adam: 2), held in fp32 and sharded exactly like the parameters (Section 5
+ * gives omega the layout of theta).  run() takes, on either side, the parameter shards followed by the
  * shards of optimizer tensor 0, then of tensor 1, ...; optimizer shards have the sizes of an fp32 plan with
  * the same tp and pp.  Optimizer state is never cast.  Errors: as nereus_transition_compile, ARG (n_opt < 0). */
 int nereus_transition_compile_state(nereus_model_desc_t desc, nereus_plan_t src, nereus_plan_t dst, int n_opt,
                                     nereus_transition_t* out);
-/* Fuses n compiled transitions into one task table that one launch executes (Section 6.2: ready primitives
- * run concurrently; a primitive is ready only after its predecessors complete).
+/* Fuses n compiled transitions into one task table that one launch executes (the readiness rule of Section
+ * 6.2: work whose predecessors are done may run side by side, nothing starts before its predecessors end).
  *   chained = 0: the parts are independent model-stages.  run() takes the concatenation of the parts'
  *                source arrays and the concatenation of their destination arrays.  One level.
  *   chained = 1: part k+1 reads what part k wrote: its source buffers ARE part k's destination buffers
@@ -180,9 +180,11 @@ int nereus_transition_num_tiles(nereus_transition_t t, uint64_t* tiles, int* lev
 
 /* Launch tuning; 0 keeps the default of a field.  tile_bytes: target bytes per claimed tile (multiple of
  * 512).  ctas_per_sm, threads: persistent grid = SMs * ctas_per_sm blocks of `threads` threads.
- * variant: 0 default (the ring where it applies), 1 register-staged vector copy, 2 bulk-copy shared-memory
- * ring (tables with a cast or with several levels always run on the vector kernel).  tile_bytes 0 = 16 KiB (32 KiB per ring stage),
- * halved for small tables until every claimer gets a few tiles.
+ * variant: 0 default (the ring for tables of 64 MiB and more, the vector kernel below), 1 register-staged
+ * vector copy, 2 bulk-copy shared-memory ring.  tile_bytes 0 = 16 KiB for the vector kernel, 32 KiB per
+ * ring stage (24 KiB when the table contains a cast: the stage then holds the fp32 source), halved for small
+ * tables until at least every other claimer gets a tile.  A ring stage must fit four times into the shared
+ * memory of an SM, else ARG at prepare.
  * Drops the device copy of the table (the next prepare/run uploads it again).  Errors: ARG. */
 int nereus_transition_tune(nereus_transition_t t, int tile_bytes, int ctas_per_sm, int threads, int variant);
 
@@ -220,8 +222,9 @@ int nereus_transition_launches(nereus_transition_t t, uint64_t* n);
 
 /* ---- cost side: the transition estimate and the admission gate (Sections 4.3 and 6) ------------------- */
 
-/* L_tran of a compiled transition: the paper estimates the critical-path cost "from bytes, link bandwidth,
- * and communicator setup" (Section 6); on one GPU the link is HBM and the set-up is the launch.  Levels run
+/* L_tran of a compiled transition: in the paper the critical-path cost is a function of the bytes moved, the
+ * bandwidth of the link and the time to set communicators up (Section 6); on one GPU the link is HBM and the
+ * set-up is the launch.  Levels run
  * one after another, so seconds = setup_seconds + sum over levels of (bytes read + written) / bandwidth.
  * gbytes_per_s: the sustained reshard bandwidth (e.g. a value bench.py measured); must be > 0.
  * Errors: ARG. */
@@ -300,8 +303,8 @@ int nereus_dag_prim(nereus_dag_t dag, int prim, nereus_prim_t* out);
 /* Copies the primitive's lists; each pointer may be NULL, else it must hold the matching count. */
 int nereus_dag_prim_lists(nereus_dag_t dag, int prim, int* src, int* dst, int* deps, int* resource_deps);
 
-/* Lowers a planned DAG to ONE task table that one launch executes (Section 6.2: a primitive is ready only
- * after its predecessors complete; ready primitives run concurrently): every data-moving primitive becomes the
+/* Lowers a planned DAG to ONE task table that one launch executes (the readiness rule of Section 6.2 becomes
+ * dependency levels): every data-moving primitive becomes the
  * tasks of a transition between its units' layouts and takes its DAG level as dependency level.
  *   Split(u -> k units of T_sub)   u's layout -> T_sub, read once, written to the k sub-units
  *   Extend(s -> n)                 T_sub -> T_sub copy of s into n

@@ -1,7 +1,7 @@
 """TEST INFRASTRUCTURE -- NOT PART OF THE PRODUCT.
 
 Plain restatement of the cost side of a transition, for the tests to hold the library against:
-the transition estimate (Section 6: "estimated from bytes, link bandwidth, and communicator setup"), the
+the transition estimate (Section 6: a function of bytes moved, link bandwidth and communicator set-up), the
 profitability gate (Eq. 2, Section 4.3) and the horizon H_x (an exponential moving average of the intervals
 between threshold crossings, one step before the first interval; Section 4.3).  The averaging weight is not
 in the paper; it is a parameter here too."""

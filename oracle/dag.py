@@ -24,7 +24,7 @@ What this build had to decide (readings, all repeated in the product's header):
   * a target unit's slots are its GPUs cut the same way; a slot already holding a sub-unit (same GPUs, same
     order) is kept in place, every other slot is filled by Extend from the lowest-numbered live sub-unit of
     the model-stage that is kept, else from the lowest-numbered one at all;
-  * resources are bytes of GPU memory ("near-capacity pool"): a unit of layout (tp, pp) keeps
+  * resources are bytes of GPU memory (the pool is assumed nearly full): a unit of layout (tp, pp) keeps
     state_bytes // (tp*pp) on each of its GPUs; every GPU has `gpu_capacity` bytes; Split needs room for the
     new sub-unit shards next to the old shard on each of the unit's GPUs and frees the old shard when it
     completes; Extend needs room for one shard on each target GPU; Merge needs room for the target shard

@@ -4,9 +4,9 @@
  * Plain, slow, single-threaded CPU oracle for the EMU reshard: the layout
  * change that carries one model-stage's parameter shards theta = {theta_i},
  * i = 1..tp*pp (EMU definition, Section 5) from a source (TP, PP) layout to a
- * target (TP, PP) layout.  Split and Merge "change placement and sharding
- * without changing logical state" (Section 6.2, "Preserving training
- * semantics"), and Split is a position-wise AllGather followed by a local
+ * target (TP, PP) layout.  Split and Merge move and re-cut state but leave
+ * the logical state as it was (Section 6.2, on preserving training
+ * semantics), and Split is a position-wise AllGather followed by a local
  * layout change (Section 6.2, "DAG Execution and Safety" and
  * "Resharding--transport interplay").  So the result has a plain definition
  * and this file is that definition written out, per logical tensor:
@@ -408,8 +408,8 @@ int oracle_reshard(const oracle_model* m, oracle_plan sp, oracle_plan dp,
     return ORACLE_OK;
 }
 
-/* k identical target units: what Extend leaves behind (Section 5.2(c): the new unit "holds replicated copies"
- * of theta and omega; use sp == dp) and what a Split into k replica units produces (Section 5.2(a)).  By
+/* k identical target units: what Extend leaves behind (Section 5.2(c): the new unit is a
+ * copy of theta and omega; use sp == dp) and what a Split into k replica units produces (Section 5.2(a)).  By
  * definition every unit is the plain reshard, so the oracle runs it once per unit.
  * dst_bufs is replica-major: unit 0's tp*pp shards, then unit 1's, ... */
 int oracle_reshard_replicated(const oracle_model* m, oracle_plan sp, oracle_plan dp, int replicas,

@@ -254,7 +254,7 @@ def reshard_replicated(model: Model, src: Plan, dst: Plan, replicas: int, src_bu
 def reshard_state(model: Model, src: Plan, dst: Plan, n_opt: int, src_bufs: list[np.ndarray],
                   fill: int = 0) -> list[np.ndarray]:
     """The EMU's state (theta, omega): the parameters src -> dst, and n_opt optimizer tensors per parameter that
-    "follow the same layout" (Section 5), held in fp32 on both sides and never cast.  Buffers on either side:
+    are sharded exactly like the parameters (Section 5), held in fp32 on both sides and never cast.  Buffers on either side:
     parameter shards, then the shards of optimizer tensor 0, then of tensor 1, ..."""
     ns = num_shards(model, src)
     out = reshard(model, src, dst, src_bufs[:ns], fill=fill)

@@ -237,7 +237,7 @@ def test_kv_head_replication(a, b):
 
 
 def test_non_nested_degrees():
-    """Split and Merge are defined for any integer factor between compatible layouts (Section 5.2): TP 3 <-> 2
+    """The primitives allow any integer ratio between compatible layouts, not only powers of two (Section 5.2): TP 3 <-> 2
     <-> 6 and PP 3 <-> 1, where destination slices straddle source slices."""
     sh = I.Shape(3, 192, 6, 6, 384, 768)                       # 6 q heads, 6 kv heads, head_dim 32
     for a, b in [((3, 1), (2, 3)), ((2, 3), (3, 1)), ((6, 1), (2, 1)), ((1, 3), (6, 1)), ((3, 3), (2, 1))]:

@@ -11,7 +11,7 @@ from paper_2609_34645_b200 import inputs as I
 
 
 def test_gate_statements_of_the_paper():
-    # "The ratio is the payback period": 12 s of transition against 1.5 s saved per step pays back in 8 steps
+    # the ratio counts the steps until the savings have paid for the move: 12 s of transition against 1.5 s saved per step pays back in 8 steps
     ok, pb = B.admit(12.0, 10.0, 8.5, gamma=0.5, h_x=16.0)
     assert pb == pytest.approx(8.0) and ok                      # 8 <= 0.5 * 16
     ok, _ = B.admit(12.0, 10.0, 8.5, gamma=0.5, h_x=15.9)
@@ -21,7 +21,7 @@ def test_gate_statements_of_the_paper():
     assert not ok and math.isinf(pb)
     ok, _ = B.admit(0.001, 10.0, 11.0, gamma=1.0, h_x=1e9)
     assert not ok
-    # "Setting gamma = 0 admits only urgent transitions", even free ones
+    # with gamma = 0 nothing but the urgent path gets through, not even a free transition
     assert not B.admit(0.0, 10.0, 5.0, gamma=0.0, h_x=100.0)[0]
     assert B.admit(1e6, 10.0, 12.0, gamma=0.0, h_x=0.0, urgent=True)[0]       # urgent waives profitability
     # the paper's 1,000-step run: six transitions, 49.5 s in all; a transition of 49.5/6 s that saves 1 s per

@@ -1,7 +1,7 @@
 """Pins of the CPU oracle against things other than itself (no GPU).
 
-The paper prints no worked numeric example of a reshard; what it fixes is the semantic contract "Split and
-Merge change placement and sharding without changing logical state" (Section 6.2) and one layout example,
+The paper prints no worked numeric example of a reshard; what it fixes is the semantic contract that Split and
+Merge re-cut and move state without touching the logical state (Section 6.2), and one layout example,
 (TP4, PP8) -> (TP4, PP2) units -> (TP8, PP2) (Section 6.1).  The pins are therefore: np.split /
 np.concatenate special cases, a brute-force per-element owner function, identity, round trips, checksum
 conservation, path independence through the paper's example, published parameter counts, and torch's

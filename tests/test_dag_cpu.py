@@ -238,3 +238,51 @@ def test_lowered_extend_then_merge():
     for k in range(2):
         for g, w in zip(got[8 + 8 * k:16 + 8 * k], want):
             assert np.array_equal(g, w)
+
+
+def test_lowered_random_dags_reach_the_target_state():
+    """Random plan changes of one or two model-stages on the MICRO shape: whatever mix of Split, Extend, Merge
+    and resource edges the planner produces, executing the lowered table level by level leaves every target
+    unit equal to the direct reshard of the stage's logical state into the target layout."""
+    sh = I.MICRO
+    m = omodel_of(sh)
+    rng = random.Random(11)
+    ran = 0
+    for trial in range(40):
+        changes, logical = [], []
+        for s in range(rng.randint(1, 2)):
+            def collection():
+                tp, pp = rng.choice([1, 2, 4, 8]), rng.choice([1, 2, 4])
+                units = []
+                for _ in range(rng.randint(1, 2)):
+                    first = rng.randrange(0, 64 - tp * pp + 1, tp * pp)
+                    units.append(D.Unit(tp, pp, tuple(range(first, first + tp * pp))))
+                return units
+            changes.append(D.StageChange(rng.choice([0, 1, 2]), collection(), collection(), 8 << 20))
+            logical.append(random_src(m, O.Plan(1, 1), 100 * trial + s, "bf16"))
+        try:
+            dag, t, descs = lowered(changes, [sh] * len(changes))
+        except B.NereusError as e:
+            assert e.code in (B.ERR_UNSUPPORTED, B.ERR_INFEASIBLE)
+            continue
+        units, prims = dag.units(), dag.prims()
+        created = {u for p in prims for u in p["dst"]}
+        src, dst_units = [], []
+        for u, (stage, tp, pp, gpus) in enumerate(units):
+            if u not in created:                       # DP replicas of a stage hold the same logical state
+                src += O.reshard(m, O.Plan(1, 1), O.Plan(tp, pp), logical[stage], fill=0xA5)
+            else:
+                dst_units.append(u)
+        n_src, n_dst = t.num_buffers()
+        assert n_src == len(src)
+        got = [np.full(t.buffer_bytes(True, j), 0xA5, np.uint8) for j in range(n_dst)]
+        interpret(t.rects(), src, got)
+        at = 0
+        for u in dst_units:
+            stage, tp, pp, gpus = units[u]
+            want = O.reshard(m, O.Plan(1, 1), O.Plan(tp, pp), logical[stage], fill=0xA5)
+            for g, w in zip(got[at:at + tp * pp], want):
+                assert np.array_equal(g, w), (trial, u)
+            at += tp * pp
+        ran += 1
+    assert ran >= 15

@@ -414,6 +414,9 @@ def run_ours(args):
     }
     if e2e is not None:
         line["e2e"] = e2e
+    per_stage = time_stages_alone(wl, keep, srcs, dsts, stream)
+    if per_stage:
+        line["config"]["ms_per_stage_alone"] = per_stage
     if not args.no_cpu_baseline and world == 1:
         try:
             from oracle import oracle as O
@@ -449,6 +452,32 @@ def host_memory_budget() -> int:
         except (OSError, ValueError):
             pass
     return avail
+
+
+def time_stages_alone(wl, keep, srcs, dsts, stream, runs=5):
+    """Multi-stage tables only: every model-stage's transition launched on its own (outside the timed region
+    of the metric), ms per launch by CUDA events."""
+    import torch
+
+    parts = keep[0]
+    if wl.dag or wl.round_trip or len(parts) < 2:
+        return None
+    out, si, di = {}, 0, 0
+    for st, part in zip(wl.stages, parts):
+        ns, nd = part.num_buffers()
+        sp = [b.data_ptr() for b in srcs[si:si + ns]]
+        dp = [b.data_ptr() for b in dsts[di:di + nd]]
+        si, di = si + ns, di + nd
+        for _ in range(2):
+            part.run(sp, dp, stream.cuda_stream)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(runs):
+            part.run(sp, dp, stream.cuda_stream)
+        b.record(stream)
+        stream.synchronize()
+        out[st.name] = a.elapsed_time(b) / runs
+    return out
 
 
 def run_e2e(args, t, srcs, dsts, sp, dp, stream, algo_bytes, world, device):

@@ -75,8 +75,11 @@ typedef struct {
 /* layout: bit 0 set = fused QKV stored group by group inside a rank's block (for each of the rank's kv heads: its
  * q heads, then its k head, then its v head) instead of [all Q; all K; all V]; bit 1 set = gate and up rows
  * interleaved row by row inside a rank's block (g0, u0, g1, u1, ...) instead of [all gate; all up].  Which
- * heads and rows a rank holds does not depend on the layout, only their order inside the fused block. */
-enum { ORACLE_QKV_GROUPED = 1, ORACLE_GATE_UP_INTERLEAVED = 2 };
+ * heads and rows a rank holds does not depend on these two, only their order inside the fused block.
+ * bit 2 set = the vocabulary dimension of embed and LM head is padded up to a multiple of 128*tp before it is
+ * cut (the habit of Megatron-style trainers): rank r stores V_pad/tp rows, of which those past row V are
+ * padding that no transition reads or writes; V need not divide by tp then. */
+enum { ORACLE_QKV_GROUPED = 1, ORACLE_GATE_UP_INTERLEAVED = 2, ORACLE_VOCAB_PADDED = 4 };
 typedef struct { int tp, pp, dtype, layout; } oracle_plan;
 
 /* kinds of logical tensor */
@@ -126,23 +129,39 @@ int oracle_logical_shape(const oracle_model* m, int64_t id, int64_t* rows, int64
 }
 
 int oracle_check_plan(const oracle_model* m, oracle_plan p) {
-    if (!m || p.tp < 1 || p.pp < 1 || (p.layout & ~3)) return ORACLE_ERR_ARG;
+    if (!m || p.tp < 1 || p.pp < 1 || (p.layout & ~7)) return ORACLE_ERR_ARG;
     if (m->L < 1 || m->H < 1 || m->nq < 1 || m->nkv < 1 || m->F < 1 || m->V < 1) return ORACLE_ERR_ARG;
     if (m->H % m->nq || m->nq % m->nkv) return ORACLE_ERR_INDIVISIBLE;
     /* tp <= nkv: whole kv heads per rank.  tp > nkv: every kv head is replicated on tp/nkv ranks, which needs
      * nkv | tp; a rank's q heads must then all belong to its one kv head, which tp | nq gives. */
     if (p.tp <= m->nkv ? m->nkv % p.tp : p.tp % m->nkv) return ORACLE_ERR_INDIVISIBLE;
-    if (m->nq % p.tp || m->F % p.tp || m->V % p.tp || m->L % p.pp) return ORACLE_ERR_INDIVISIBLE;
+    if (m->nq % p.tp || m->F % p.tp || m->L % p.pp) return ORACLE_ERR_INDIVISIBLE;
+    if (!(p.layout & ORACLE_VOCAB_PADDED) && m->V % p.tp) return ORACLE_ERR_INDIVISIBLE;
     return ORACLE_OK;
 }
 
 /* The part of a logical tensor of `kind` that TP rank r of t holds:
  * rows [*r0, *r0 + *nr), columns [*c0, *c0 + *nc) of the full tensor. */
-static void rank_part(const oracle_model* m, int kind, int64_t r, int64_t t,
+static int64_t padded_vocab(const oracle_model* m, int64_t t) {
+    return (m->V + 128 * t - 1) / (128 * t) * (128 * t);
+}
+
+static int vocab_cut(const oracle_model* m, int kind) {
+    return kind == K_EMBED || (kind == K_HEAD && !m->value_head);
+}
+
+static void rank_part(const oracle_model* m, oracle_plan pl, int kind, int64_t r,
                       int64_t* r0, int64_t* nr, int64_t* c0, int64_t* nc) {
-    int64_t rows, cols;
+    int64_t rows, cols, t = pl.tp;
     kind_shape(m, kind, &rows, &cols);
     *r0 = 0; *nr = rows; *c0 = 0; *nc = cols;
+    if (vocab_cut(m, kind) && (pl.layout & ORACLE_VOCAB_PADDED)) {
+        int64_t per = padded_vocab(m, t) / t, lo = r * per, hi = (r + 1) * per;   /* rows of the padded table */
+        if (lo > rows) lo = rows;
+        if (hi > rows) hi = rows;
+        *r0 = lo; *nr = hi - lo;                                /* the real rows among them, maybe none */
+        return;
+    }
     switch (kind) {
     case K_WK: case K_WV:
         if (t > m->nkv) {                                       /* replicated kv heads: rank r holds the one */
@@ -163,9 +182,11 @@ static void rank_part(const oracle_model* m, int kind, int64_t r, int64_t t,
 }
 
 /* Elements of `kind` stored by one TP rank of t. */
-static int64_t rank_elems(const oracle_model* m, int kind, int64_t t) {
+static int64_t rank_elems(const oracle_model* m, oracle_plan pl, int kind) {
     int64_t r0, nr, c0, nc;
-    rank_part(m, kind, 0, t, &r0, &nr, &c0, &nc);
+    if (vocab_cut(m, kind) && (pl.layout & ORACLE_VOCAB_PADDED))
+        return padded_vocab(m, pl.tp) / pl.tp * m->H;           /* padding rows take room in every shard */
+    rank_part(m, pl, kind, 0, &r0, &nr, &c0, &nc);
     return nr * nc;
 }
 
@@ -199,43 +220,43 @@ static int64_t part_rowpos(const oracle_model* m, oracle_plan pl, int kind, int6
  * stage does not hold it.  *total gets the shard buffer length. */
 static int64_t pack_offset(const oracle_model* m, oracle_plan pl, int64_t p,
                            int want_kind, int64_t want_layer, int64_t* total) {
-    int64_t es = plan_es(m, pl), t = pl.tp, cur = 0, found = -1;
+    int64_t es = plan_es(m, pl), cur = 0, found = -1;
     int64_t lps = m->L / pl.pp;
     if (p == 0) {
         cur = align256(cur);
         if (want_kind == K_EMBED) found = cur;
-        cur += rank_elems(m, K_EMBED, t) * es;
+        cur += rank_elems(m, pl, K_EMBED) * es;
     }
     for (int64_t l = p * lps; l < (p + 1) * lps; ++l) {
         int hit = (l == want_layer);
         cur = align256(cur);                                    /* ln1 */
         if (hit && want_kind == K_LN1) found = cur;
-        cur += rank_elems(m, K_LN1, t) * es;
+        cur += rank_elems(m, pl, K_LN1) * es;
         cur = align256(cur);                                    /* fused q;k;v: row 0 of each part */
         if (hit && (want_kind == K_WQ || want_kind == K_WK || want_kind == K_WV))
             found = cur + part_rowpos(m, pl, want_kind, 0) * m->H * es;
-        cur += (rank_elems(m, K_WQ, t) + rank_elems(m, K_WK, t) + rank_elems(m, K_WV, t)) * es;
+        cur += (rank_elems(m, pl, K_WQ) + rank_elems(m, pl, K_WK) + rank_elems(m, pl, K_WV)) * es;
         cur = align256(cur);                                    /* wo */
         if (hit && want_kind == K_WO) found = cur;
-        cur += rank_elems(m, K_WO, t) * es;
+        cur += rank_elems(m, pl, K_WO) * es;
         cur = align256(cur);                                    /* ln2 */
         if (hit && want_kind == K_LN2) found = cur;
-        cur += rank_elems(m, K_LN2, t) * es;
+        cur += rank_elems(m, pl, K_LN2) * es;
         cur = align256(cur);                                    /* fused gate;up: row 0 of each part */
         if (hit && (want_kind == K_WGATE || want_kind == K_WUP))
             found = cur + part_rowpos(m, pl, want_kind, 0) * m->H * es;
-        cur += (rank_elems(m, K_WGATE, t) + rank_elems(m, K_WUP, t)) * es;
+        cur += (rank_elems(m, pl, K_WGATE) + rank_elems(m, pl, K_WUP)) * es;
         cur = align256(cur);                                    /* wdown */
         if (hit && want_kind == K_WDOWN) found = cur;
-        cur += rank_elems(m, K_WDOWN, t) * es;
+        cur += rank_elems(m, pl, K_WDOWN) * es;
     }
     if (p == pl.pp - 1) {
         cur = align256(cur);
         if (want_kind == K_LNF) found = cur;
-        cur += rank_elems(m, K_LNF, t) * es;
+        cur += rank_elems(m, pl, K_LNF) * es;
         cur = align256(cur);
         if (want_kind == K_HEAD) found = cur;
-        cur += rank_elems(m, K_HEAD, t) * es;
+        cur += rank_elems(m, pl, K_HEAD) * es;
     }
     if (total) *total = align256(cur);
     return found;
@@ -273,7 +294,7 @@ int oracle_locate(const oracle_model* m, oracle_plan pl, int64_t shard, int64_t 
     off = pack_offset(m, pl, shard / pl.tp, kind, layer, NULL);
     *held = off >= 0;
     *offset = off >= 0 ? off : 0;
-    rank_part(m, kind, shard % pl.tp, pl.tp, r0, nr, c0, nc);
+    rank_part(m, pl, kind, shard % pl.tp, r0, nr, c0, nc);
     if (!*held) { *nr = 0; *nc = 0; }
     return ORACLE_OK;
 }

@@ -27,6 +27,7 @@ BF16 = 1
 FP32 = 2
 QKV_GROUPED = 1
 GATE_UP_INTERLEAVED = 2
+VOCAB_PADDED = 4
 
 OK = 0
 ERR_ARG = -1
@@ -83,7 +84,7 @@ class Plan:
     tp: int
     pp: int
     dtype: int = 0  # 0 = the model's dtype
-    layout: int = 0  # QKV_GROUPED | GATE_UP_INTERLEAVED
+    layout: int = 0  # QKV_GROUPED | GATE_UP_INTERLEAVED | VOCAB_PADDED
 
     def c(self) -> _Plan:
         return _Plan(self.tp, self.pp, self.dtype, self.layout)

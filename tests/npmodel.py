@@ -61,7 +61,7 @@ def position_coded(sh, es, salt, value_head=False):
     return out
 
 
-QKV_GROUPED, GATE_UP_INTERLEAVED = 1, 2
+QKV_GROUPED, GATE_UP_INTERLEAVED, VOCAB_PADDED = 1, 2, 4
 
 
 def _stored_blocks(sh, tp, pp, p, r, logical, value_head, layout=0):
@@ -77,6 +77,13 @@ def _stored_blocks(sh, tp, pp, p, r, logical, value_head, layout=0):
     def d1(x):
         return np.split(x, tp, axis=1)[r]
 
+    def dvocab(x):           # vocabulary rows: cut evenly, or padded to a multiple of 128*tp first
+        if not layout & VOCAB_PADDED:
+            return d0(x)
+        v_pad = -(-sh.vocab // (128 * tp)) * 128 * tp
+        filler = np.full((v_pad - sh.vocab, x.shape[1]), np.iinfo(x.dtype).max // 0xFF * 0xA5, x.dtype)   # 0xA5 bytes
+        return np.split(np.concatenate([x, filler], axis=0), tp, axis=0)[r]
+
     def dkv(x):              # kv heads: cut like any row block, or, past one head per rank, replicated
         if tp <= sh.kv_heads:
             return d0(x)
@@ -85,7 +92,7 @@ def _stored_blocks(sh, tp, pp, p, r, logical, value_head, layout=0):
     lps = sh.layers // pp
     blocks = []
     if p == 0:
-        blocks.append(d0(logical["embed"]))
+        blocks.append(dvocab(logical["embed"]))
     for l in range(p * lps, (p + 1) * lps):
         g = lambda k: logical[f"{k}.{l}"]
         blocks.append(g("ln1"))
@@ -106,7 +113,7 @@ def _stored_blocks(sh, tp, pp, p, r, logical, value_head, layout=0):
         blocks.append(d1(g("wdown")))
     if p == pp - 1:
         blocks.append(logical["ln_f"])
-        blocks.append(logical["head"] if value_head else d0(logical["head"]))
+        blocks.append(logical["head"] if value_head else dvocab(logical["head"]))
     return blocks
 
 

@@ -192,6 +192,31 @@ def test_kv_head_replication_against_np():
     assert e.value.code == O.ERR_REPLICA_MISMATCH
 
 
+def test_padded_vocabulary_against_np():
+    """Vocabulary padded to a multiple of 128*tp before the cut (np.concatenate with filler rows, then np.split):
+    the padding rows take room in the shards, are never read and never written, and V need not divide by tp."""
+    sh = I.Shape(2, 64, 4, 4, 128, 1000)                         # V = 1000: divisible by neither 128 nor 3... by 1, 2, 4
+    m = model_of(sh)
+    logical = npmodel.random_logical(sh, 2, seed=17)
+    assert O.check_plan(model_of(I.Shape(2, 64, 4, 4, 128, 1001)), O.Plan(2, 1)) == O.ERR_INDIVISIBLE
+    assert O.check_plan(model_of(I.Shape(2, 64, 4, 4, 128, 1001)), O.Plan(2, 1, 0, 4)) == O.OK
+    assert O.shard_bytes(m, O.Plan(4, 1, 0, 4), 0) > O.shard_bytes(m, O.Plan(4, 1), 0)      # 1024/4 vs 1000/4 rows
+    cases = [((1, 1, 0), (4, 2, 4)), ((4, 2, 4), (1, 1, 0)), ((2, 1, 4), (4, 1, 4)), ((4, 1, 4), (2, 2, 0)),
+             ((2, 2, 5), (4, 1, 6)), ((1, 2, 4), (1, 1, 4))]
+    for (ta, pa, la), (tb, pb, lb) in cases:
+        src = npmodel.build_shards(sh, ta, pa, logical, layout=la)
+        want = npmodel.build_shards(sh, tb, pb, logical, layout=lb)
+        got = O.reshard(m, O.Plan(ta, pa, 0, la), O.Plan(tb, pb, 0, lb), src, fill=0xA5)
+        for g, w in zip(got, want):
+            assert g.size == w.size and np.array_equal(g, w), ((ta, pa, la), (tb, pb, lb))
+    odd = I.Shape(2, 64, 4, 4, 128, 1001)                        # only the padded cut can shard this vocabulary
+    mo = model_of(odd)
+    lo = npmodel.random_logical(odd, 2, seed=18)
+    got = O.reshard(mo, O.Plan(1, 1), O.Plan(4, 1, 0, 4), npmodel.build_shards(odd, 1, 1, lo), fill=0xA5)
+    for g, w in zip(got, npmodel.build_shards(odd, 4, 1, lo, layout=4)):
+        assert np.array_equal(g, w)
+
+
 # ---------------------------------------------------------------- brute-force owner function
 
 @pytest.mark.parametrize("es", [2, 4])

@@ -86,9 +86,15 @@ typedef struct nereus_transition_s* nereus_transition_t;   /* opaque, host; owns
  *                               Megatron-style trainers keep), instead of [all Q ; all K ; all V]
  *   NEREUS_GATE_UP_INTERLEAVED  g0, u0, g1, u1, ... row by row (what some fused SwiGLU kernels read), instead
  *                               of [all gate ; all up]
- * A transition may convert between layouts, e.g. grouped fp32 training weights to blocked bf16 for generation. */
+ * A transition may convert between layouts, e.g. grouped fp32 training weights to blocked bf16 for generation.
+ *   NEREUS_VOCAB_PADDED         the vocabulary dimension of embed and LM head is padded up to a multiple of
+ *                               128*tp before it is cut (what Megatron-style trainers do): rank r stores
+ *                               V_pad/tp rows; rows past V are padding, never read and never written; V need
+ *                               not divide by tp under this flag
+ */
 #define NEREUS_QKV_GROUPED          1
 #define NEREUS_GATE_UP_INTERLEAVED  2
+#define NEREUS_VOCAB_PADDED         4
 
 /* A (TP, PP) layout.  dtype 0 means "the descriptor's dtype"; layout is a mask of the flags above. */
 typedef struct { int tp; int pp; int dtype; int layout; } nereus_plan_t;

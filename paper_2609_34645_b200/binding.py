@@ -17,6 +17,7 @@ FP32 = 2
 DTYPES = {"bf16": BF16, "fp32": FP32}
 QKV_GROUPED = 1
 GATE_UP_INTERLEAVED = 2
+VOCAB_PADDED = 4
 
 OK = 0
 ERR_ARG, ERR_INDIVISIBLE, ERR_UNSUPPORTED, ERR_ALIAS = -1, -2, -3, -4

@@ -17,13 +17,13 @@ namespace nereus {
 // ---------------------------------------------------------------------------------------------------
 
 static StoredTensor whole(int64_t rows, int64_t cols, int layer) {
-    return StoredTensor{Cut::Whole, 1, {rows, 0, 0}, {0, 0, 0}, cols, layer};
+    return StoredTensor{Cut::Whole, 1, {rows, 0, 0}, {0, 0, 0}, 0, cols, layer};
 }
 static StoredTensor by_rows(int nseg, int64_t r0, int64_t r1, int64_t r2, int64_t cols, int layer) {
-    return StoredTensor{Cut::Rows, nseg, {r0, r1, r2}, {0, 0, 0}, cols, layer};
+    return StoredTensor{Cut::Rows, nseg, {r0, r1, r2}, {0, 0, 0}, 0, cols, layer};
 }
 static StoredTensor by_cols(int64_t rows, int64_t cols, int layer) {
-    return StoredTensor{Cut::Cols, 1, {rows, 0, 0}, {0, 0, 0}, cols, layer};
+    return StoredTensor{Cut::Cols, 1, {rows, 0, 0}, {0, 0, 0}, 0, cols, layer};
 }
 
 void build_catalogue(nereus_model_desc_s& d) {
@@ -31,6 +31,7 @@ void build_catalogue(nereus_model_desc_s& d) {
     d.catalogue.clear();
     d.catalogue.reserve(6 * d.L + 3);
     d.catalogue.push_back(by_rows(1, d.V, 0, 0, d.H, -1));                                   // embed
+    d.catalogue.back().pad_to = 128;
     for (int l = 0; l < d.L; ++l) {
         d.catalogue.push_back(whole(1, d.H, l));                                             // ln1
         d.catalogue.push_back(by_rows(3, d.nq * hd, d.nkv * hd, d.nkv * hd, d.H, l));        // q;k;v
@@ -42,15 +43,17 @@ void build_catalogue(nereus_model_desc_s& d) {
     }
     d.catalogue.push_back(whole(1, d.H, -2));                                                // ln_f
     d.catalogue.push_back(d.value_head ? whole(1, d.H, -2) : by_rows(1, d.V, 0, 0, d.H, -2)); // head
+    if (!d.value_head) d.catalogue.back().pad_to = 128;
 }
 
 int check_plan(const nereus_model_desc_s& d, nereus_plan_t p) {
     if (p.tp < 1 || p.pp < 1) return NEREUS_ERR_ARG;
     if (p.dtype != 0 && p.dtype != NEREUS_BF16 && p.dtype != NEREUS_FP32) return NEREUS_ERR_ARG;
-    if (p.layout & ~(NEREUS_QKV_GROUPED | NEREUS_GATE_UP_INTERLEAVED)) return NEREUS_ERR_ARG;
+    if (p.layout & ~(NEREUS_QKV_GROUPED | NEREUS_GATE_UP_INTERLEAVED | NEREUS_VOCAB_PADDED)) return NEREUS_ERR_ARG;
     // tp <= nkv: whole kv heads per rank; tp > nkv: each kv head replicated on tp/nkv ranks (needs nkv | tp)
     if (p.tp <= d.nkv ? d.nkv % p.tp : p.tp % d.nkv) return NEREUS_ERR_INDIVISIBLE;
-    if (d.nq % p.tp || d.F % p.tp || d.V % p.tp || d.L % p.pp) return NEREUS_ERR_INDIVISIBLE;
+    if (d.nq % p.tp || d.F % p.tp || d.L % p.pp) return NEREUS_ERR_INDIVISIBLE;
+    if (!(p.layout & NEREUS_VOCAB_PADDED) && d.V % p.tp) return NEREUS_ERR_INDIVISIBLE;
     return NEREUS_OK;
 }
 
@@ -61,7 +64,17 @@ int owning_stage(const nereus_model_desc_s& d, int id, int pp) {
     return layer / (int)(d.L / pp);
 }
 
-void stored_block(const StoredTensor& t, int tp, int64_t& rows, int64_t& cols) {
+// Rows one rank keeps of a padded segment: the padded total cut evenly.
+static int64_t padded_share(const StoredTensor& t, int tp) {
+    const int64_t q = t.pad_to * tp;
+    return (t.seg_rows[0] + q - 1) / q * q / tp;
+}
+
+void stored_block(const StoredTensor& t, int tp, int layout, int64_t& rows, int64_t& cols) {
+    if (t.cut == Cut::Rows && t.pad_to && (layout & NEREUS_VOCAB_PADDED)) {
+        rows = padded_share(t, tp); cols = t.cols;      // padding rows take room in every shard
+        return;
+    }
     switch (t.cut) {
     case Cut::Whole: rows = t.seg_rows[0]; cols = t.cols; break;
     case Cut::Cols:  rows = t.seg_rows[0]; cols = t.cols / tp; break;
@@ -73,7 +86,16 @@ void stored_block(const StoredTensor& t, int tp, int64_t& rows, int64_t& cols) {
     }
 }
 
-void segment_share(const StoredTensor& t, int s, int r, int tp, int64_t& lo, int64_t& n, bool& primary) {
+void segment_share(const StoredTensor& t, int s, int r, int tp, int layout, int64_t& lo, int64_t& n,
+                   bool& primary) {
+    if (t.pad_to && (layout & NEREUS_VOCAB_PADDED)) {
+        // the real rows among the rank's share of the padded table (none on ranks that hold padding only)
+        const int64_t per = padded_share(t, tp);
+        lo = std::min<int64_t>((int64_t)r * per, t.seg_rows[s]);
+        n = std::min<int64_t>((int64_t)(r + 1) * per, t.seg_rows[s]) - lo;
+        primary = true;
+        return;
+    }
     const int64_t even = t.seg_rows[s] / tp;
     if (even >= t.seg_unit[s]) { lo = r * even; n = even; primary = true; return; }
     // fewer rows than one unit per rank: units are replicated, `copies` consecutive ranks hold the same unit
@@ -91,7 +113,7 @@ void stage_layout(const nereus_model_desc_s& d, nereus_plan_t p, int stage, Stag
     for (int id = 0; id < n; ++id) {          // the catalogue order is the packing order
         if (owning_stage(d, id, p.pp) != stage) continue;
         int64_t rows, cols;
-        stored_block(d.catalogue[id], p.tp, rows, cols);
+        stored_block(d.catalogue[id], p.tp, p.layout, rows, cols);
         cur = round_up(cur, 256);
         out.offset[id] = cur;
         cur += (uint64_t)rows * (uint64_t)cols * es;
@@ -123,7 +145,7 @@ void row_pieces(const nereus_model_desc_s& d, const StoredTensor& x, int layout,
                 std::vector<RowPiece>& out) {
     out.clear();
     int64_t lo[3], n[3]; bool primary[3];
-    for (int s = 0; s < x.nseg; ++s) segment_share(x, s, r, t, lo[s], n[s], primary[s]);
+    for (int s = 0; s < x.nseg; ++s) segment_share(x, s, r, t, layout, lo[s], n[s], primary[s]);
     if (x.nseg == 3 && (layout & NEREUS_QKV_GROUPED)) {
         const int64_t hd = d.H / d.nq, heads = n[1] / hd;          // kv heads this rank holds
         const int64_t q_rows = n[0] / heads, group_rows = q_rows + 2 * hd;
@@ -220,10 +242,11 @@ static int compile_one(const nereus_model_desc_s& d, nereus_plan_t sp, nereus_pl
                     r.rows = 1; r.width_dst = (uint64_t)x.seg_rows[0] * x.cols * des;
                     em.emit(r);
                 } else if (x.cut == Cut::Rows) {
-                    if (ts == td && sp.layout == dp.layout) {
+                    if (ts == td && sp.layout == dp.layout && !(x.pad_to && (dp.layout & NEREUS_VOCAB_PADDED))) {
                         // same cut and same order on both sides: the rank's stored block moves as one run
+                        // (a padded block goes the general way, which leaves its padding rows alone)
                         int64_t brows, bcols;
-                        stored_block(x, td, brows, bcols);
+                        stored_block(x, td, dp.layout, brows, bcols);
                         r.src_buf = ps * ts + rd;
                         r.src_off = soff; r.dst_off = doff;
                         r.rows = 1; r.width_dst = (uint64_t)brows * bcols * des;
@@ -407,7 +430,7 @@ int nereus_plan_tensor_slice(nereus_model_desc_t d, nereus_plan_t p, int shard, 
     if (replicated) *replicated = d->catalogue[tensor_id].cut == Cut::Whole;
     if (sl.offset[tensor_id] == kNotHeld) { *offset = 0; *rows = 0; *cols = 0; return NEREUS_OK; }
     int64_t r, c;
-    stored_block(d->catalogue[tensor_id], p.tp, r, c);
+    stored_block(d->catalogue[tensor_id], p.tp, p.layout, r, c);
     *offset = (size_t)sl.offset[tensor_id]; *rows = (size_t)r; *cols = (size_t)c;
     return NEREUS_OK;
     NEREUS_GUARD_END

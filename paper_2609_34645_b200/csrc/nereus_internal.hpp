@@ -27,6 +27,8 @@ struct StoredTensor {
     int64_t seg_rows[3]; // Rows: logical rows of each segment; Whole/Cols: seg_rows[0] = rows
     int64_t seg_unit[3]; // Rows: smallest block of rows a rank may hold (head_dim for K and V, else 0): when a
                          //       rank's share would be smaller, the block is replicated over ranks instead
+    int64_t pad_to;      // Rows, one segment: with NEREUS_VOCAB_PADDED the rows are padded to a multiple of
+                         //       pad_to * tp before the cut (128 for embed and LM head, else 0)
     int64_t cols;        // logical columns (the contiguous dimension)
     int     layer;       // owning layer, -1 embed (first stage), -2 final norm / head (last stage)
 };
@@ -60,10 +62,10 @@ constexpr uint64_t kNotHeld = ~0ull;
 int  owning_stage(const nereus_model_desc_s& d, int id, int pp);
 void stage_layout(const nereus_model_desc_s& d, nereus_plan_t p, int stage, StageLayout& out);
 // Rows x cols (elements) of the block one TP rank of `tp` stores for tensor `t`.
-void stored_block(const StoredTensor& t, int tp, int64_t& rows, int64_t& cols);
+void stored_block(const StoredTensor& t, int tp, int layout, int64_t& rows, int64_t& cols);
 // Segment s of a Rows-cut tensor on rank r of t: first logical row, row count, and whether r is the first
 // rank holding these rows (false on the later copies of a replicated block).
-void segment_share(const StoredTensor& t, int s, int r, int tp, int64_t& lo, int64_t& n, bool& primary);
+void segment_share(const StoredTensor& t, int s, int r, int tp, int layout, int64_t& lo, int64_t& n, bool& primary);
 
 // ---------------------------------------------------------------------------------------------------
 // Task table

@@ -31,6 +31,7 @@ DENSE_32B = Shape(64, 5120, 40, 8, 27648, 152064)  # 32B-shaped decoder
 
 QKV_GROUPED = 1            # layout flags of a plan: order of the rows inside a rank's fused blocks
 GATE_UP_INTERLEAVED = 2
+VOCAB_PADDED = 4
 
 
 def layout_of(plan: tuple) -> int:

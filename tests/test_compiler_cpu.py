@@ -172,11 +172,11 @@ def check_transition(sh, a, b, sdt="bf16", ddt="bf16", vh=False, seed=0, la=0, l
     rects = t.rects()
     interpret(rects, src, got, counts)
     m_dst = omodel_of(sh, odt[ddt], vh)
-    for j, (g, w, c, mask) in enumerate(zip(got, want, counts, payload_mask(m_dst, O.Plan(b[0], b[1])))):
+    for j, (g, w, c, mask) in enumerate(zip(got, want, counts, payload_mask(m_dst, O.Plan(b[0], b[1], 0, lb & 4)))):
         assert np.array_equal(g, w), (a, b, j)
         assert np.array_equal(c == 1, mask), "every payload byte written exactly once, padding never"
     rd, wr = t.bytes()
-    assert wr == sum(int(mk.sum()) for mk in payload_mask(m_dst, O.Plan(b[0], b[1])))
+    assert wr == sum(int(mk.sum()) for mk in payload_mask(m_dst, O.Plan(b[0], b[1], 0, lb & 4)))
     assert rd == wr * (2 if sdt != ddt else 1)
     for r in rects:
         assert r.src_off % 16 == 0 and r.dst_off % 16 == 0 and r.width_bytes_dst % 16 == 0
@@ -218,7 +218,7 @@ def test_layout_variant_task_shapes():
     rects = t.rects()
     pitched = {(r.rows, r.width_bytes_dst, r.src_pitch) for r in rects if r.rows > 1 and r.width_bytes_dst == 8192}
     assert pitched == {(14336 // 4, 8192, 32768)}             # gate / up rows picked out of the interleaved source
-    assert d.plan_check(B.Plan(2, 2, 0, 4)) == B.ERR_ARG       # unknown layout flag
+    assert d.plan_check(B.Plan(2, 2, 0, 8)) == B.ERR_ARG       # unknown layout flag
     same = d.compile(B.Plan(2, 2, 0, 3), B.Plan(2, 2, 0, 3))
     assert all(r.rows == 1 for r in same.rects())              # same layout on both sides: runs only
 
@@ -243,6 +243,22 @@ def test_non_nested_degrees():
     for a, b in [((3, 1), (2, 3)), ((2, 3), (3, 1)), ((6, 1), (2, 1)), ((1, 3), (6, 1)), ((3, 3), (2, 1))]:
         check_transition(sh, a, b, seed=4)
         check_transition(sh, a, b, "fp32", "bf16", seed=5, la=1, lb=2)
+
+
+def test_padded_vocabulary():
+    """NEREUS_VOCAB_PADDED on either side: padding rows take room, are never read and never written; a vocabulary
+    that tp does not divide can only be cut this way."""
+    sh = I.Shape(2, 64, 4, 4, 128, 1000)
+    for (a, la), (b, lb) in [(((1, 1), 0), ((4, 2), 4)), (((4, 2), 4), ((1, 1), 0)), (((2, 1), 4), ((4, 1), 4)),
+                             (((4, 1), 4), ((2, 2), 0)), (((2, 2), 5), ((4, 1), 6)), (((2, 1), 4), ((2, 1), 4))]:
+        check_transition(sh, a, b, seed=7, la=la, lb=lb)
+        check_transition(sh, a, b, "fp32", "bf16", seed=8, la=la, lb=lb)
+    odd = I.Shape(2, 64, 4, 4, 128, 1001)
+    d = desc_of(odd)
+    assert d.plan_check(B.Plan(2, 1)) == B.ERR_INDIVISIBLE and d.plan_check(B.Plan(2, 1, 0, 4)) == B.OK
+    check_transition(odd, (1, 1), (4, 1), seed=9, la=0, lb=4)
+    d8 = desc_of(I.Shape(2, 64, 4, 4, 128, 1000))
+    assert d8.shard_bytes(B.Plan(4, 1, 0, 4), 0) > d8.shard_bytes(B.Plan(4, 1), 0)
 
 
 def test_value_head_and_fp32():

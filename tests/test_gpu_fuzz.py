@@ -13,25 +13,28 @@ from paper_2609_34645_b200 import inputs as I
 pytestmark = pytest.mark.gpu
 
 SHAPES = [I.SMALL, I.MICRO, I.TINY, I.Shape(2, 128, 16, 2, 256, 256), I.Shape(3, 192, 6, 3, 384, 768),
-          I.Shape(3, 192, 6, 6, 384, 768)]              # 6 kv heads: TP 2 and 3 do not nest
+          I.Shape(3, 192, 6, 6, 384, 768),              # 6 kv heads: TP 2 and 3 do not nest
+          I.Shape(2, 64, 4, 4, 128, 1000)]              # vocabulary that only tp 1, 2, 4 divide
 
 
-def valid_plans(sh):
+def valid_plans(sh, padded=False):
     out = []
     for tp in (1, 2, 3, 4, 6, 8, 16):
         for pp in (1, 2, 3, 4, 8):
             kv_ok = sh.kv_heads % tp == 0 if tp <= sh.kv_heads else tp % sh.kv_heads == 0
-            if kv_ok and sh.heads % tp == 0 and sh.ffn % tp == 0 and sh.vocab % tp == 0 and sh.layers % pp == 0:
+            if kv_ok and sh.heads % tp == 0 and sh.ffn % tp == 0 and (padded or sh.vocab % tp == 0) \
+                    and sh.layers % pp == 0:
                 out.append((tp, pp))
     return out
 
 
 def draw(rng):
     sh = rng.choice(SHAPES)
-    a, b = rng.choice(valid_plans(sh)), rng.choice(valid_plans(sh))
+    pad_a, pad_b = (4 if rng.random() < 0.25 else 0), (4 if rng.random() < 0.25 else 0)   # padded vocabulary
+    a, b = rng.choice(valid_plans(sh, pad_a)), rng.choice(valid_plans(sh, pad_b))
     sdt = rng.choice(["bf16", "bf16", "fp32"])
     ddt = "bf16" if sdt == "bf16" else rng.choice(["fp32", "bf16"])
-    return dict(sh=sh, a=a, b=b, sdt=sdt, ddt=ddt, la=rng.randrange(4), lb=rng.randrange(4),
+    return dict(sh=sh, a=a, b=b, sdt=sdt, ddt=ddt, la=rng.randrange(4) | pad_a, lb=rng.randrange(4) | pad_b,
                 vh=rng.random() < 0.25, k=rng.choice([1, 1, 1, 2, 3]), variant=rng.choice([1, 2]),
                 tile=rng.choice([512, 1024, 4096, 16384]))
 

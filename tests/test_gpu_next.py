@@ -327,3 +327,25 @@ def test_mixed_cast_and_copy_table(variant):
     for g, w in zip(dst.bufs, want):
         assert np.array_equal(g.cpu().numpy(), w)
     assert dst.guards_intact()
+
+
+@pytest.mark.parametrize("variant", [1, 2])
+def test_padded_vocabulary_on_the_gpu(variant):
+    """Vocabulary padded to a multiple of 128*tp on either side: padding rows stay as they were (sentinel)."""
+    sh = I.Shape(2, 64, 4, 4, 128, 1000)
+    for (a, la), (b, lb), sdt, ddt in [(((1, 1), 0), ((4, 2), 4), "bf16", "bf16"),
+                                       (((4, 2), 4), ((2, 1), 0), "bf16", "bf16"),
+                                       (((2, 1), 4), ((4, 1), 4), "fp32", "bf16"),
+                                       (((4, 1), 5), ((2, 2), 6), "fp32", "fp32")]:
+        desc = G.desc_of(sh, sdt)
+        pa, pb = B.Plan(a[0], a[1], 0, la), B.Plan(b[0], b[1], B.DTYPES[ddt], lb)
+        t = desc.compile(pa, pb)
+        t.tune(variant=variant, tile_bytes=1024)
+        src = G.device_sources_by_oracle(sh, O.Plan(a[0], a[1], 0, la), sdt, 41)
+        dst = G.Guarded([t.buffer_bytes(True, j) for j in range(t.num_buffers()[1])])
+        G.run_transition(t, src, dst.bufs)
+        want = O.reshard(G.omodel_of(sh, sdt), O.Plan(a[0], a[1], 0, la), O.Plan(b[0], b[1], G.ODT[ddt], lb),
+                         [s.cpu().numpy() for s in src], fill=G.SENTINEL)
+        for g, w in zip(dst.bufs, want):
+            assert np.array_equal(g.cpu().numpy(), w)
+        assert dst.guards_intact()

@@ -333,8 +333,8 @@ int nereus_dag_lower(nereus_dag_t dag, const nereus_model_desc_t* descs, int n_d
  * and at a near-capacity boundary the table upload of nereus_transition_prepare may fail.
  *
  * Same contract, arguments and result as nereus_transition_run, but it calls no cudaMalloc, cudaFree or any
- * other allocating routine and never touches the handle's device copy: the task table and the control
- * words go into one fixed array in the library's device image, NEREUS_STATIC_MAX_RECTS tasks at most
+ * other allocating routine, on the device or on the host heap, and never touches the handle's device copy:
+ * the task table and the control words go into one fixed array in the library's device image, NEREUS_STATIC_MAX_RECTS tasks at most
  * (about 272 KiB, held on every GPU the process uses until it exits).  The table is copied there on
  * `cuda_stream` by every call (two small cudaMemcpyAsync and a memset ahead of the kernel).
  *   - A transition with more tasks (nereus_transition_num_rects) is refused with NEREUS_ERR_TOO_LARGE.

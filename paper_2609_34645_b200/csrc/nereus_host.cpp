@@ -311,10 +311,16 @@ static void finish(nereus_transition_s& t) {
 
 uint64_t tile_table(const nereus_transition_s& t, uint32_t tile_bytes, std::vector<RectDev>& out,
                     std::vector<uint32_t>& first, uint32_t level_end[kMaxLevels]) {
-    out.clear(); first.clear();
-    out.reserve(t.rects.size()); first.reserve(t.rects.size() + 1);
+    out.resize(t.rects.size());
+    first.resize(t.rects.size() + 1);
+    return tile_table_raw(t, tile_bytes, out.data(), first.data(), level_end);
+}
+
+uint64_t tile_table_raw(const nereus_transition_s& t, uint32_t tile_bytes, RectDev* out, uint32_t* first,
+                        uint32_t level_end[kMaxLevels]) {
     for (int k = 0; k < kMaxLevels; ++k) level_end[k] = 0;
     uint64_t total = 0;
+    size_t   i = 0;
     for (const Rect& r : t.rects) {
         RectDev q{};
         q.src_off = r.src_off; q.dst_off = r.dst_off; q.width = r.width_dst;
@@ -338,12 +344,12 @@ uint64_t tile_table(const nereus_transition_s& t, uint32_t tile_bytes, std::vect
         }
         if (total + ntiles > 0xFFFFFFF0ull) return 0;
         q.first_tile = (uint32_t)total;
-        first.push_back((uint32_t)total);
+        first[i] = (uint32_t)total;
         total += ntiles;
         level_end[r.level] = (uint32_t)total;
-        out.push_back(q);
+        out[i++] = q;
     }
-    first.push_back((uint32_t)total);
+    first[i] = (uint32_t)total;
     for (int k = 1; k < kMaxLevels; ++k) level_end[k] = std::max(level_end[k], level_end[k - 1]);
     return total;
 }

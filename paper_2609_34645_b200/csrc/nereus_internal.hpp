@@ -190,6 +190,10 @@ namespace nereus {
 uint64_t tile_table(const nereus_transition_s& t, uint32_t tile_bytes, std::vector<RectDev>& out,
                     std::vector<uint32_t>& first, uint32_t level_end[kMaxLevels]);
 
+// Same into caller-provided arrays (rects.size() entries and rects.size() + 1 entries): no allocation.
+uint64_t tile_table_raw(const nereus_transition_s& t, uint32_t tile_bytes, RectDev* out, uint32_t* first,
+                        uint32_t level_end[kMaxLevels]);
+
 void set_cuda_error(int e);
 
 }  // namespace nereus

@@ -1056,17 +1056,21 @@ extern "C" int nereus_transition_run_static(nereus_transition_t t, const void* c
         if (int rc = resolve_launch(*t, sms, L)) return rc;
 
         WalkParams p;
-        std::vector<RectDev>  rects;        // host memory only
-        std::vector<uint32_t> first;
-        const uint64_t n_tiles = tile_table(*t, (uint32_t)L.tile_bytes, rects, first, p.level_end);
-        if (n_tiles == 0 && !t->rects.empty()) return NEREUS_ERR_UNSUPPORTED;
+        // the tiled table is built in fixed host arrays of the calling thread: no heap allocation either
+        static thread_local RectDev  rects[kStaticMaxRects];
+        static thread_local uint32_t first[kStaticMaxRects + 1];
+        const size_t   n_rects = t->rects.size();
+        const uint64_t n_tiles = tile_table_raw(*t, (uint32_t)L.tile_bytes, rects, first, p.level_end);
+        if (n_tiles == 0 && n_rects != 0) return NEREUS_ERR_UNSUPPORTED;
 
         RectDev*  d_rects = reinterpret_cast<RectDev*>(scratch);
         uint32_t* d_first = reinterpret_cast<uint32_t*>(scratch + kStaticRectBytes);
         Ctrl*     d_ctrl  = reinterpret_cast<Ctrl*>(scratch + kStaticRectBytes + kStaticFirstBytes);
         // the array keeps whatever the previous call left: overwrite the table, zero the control words
-        NEREUS_CUDA(cudaMemcpyAsync(d_rects, rects.data(), rects.size() * sizeof(RectDev), cudaMemcpyHostToDevice, stream));
-        NEREUS_CUDA(cudaMemcpyAsync(d_first, first.data(), first.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, stream));
+        // pageable host memory: the runtime has staged the bytes by the time each call returns, so the arrays may
+        // be reused by the next call
+        NEREUS_CUDA(cudaMemcpyAsync(d_rects, rects, n_rects * sizeof(RectDev), cudaMemcpyHostToDevice, stream));
+        NEREUS_CUDA(cudaMemcpyAsync(d_first, first, (n_rects + 1) * sizeof(uint32_t), cudaMemcpyHostToDevice, stream));
         NEREUS_CUDA(cudaMemsetAsync(d_ctrl, 0, sizeof(Ctrl), stream));
 
         p.rects = d_rects; p.first = d_first; p.ctrl = d_ctrl;

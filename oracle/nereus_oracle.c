@@ -32,7 +32,8 @@
  *   model      L layers, hidden H, nq query heads, nkv KV heads, hd = H / nq,
  *              FFN F, vocabulary V, element size es (2 = bf16, 4 = fp32),
  *              optional value head [1, H] in place of the LM head [V, H].
- *   plan       (tp, pp): pipeline stage p owns layers [p*L/pp, (p+1)*L/pp),
+ *   plan       (tp, pp): pipeline stage p owns layers [p*L/pp, (p+1)*L/pp) (when pp does not
+ *              divide L, the first L mod pp stages own one layer more than the others),
  *              the embedding lives on stage 0, final norm + head on stage
  *              pp-1; shard index = p * tp + r  (TP rank fastest).
  *   TP rank r of t holds
@@ -135,7 +136,8 @@ int oracle_check_plan(const oracle_model* m, oracle_plan p) {
     /* tp <= nkv: whole kv heads per rank.  tp > nkv: every kv head is replicated on tp/nkv ranks, which needs
      * nkv | tp; a rank's q heads must then all belong to its one kv head, which tp | nq gives. */
     if (p.tp <= m->nkv ? m->nkv % p.tp : p.tp % m->nkv) return ORACLE_ERR_INDIVISIBLE;
-    if (m->nq % p.tp || m->F % p.tp || m->L % p.pp) return ORACLE_ERR_INDIVISIBLE;
+    if (m->nq % p.tp || m->F % p.tp) return ORACLE_ERR_INDIVISIBLE;
+    if (p.pp > m->L) return ORACLE_ERR_INDIVISIBLE;         /* every stage needs a layer */
     if (!(p.layout & ORACLE_VOCAB_PADDED) && m->V % p.tp) return ORACLE_ERR_INDIVISIBLE;
     return ORACLE_OK;
 }
@@ -221,13 +223,16 @@ static int64_t part_rowpos(const oracle_model* m, oracle_plan pl, int kind, int6
 static int64_t pack_offset(const oracle_model* m, oracle_plan pl, int64_t p,
                            int want_kind, int64_t want_layer, int64_t* total) {
     int64_t es = plan_es(m, pl), cur = 0, found = -1;
-    int64_t lps = m->L / pl.pp;
+    /* layers [first, last) of stage p: an even cut; when pp does not divide L the first L mod pp stages hold
+     * one layer more (the split numpy's array_split makes) */
+    int64_t base = m->L / pl.pp, extra = m->L % pl.pp;
+    int64_t first = p * base + (p < extra ? p : extra), last = first + base + (p < extra ? 1 : 0);
     if (p == 0) {
         cur = align256(cur);
         if (want_kind == K_EMBED) found = cur;
         cur += rank_elems(m, pl, K_EMBED) * es;
     }
-    for (int64_t l = p * lps; l < (p + 1) * lps; ++l) {
+    for (int64_t l = first; l < last; ++l) {
         int hit = (l == want_layer);
         cur = align256(cur);                                    /* ln1 */
         if (hit && want_kind == K_LN1) found = cur;

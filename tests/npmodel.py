@@ -89,11 +89,11 @@ def _stored_blocks(sh, tp, pp, p, r, logical, value_head, layout=0):
             return d0(x)
         return np.split(x, sh.kv_heads, axis=0)[r // (tp // sh.kv_heads)]
 
-    lps = sh.layers // pp
+    mine = np.array_split(np.arange(sh.layers), pp)[p]      # an uneven cut gives the first stages one layer more
     blocks = []
     if p == 0:
         blocks.append(dvocab(logical["embed"]))
-    for l in range(p * lps, (p + 1) * lps):
+    for l in mine:
         g = lambda k: logical[f"{k}.{l}"]
         blocks.append(g("ln1"))
         if layout & QKV_GROUPED:
@@ -143,7 +143,7 @@ def owner(sh, tp, pp, es, name, i, j, value_head=False, layout=0):
     hd = sh.hidden // sh.heads
     H, F, V = sh.hidden, sh.ffn, sh.vocab
     nq, nkv = sh.heads, sh.kv_heads
-    lps = sh.layers // pp
+    bounds = [(int(c[0]), int(c[-1]) + 1) for c in np.array_split(np.arange(sh.layers), pp)]
     qr, kr, fr, vr = nq * hd // tp, nkv * hd // tp, F // tp, V // tp
     up = lambda x: -(-x // 256) * 256
     # byte sizes of the stored blocks of one layer, in order
@@ -154,7 +154,7 @@ def owner(sh, tp, pp, es, name, i, j, value_head=False, layout=0):
         cur = 0
         if p == 0:
             cur = up(cur) + vr * H * es
-        for _ in range(p * lps, l):
+        for _ in range(bounds[p][0], l):
             for _, n in layer_blocks:
                 cur = up(cur) + n * es
         return cur
@@ -174,7 +174,7 @@ def owner(sh, tp, pp, es, name, i, j, value_head=False, layout=0):
         return [(0 * tp + r, up(0) + ((i % vr) * H + j) * es)]
     if name in ("ln_f", "head"):
         p = pp - 1
-        cur = layer_base(p, (p + 1) * lps)
+        cur = layer_base(p, bounds[p][1])
         lnf = up(cur)
         head = up(lnf + H * es)
         if name == "ln_f":
@@ -185,7 +185,7 @@ def owner(sh, tp, pp, es, name, i, j, value_head=False, layout=0):
         return [(p * tp + r, head + ((i % vr) * H + j) * es)]
     kind, l = name.split(".")
     l = int(l)
-    p = l // lps
+    p = next(k for k, (lo, hi) in enumerate(bounds) if lo <= l < hi)
     base = layer_base(p, l)
     blk = {"ln1": 0, "wq": 1, "wk": 1, "wv": 1, "wo": 2, "ln2": 3, "wgate": 4, "wup": 4, "wdown": 5}[kind]
     start = within_layer(blk)(base)

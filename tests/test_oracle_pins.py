@@ -217,6 +217,23 @@ def test_padded_vocabulary_against_np():
         assert np.array_equal(g, w)
 
 
+def test_uneven_pipeline_cut_against_np():
+    """pp that does not divide the layer count: the first L mod pp stages hold one layer more (np.array_split)."""
+    sh = I.Shape(7, 64, 4, 4, 128, 256)
+    m = model_of(sh)
+    logical = npmodel.random_logical(sh, 2, seed=23)
+    pls = [(1, 1), (2, 2), (1, 3), (4, 4), (2, 5), (1, 7)]
+    assert O.check_plan(m, O.Plan(1, 8)) == O.ERR_INDIVISIBLE      # more stages than layers
+    for a, b in itertools.product(pls, repeat=2):
+        src = npmodel.build_shards(sh, a[0], a[1], logical)
+        want = npmodel.build_shards(sh, b[0], b[1], logical)
+        got = O.reshard(m, O.Plan(*a), O.Plan(*b), src, fill=0xA5)
+        for g, w in zip(got, want):
+            assert g.size == w.size and np.array_equal(g, w), (a, b)
+    sizes = [O.shard_bytes(m, O.Plan(1, 3), s) for s in range(3)]   # 3 + 2 + 2 layers
+    assert sizes[0] > sizes[1]
+
+
 # ---------------------------------------------------------------- brute-force owner function
 
 @pytest.mark.parametrize("es", [2, 4])
@@ -440,7 +457,7 @@ def test_refusals():
     m = model_of(I.TINY)
     assert O.check_plan(m, O.Plan(4, 1)) == O.OK                    # tp > kv_heads: kv heads replicated
     assert O.check_plan(m, O.Plan(8, 1)) == O.ERR_INDIVISIBLE       # more ranks than q heads
-    assert O.check_plan(m, O.Plan(1, 4)) == O.ERR_INDIVISIBLE       # 2 layers over 4 stages
+    assert O.check_plan(m, O.Plan(1, 4)) == O.ERR_INDIVISIBLE       # 2 layers over 4 stages: a stage without a layer
     assert O.check_plan(model_of(I.Shape(2, 256, 4, 2, 689, 1024)), O.Plan(2, 1)) == O.ERR_INDIVISIBLE
     assert O.check_plan(m, O.Plan(0, 1)) == O.ERR_ARG
     src = _random_src(model_of(I.TINY, O.BF16), O.Plan(1, 1), 0, "bf16")

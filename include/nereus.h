@@ -26,7 +26,8 @@
  *   logical tensors, row-major [out, in]:
  *            embed [V,H]; per layer ln1 [H], wq [nq*hd,H], wk [nkv*hd,H], wv [nkv*hd,H], wo [H,nq*hd],
  *            ln2 [H], wgate [F,H], wup [F,H], wdown [H,F]; ln_f [H]; head [V,H] (or a value head [1,H]).
- *   plan     (tp, pp, dtype).  Pipeline stage p owns layers [p*L/pp, (p+1)*L/pp); embed lives on stage 0,
+ *   plan     (tp, pp, dtype).  Pipeline stage p owns layers [p*L/pp, (p+1)*L/pp) (when pp does not divide L the
+ *            first L mod pp stages own one layer more than the others); embed lives on stage 0,
  *            ln_f and the head on stage pp-1.  Shard index = p*tp + r (TP rank r fastest).
  *   TP rank r of t stores
  *            embed, LM head   rows [r*V/t, (r+1)*V/t)                        (vocabulary-parallel)
@@ -45,7 +46,7 @@
  *   layout variants (nereus_plan_t.layout) reorder the rows inside qkv and gate_up, see the flags below.
  *   tp > nkv (nkv | tp): every kv head is replicated on tp/nkv consecutive ranks; rank r stores head
  *            r / (tp/nkv), the one its q heads attend to; as a source only the first copy of a head is read.
- *   required: tp | nkv or nkv | tp, tp | nq, tp | F, tp | V, pp | L, and every contiguous piece
+ *   required: tp | nkv or nkv | tp, tp | nq, tp | F, tp | V (unless padded), pp <= L, and every contiguous piece
  *            a transition moves must start on and span a multiple of 16 bytes on both sides (for the cast: 8
  *            elements).
  */

@@ -52,7 +52,8 @@ int check_plan(const nereus_model_desc_s& d, nereus_plan_t p) {
     if (p.layout & ~(NEREUS_QKV_GROUPED | NEREUS_GATE_UP_INTERLEAVED | NEREUS_VOCAB_PADDED)) return NEREUS_ERR_ARG;
     // tp <= nkv: whole kv heads per rank; tp > nkv: each kv head replicated on tp/nkv ranks (needs nkv | tp)
     if (p.tp <= d.nkv ? d.nkv % p.tp : p.tp % d.nkv) return NEREUS_ERR_INDIVISIBLE;
-    if (d.nq % p.tp || d.F % p.tp || d.L % p.pp) return NEREUS_ERR_INDIVISIBLE;
+    if (d.nq % p.tp || d.F % p.tp) return NEREUS_ERR_INDIVISIBLE;
+    if (p.pp > d.L) return NEREUS_ERR_INDIVISIBLE;                   // every stage needs a layer
     if (!(p.layout & NEREUS_VOCAB_PADDED) && d.V % p.tp) return NEREUS_ERR_INDIVISIBLE;
     return NEREUS_OK;
 }
@@ -61,7 +62,9 @@ int owning_stage(const nereus_model_desc_s& d, int id, int pp) {
     const int layer = d.catalogue[id].layer;
     if (layer == -1) return 0;
     if (layer == -2) return pp - 1;
-    return layer / (int)(d.L / pp);
+    // even cut; when pp does not divide L the first L mod pp stages own one layer more
+    const int base = (int)(d.L / pp), extra = (int)(d.L % pp), big = extra * (base + 1);
+    return layer < big ? layer / (base + 1) : extra + (layer - big) / base;
 }
 
 // Rows one rank keeps of a padded segment: the padded total cut evenly.

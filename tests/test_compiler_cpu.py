@@ -92,7 +92,7 @@ def test_argument_errors():
     d = desc_of(I.TINY)
     assert d.plan_check(B.Plan(4, 1)) == B.OK                      # tp > kv_heads: kv heads are replicated
     assert d.plan_check(B.Plan(8, 1)) == B.ERR_INDIVISIBLE         # more ranks than q heads
-    assert d.plan_check(B.Plan(1, 4)) == B.ERR_INDIVISIBLE
+    assert d.plan_check(B.Plan(1, 4)) == B.ERR_INDIVISIBLE         # 2 layers over 4 stages
     assert d.plan_check(B.Plan(0, 1)) == B.ERR_ARG
     assert d.plan_check(B.Plan(1, 1, 7)) == B.ERR_ARG
     with pytest.raises(B.NereusError) as e:
@@ -259,6 +259,14 @@ def test_padded_vocabulary():
     check_transition(odd, (1, 1), (4, 1), seed=9, la=0, lb=4)
     d8 = desc_of(I.Shape(2, 64, 4, 4, 128, 1000))
     assert d8.shard_bytes(B.Plan(4, 1, 0, 4), 0) > d8.shard_bytes(B.Plan(4, 1), 0)
+
+
+def test_uneven_pipeline_cut():
+    """pp that does not divide the layer count, on either side."""
+    sh = I.Shape(7, 64, 4, 4, 128, 256)
+    for a, b in [((1, 1), (2, 3)), ((2, 3), (4, 4)), ((4, 4), (1, 7)), ((2, 5), (2, 2)), ((1, 7), (1, 3))]:
+        check_transition(sh, a, b, seed=11)
+        check_transition(sh, a, b, "fp32", "bf16", seed=12, la=3, lb=0)
 
 
 def test_value_head_and_fp32():

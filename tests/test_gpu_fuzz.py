@@ -14,7 +14,8 @@ pytestmark = pytest.mark.gpu
 
 SHAPES = [I.SMALL, I.MICRO, I.TINY, I.Shape(2, 128, 16, 2, 256, 256), I.Shape(3, 192, 6, 3, 384, 768),
           I.Shape(3, 192, 6, 6, 384, 768),              # 6 kv heads: TP 2 and 3 do not nest
-          I.Shape(2, 64, 4, 4, 128, 1000)]              # vocabulary that only tp 1, 2, 4 divide
+          I.Shape(2, 64, 4, 4, 128, 1000),              # vocabulary that only tp 1, 2, 4 divide
+          I.Shape(7, 64, 4, 4, 128, 256)]               # 7 layers: uneven pipeline cuts
 
 
 def valid_plans(sh, padded=False):
@@ -23,7 +24,7 @@ def valid_plans(sh, padded=False):
         for pp in (1, 2, 3, 4, 8):
             kv_ok = sh.kv_heads % tp == 0 if tp <= sh.kv_heads else tp % sh.kv_heads == 0
             if kv_ok and sh.heads % tp == 0 and sh.ffn % tp == 0 and (padded or sh.vocab % tp == 0) \
-                    and sh.layers % pp == 0:
+                    and pp <= sh.layers:
                 out.append((tp, pp))
     return out
 

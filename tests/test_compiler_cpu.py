@@ -466,3 +466,18 @@ int main(void) {
                            "-o", str(exe), "-L", libdir, "-lnereus", f"-Wl,-rpath,{libdir}"])
     out = subprocess.check_output([str(exe)], text=True).split()
     assert out[0] == out[1] == str(1_975_552 * 2) and int(out[2]) > 0
+
+
+def test_binding_fails_loudly_without_the_library(tmp_path):
+    """No CPU fallback: importing the binding next to no libnereus.so raises, it never degrades to something
+    else."""
+    import shutil
+    import subprocess
+    import sys
+    pkg = tmp_path / "paper_2609_34645_b200"
+    pkg.mkdir()
+    for name in ("__init__.py", "binding.py"):
+        shutil.copy(os.path.join(ROOT, "paper_2609_34645_b200", name), pkg / name)
+    r = subprocess.run([sys.executable, "-c", "import paper_2609_34645_b200.binding"], cwd=tmp_path,
+                       capture_output=True, text=True)
+    assert r.returncode != 0 and "ImportError" in r.stderr and "no CPU fallback" in r.stderr

@@ -355,6 +355,9 @@ int oracle_reshard_tensor_parts(const oracle_model* m, oracle_plan sp, oracle_pl
         if (!part) { free(full); return ORACLE_ERR_ARG; }
         int repeat = 0;
         for (int q = 0; q < n_seen; ++q) repeat |= (seen_r0[q] == r0 && seen_c0[q] == c0);
+        /* a guard, not arithmetic: more distinct parts than the record holds (tp > 64) is refused rather than
+         * checked against an incomplete record */
+        if (!repeat && n_seen == 64) { free(full); return ORACLE_ERR_UNSUPPORTED; }
         for (int64_t i = 0; i < nr; ++i) {
             int64_t at = oracle_part_row(m, sp, id, i);                 /* where the plan's layout keeps row i */
             for (int64_t j = 0; j < nc; ++j) {
@@ -364,7 +367,7 @@ int oracle_reshard_tensor_parts(const oracle_model* m, oracle_plan sp, oracle_pl
                 else if (memcmp(to, from, (size_t)ses) != 0) { free(full); return ORACLE_ERR_REPLICA_MISMATCH; }
             }
         }
-        if (!repeat && n_seen < 64) { seen_r0[n_seen] = r0; seen_c0[n_seen] = c0; ++n_seen; }
+        if (!repeat) { seen_r0[n_seen] = r0; seen_c0[n_seen] = c0; ++n_seen; }
     }
 
     /* 2. CAST */

@@ -132,6 +132,64 @@ def test_any_plan_pair_against_np_split():
             assert np.array_equal(g, w), (a, b)
 
 
+def test_replicated_units_against_np_split():
+    """k target units (a Split into k replica units, a weight sync to k units, Extend): unit r of the result is
+    numpy's shard image of the target plan, for every r; with equal plans (Extend) every unit is the source image
+    itself.  Target plans with pp > 1 and tp > 1 make a wrong unit stride land in the wrong buffer."""
+    sh = I.MICRO
+    m = model_of(sh)
+    logical = npmodel.random_logical(sh, 2, seed=21)
+    images = {pl: npmodel.build_shards(sh, pl[0], pl[1], logical) for pl in [(1, 1), (2, 2), (4, 2), (8, 1), (2, 4)]}
+    for (a, b), k in itertools.product(itertools.product(images, images), (1, 2, 3)):
+        got = O.reshard_replicated(m, O.Plan(*a), O.Plan(*b), k, images[a], fill=0xA5)
+        n = b[0] * b[1]
+        assert len(got) == k * n
+        for r in range(k):
+            for j in range(n):
+                assert np.array_equal(got[r * n + j], images[b][j]), (a, b, k, r, j)
+            if a == b:
+                for j in range(n):
+                    assert np.array_equal(got[r * n + j], images[a][j])
+
+
+def test_state_with_optimizer_tensors_against_np_split():
+    """(theta, omega): bf16 parameters and n_opt fp32 tensors of the parameters' layout, each with contents of
+    its own, so that a slice of the buffer list taken at the wrong place, or a cast applied to omega, shows."""
+    sh = I.MICRO
+    m = model_of(sh)
+    theta = npmodel.random_logical(sh, 2, seed=31)
+    omega = [npmodel.random_logical(sh, 4, seed=32 + k) for k in range(3)]
+    for a, b in [((2, 2), (4, 1)), ((4, 2), (1, 1)), ((1, 1), (2, 4)), ((8, 1), (8, 1))]:
+        for n_opt in (0, 1, 3):
+            src = npmodel.build_shards(sh, a[0], a[1], theta)
+            want = npmodel.build_shards(sh, b[0], b[1], theta)
+            for k in range(n_opt):
+                src += npmodel.build_shards(sh, a[0], a[1], omega[k])
+                want += npmodel.build_shards(sh, b[0], b[1], omega[k])
+            got = O.reshard_state(m, O.Plan(*a), O.Plan(*b), n_opt, src, fill=0xA5)
+            assert len(got) == len(want) == (1 + n_opt) * b[0] * b[1]
+            for j, (g, w) in enumerate(zip(got, want)):
+                assert g.size == w.size and np.array_equal(g, w), (a, b, n_opt, j)
+    # omega stays fp32 when theta is cast: the parameters come out as torch's bf16 of the fp32 values
+    m32 = model_of(sh, O.FP32)
+    th32 = npmodel.random_logical(sh, 4, seed=41)
+    src = npmodel.build_shards(sh, 2, 2, th32) + npmodel.build_shards(sh, 2, 2, omega[0])
+    got = O.reshard_state(m32, O.Plan(2, 2), O.Plan(4, 1, O.BF16), 1, src, fill=0xA5)
+    th16 = {n: O.rne_bf16_array(x).reshape(x.shape) for n, x in th32.items()}
+    want = npmodel.build_shards(sh, 4, 1, th16) + npmodel.build_shards(sh, 4, 1, omega[0])
+    for j, (g, w) in enumerate(zip(got, want)):
+        assert np.array_equal(g, w), j
+
+
+def test_more_distinct_parts_than_the_replica_record_holds_is_refused():
+    sh = I.Shape(1, 1024, 128, 128, 256, 256)
+    m = model_of(sh)
+    src = [np.zeros(O.shard_bytes(m, O.Plan(128, 1), s), np.uint8) for s in range(128)]
+    with pytest.raises(O.OracleError) as e:
+        O.reshard(m, O.Plan(128, 1), O.Plan(1, 1), src)
+    assert e.value.code == O.ERR_UNSUPPORTED
+
+
 @pytest.mark.parametrize("sh", [I.TINY, I.MICRO])
 def test_layout_variants_against_np(sh):
     """Grouped QKV and row-interleaved gate/up on either side: shards built by numpy (reshape to head groups,

@@ -63,19 +63,23 @@ extern "C" {
 #define NEREUS_OK                 0
 #define NEREUS_ERR_ARG           -1   /* null pointer, negative or zero size, index out of range          */
 #define NEREUS_ERR_INDIVISIBLE   -2   /* a divisibility or 16-byte rule of the layout contract fails       */
-#define NEREUS_ERR_UNSUPPORTED   -3   /* dtype pair other than same->same or fp32->bf16;                   */
-                                      /* more buffers than one launch can address                          */
+#define NEREUS_ERR_UNSUPPORTED   -3   /* dtype pair other than same->same or fp32->bf16; more buffers than */
+                                      /* one launch can address; a call that is not allowed in this state  */
 #define NEREUS_ERR_ALIAS         -4   /* a destination buffer overlaps a source or another destination     */
 #define NEREUS_ERR_CUDA          -5   /* a CUDA call failed; see nereus_last_cuda_error                    */
 #define NEREUS_ERR_NOMEM         -6   /* host allocation failed                                            */
 #define NEREUS_ERR_MISMATCH      -7   /* parts of a chained fuse do not connect (buffer count or sizes)    */
 #define NEREUS_ERR_ALIGN         -8   /* a shard pointer is not 16-byte aligned                            */
 #define NEREUS_ERR_TOO_LARGE     -9   /* more tasks than the fixed scratch of nereus_transition_run_static */
+/* -10 is NEREUS_ERR_INFEASIBLE, declared with the transition DAG below */
+#define NEREUS_ERR_TABLE         -11  /* the task table failed the host-side check that precedes every upload */
 
 /* device status word (nereus_transition_status) */
 #define NEREUS_DEV_OK             0
 #define NEREUS_DEV_BOUNDS         1   /* a claimed tile did not resolve to a task: corrupted table         */
-#define NEREUS_DEV_TIMEOUT        2   /* a dependency wait gave up after its poll limit                    */
+#define NEREUS_DEV_TIMEOUT        2   /* a wait inside the kernel gave up: a dependency gate after about   */
+                                      /* 0.5 s of polling, a shared-memory barrier after 0.5 s on the GPU's */
+                                      /* global timer (with a cap of 2^22 attempts behind it)              */
 
 typedef enum { NEREUS_BF16 = 1, NEREUS_FP32 = 2 } nereus_dtype_t;
 
@@ -184,6 +188,17 @@ int nereus_transition_num_rects(nereus_transition_t t, int* n);
 int nereus_transition_get_rect(nereus_transition_t t, int index, nereus_rect_t* out);
 /* Tiles one run claims, and dependency levels. */
 int nereus_transition_num_tiles(nereus_transition_t t, uint64_t* tiles, int* levels);
+/* Checks the task table on the host, as nereus_transition_prepare and nereus_transition_run_static do before
+ * anything reaches a device (Section 6.2, "Safe concurrent execution": a buffer is only read or written inside
+ * its declared extent and nothing writes where another task of the same step writes): every task lies inside
+ * nereus_transition_buffer_bytes of its source and of each destination replica, offsets, widths and pitches
+ * follow the 16-byte rule, a pitch is at least a width, buffer indices and levels are in range and in
+ * execution order, a chained task reads only what an earlier level wrote, and the destinations of all tasks
+ * are pairwise disjoint.  Errors: ARG, NEREUS_ERR_TABLE, NOMEM. */
+int nereus_transition_validate(nereus_transition_t t);
+/* Test hook: overwrites task `index` of a table that has not been uploaded yet, without any check, so that the
+ * validator can be shown a corrupted table.  Errors: ARG, UNSUPPORTED (the table is already on a device). */
+int nereus_debug_set_rect(nereus_transition_t t, int index, const nereus_rect_t* task);
 
 /* Launch tuning; 0 keeps the default of a field.  tile_bytes: target bytes per claimed tile (multiple of
  * 512).  ctas_per_sm, threads: persistent grid = SMs * ctas_per_sm blocks of `threads` threads.
@@ -201,8 +216,10 @@ int nereus_transition_launch_info(nereus_transition_t t, int* variant, int* tile
 
 /* ---- execution (the local layout change of Section 6.2) ---------------------------------------------- */
 
-/* Uploads the task table to the current device (cudaMalloc + synchronous copy).  Optional: run() does it
- * on first use.  Call it ahead of time to keep allocation out of a timed or captured region. */
+/* Checks the task table (nereus_transition_validate, plus the tiling) and uploads it to the current device
+ * (cudaMalloc + synchronous copy).  Optional: run() does it on first use.  Call it ahead of time to keep
+ * allocation out of a timed or captured region.  Tables of up to 2^17 tiles also get one 48-byte record per
+ * tile, which saves the kernel the search for a tile's task.  Errors: ARG, UNSUPPORTED, NEREUS_ERR_TABLE, CUDA. */
 int nereus_transition_prepare(nereus_transition_t t);
 /* Enqueues the whole transition on `cuda_stream` (a cudaStream_t; NULL = the default stream) as one
  * persistent kernel and returns without synchronising.
@@ -212,7 +229,11 @@ int nereus_transition_prepare(nereus_transition_t t);
  * Both arrays are copied before the call returns.  Every pointer must be 16-byte aligned and address at
  * least nereus_transition_buffer_bytes bytes.  Sources stay live until the stream reaches the end of the
  * run (Section 6.2: source buffers live until their readers complete).
- * Errors: ARG (null), ALIGN, ALIAS, CUDA.  Runs of the same handle must not overlap on the device. */
+ * A prepared run enqueues nothing but the kernel: the control words are left zeroed by every launch (the last
+ * block to finish clears them), so the launch may be captured into a CUDA graph and replayed, each replay
+ * moving whatever the buffers hold by then.
+ * Errors: ARG (null), ALIGN, ALIAS, CUDA, and what prepare reports.  Runs of the same handle must not overlap
+ * on the device. */
 int nereus_transition_run(nereus_transition_t t, const void* const* src_ptrs, void* const* dst_ptrs,
                           void* cuda_stream);
 /* Environment variables read by run(): NEREUS_TILE_BYTES, NEREUS_CTAS_PER_SM, NEREUS_THREADS, NEREUS_VARIANT
@@ -221,8 +242,9 @@ int nereus_transition_run(nereus_transition_t t, const void* const* src_ptrs, vo
  * the gate cannot open; the waits then run into their poll limit (about half a second), the run ends with
  * device status NEREUS_DEV_TIMEOUT and the destinations of the gated levels stay unwritten. */
 
-/* Reads the device status word of the last run (NEREUS_DEV_*).  The caller must have synchronised the
- * stream first; this call copies 4 bytes from the device synchronously. */
+/* Reads the device status word (NEREUS_DEV_*): the first failure of any run of this handle since the word was
+ * last read, NEREUS_DEV_OK if there was none; a failure that has been read is cleared.  The caller must have
+ * synchronised the stream first; this call copies a few bytes from the device synchronously. */
 int nereus_transition_status(nereus_transition_t t, int* device_status);
 /* Kernels this handle has launched since it was created (one per run). */
 int nereus_transition_launches(nereus_transition_t t, uint64_t* n);
@@ -265,8 +287,9 @@ int nereus_horizon_crossing(nereus_horizon_t* h, double interval_steps);
  *     k = tp*pp / |T_sub| replica units on the unit's own GPUs, sub-unit j on GPUs [j*|T_sub|, (j+1)*|T_sub|);
  *   - the target units' GPUs are cut into slots the same way; a slot that already holds a sub-unit (same
  *     GPUs, same order) keeps it; every other sub-unit is redundant and gets a Destroy; every other slot is
- *     filled by an Extend from the lowest-numbered kept sub-unit (else the lowest-numbered one), and a unit
- *     that an Extend still reads is destroyed only after it; Merge fuses a target unit's slots;
+ *     filled by an Extend from the lowest-numbered kept sub-unit that shares no GPU with the slot (else the
+ *     lowest-numbered such sub-unit at all: Extend copies onto a disjoint GPU set), and a unit that an Extend
+ *     still reads is destroyed only after it; Merge fuses a target unit's slots;
  *   - resources are bytes of GPU memory: a unit keeps state_bytes / (tp*pp) on each of its GPUs, every GPU
  *     has gpu_capacity bytes; Split / Extend / Merge need room for what they create, Split / Destroy / Merge
  *     free what they consume when they complete;
@@ -301,7 +324,8 @@ int nereus_dag_add_stage(nereus_dag_t dag, int kind, uint64_t state_bytes, int* 
 /* Adds a unit to a stage's current (is_target = 0) or target collection; gpus (host) has tp*pp entries. */
 int nereus_dag_add_unit(nereus_dag_t dag, int stage, int is_target, int tp, int pp, const int* gpus);
 /* Plans.  gpu_capacity 0 = unlimited.  Errors: ARG (a stage without units, mixed layouts inside a collection,
- * a layout T_sub does not divide), NEREUS_ERR_INFEASIBLE. */
+ * a layout T_sub does not divide), UNSUPPORTED (a target slot that overlaps every unit it could be copied
+ * from without coinciding with one), NEREUS_ERR_INFEASIBLE. */
 int nereus_dag_plan(nereus_dag_t dag, uint64_t gpu_capacity);
 int nereus_dag_num_units(nereus_dag_t dag, int* n);          /* current units first, then created ones */
 int nereus_dag_unit(nereus_dag_t dag, int unit, int* stage, int* tp, int* pp, int* gpus, int gpus_cap);
@@ -322,7 +346,8 @@ int nereus_dag_prim_lists(nereus_dag_t dag, int prim, int* src, int* dst, int* d
  * src_ptrs the shards of the current units, unit by unit in unit order, and as dst_ptrs the shards of every
  * created unit (sub-units, extended units, target units) in unit order; a destroyed unit's memory may be
  * reused for a unit created after the last primitive that reads it.
- * Errors: ARG (not planned), UNSUPPORTED (more than 8 data-moving levels or too many buffers), and whatever
+ * Errors: ARG (not planned, or planned without success: an infeasible DAG has no schedule to lower),
+ * UNSUPPORTED (more than 8 data-moving levels or too many buffers), and whatever
  * nereus_transition_compile reports for a layout. */
 int nereus_dag_lower(nereus_dag_t dag, const nereus_model_desc_t* descs, int n_descs, nereus_transition_t* out);
 
@@ -335,20 +360,34 @@ int nereus_dag_lower(nereus_dag_t dag, const nereus_model_desc_t* descs, int n_d
  *
  * Same contract, arguments and result as nereus_transition_run, but it calls no cudaMalloc, cudaFree or any
  * other allocating routine, on the device or on the host heap, and never touches the handle's device copy:
- * the task table and the control words go into one fixed array in the library's device image, NEREUS_STATIC_MAX_RECTS tasks at most
- * (about 272 KiB, held on every GPU the process uses until it exits).  The table is copied there on
- * `cuda_stream` by every call (two small cudaMemcpyAsync and a memset ahead of the kernel).
- *   - A transition with more tasks (nereus_transition_num_rects) is refused with NEREUS_ERR_TOO_LARGE.
+ * the task table and the control words go into one fixed array in the library's device image,
+ * NEREUS_STATIC_MAX_RECTS tasks at most (about 272 KiB, held on every GPU the process uses until it exits),
+ * and the host side stages the table in fixed arrays of the library's own image.  The table is checked
+ * (as by nereus_transition_validate) and copied there on `cuda_stream` by every call (two small
+ * cudaMemcpyAsync and a 12-byte memset ahead of the kernel).
+ *   - A transition with more tasks (nereus_transition_num_rects), or with more than 4 * NEREUS_STATIC_MAX_RECTS
+ *     (task, replica) pairs, is refused with NEREUS_ERR_TOO_LARGE.
  *   - The first call on a device looks the array's device address up (cudaGetSymbolAddress) and reads the
- *     SM count; make that first call outside any stream capture.
+ *     SM count.  While `cuda_stream` is being captured the call is refused with NEREUS_ERR_UNSUPPORTED: the
+ *     table is uploaded from host arrays that the next call overwrites, so a captured upload would replay
+ *     whichever table came last.
+ *   - The uploads read pageable host memory: the runtime takes the bytes before each copy call returns, and
+ *     to do so it may wait for earlier work of the stream.  Unlike nereus_transition_run the call can
+ *     therefore block for as long as the stream's backlog.
  *   - All handles and all calls on one device share the array, which keeps the previous call's contents
  *     until the next one overwrites it: two calls whose work overlaps on the GPU (different streams, or
- *     different threads) race on it.  Issue them on one stream, or order them with events.
- *   - nereus_transition_status does not see these runs: their status word lives in the shared array and is
- *     not exported.  It only ever matters for chained tables (a dependency wait that gives up). */
+ *     different threads) race on it.  Issue them on one stream, or order them with events.  (Host threads
+ *     are serialised by a lock around the staging arrays; that does not order their work on the GPU.)
+ *   - nereus_transition_status does not see these runs: their status word lives in the shared array; read
+ *     it with nereus_static_status. */
 #define NEREUS_STATIC_MAX_RECTS 4096
 int nereus_transition_run_static(nereus_transition_t t, const void* const* src_ptrs, void* const* dst_ptrs,
                                  void* cuda_stream);
+/* Device status (NEREUS_DEV_*) of the static runs on the current device: the first failure since the word was
+ * last read (NEREUS_DEV_OK if none, or if no static run was made on this device); reading clears it.  The
+ * caller must have synchronised the stream of those runs.  Allocates nothing; copies a few bytes from the
+ * device synchronously.  Like the entry point it serves, it has no counterpart in the paper. */
+int nereus_static_status(int* device_status);
 
 const char* nereus_strerror(int code);
 /* cudaError_t of the last failed CUDA call made by this library on the calling thread (0 if none). */

@@ -24,6 +24,7 @@ ERR_ARG, ERR_INDIVISIBLE, ERR_UNSUPPORTED, ERR_ALIAS = -1, -2, -3, -4
 ERR_CUDA, ERR_NOMEM, ERR_MISMATCH, ERR_ALIGN = -5, -6, -7, -8
 ERR_TOO_LARGE = -9
 ERR_INFEASIBLE = -10
+ERR_TABLE = -11
 GENERATION, INFERENCE, TRAINING = 0, 1, 2
 OP_SPLIT, OP_DESTROY, OP_EXTEND, OP_MERGE = 0, 1, 2, 3
 STATIC_MAX_RECTS = 4096
@@ -130,6 +131,9 @@ _SIGS = {
     "nereus_horizon_init": [_P(Horizon), ctypes.c_double],
     "nereus_horizon_crossing": [_P(Horizon), ctypes.c_double],
     "nereus_transition_run_static": [_vp, _P(_vp), _P(_vp), _vp],
+    "nereus_static_status": [_P(_i)],
+    "nereus_transition_validate": [_vp],
+    "nereus_debug_set_rect": [_vp, _i, _P(Rect)],
 }
 for _name, _args in _SIGS.items():
     _f = getattr(_lib, _name)          # AttributeError here = the library does not export a declared symbol
@@ -257,6 +261,17 @@ class Transition:
             out.append(r)
         return out
 
+    def validate(self) -> int:
+        """nereus_transition_validate: the host-side check of the task table; returns the error code."""
+        return _lib.nereus_transition_validate(self._h)
+
+    def debug_set_rect(self, index: int, rect: Rect) -> None:
+        """Test hook: overwrite one task of a table that has not been uploaded, unchecked."""
+        _ck(_lib.nereus_debug_set_rect(self._h, index, ctypes.byref(rect)), "nereus_debug_set_rect")
+
+    def prepare_raw(self) -> int:
+        return _lib.nereus_transition_prepare(self._h)
+
     def num_tiles(self):
         t, l = ctypes.c_uint64(), _i()
         _ck(_lib.nereus_transition_num_tiles(self._h, ctypes.byref(t), ctypes.byref(l)), "nereus_transition_num_tiles")
@@ -306,7 +321,8 @@ class Transition:
     def run_static(self, src_ptrs, dst_ptrs, stream=0):
         """nereus_transition_run_static: the same transition without any device allocation, for callers
         whose memory pool owns the whole GPU.  At most STATIC_MAX_RECTS tasks; calls that overlap on the
-        device race on the shared table; make the first call on a device outside stream capture."""
+        device race on the shared table; refused while the stream is being captured; its device status is
+        read with static_status()."""
         if not isinstance(src_ptrs, ctypes.Array):
             src_ptrs = self.pointer_array(src_ptrs)
         if not isinstance(dst_ptrs, ctypes.Array):
@@ -419,6 +435,13 @@ def admit(l_tran, l_step_current, l_step_target, gamma=0.5, h_x=1.0, urgent=Fals
     _ck(_lib.nereus_admit(l_tran, l_step_current, l_step_target, gamma, h_x, int(urgent), ctypes.byref(a),
                           ctypes.byref(pb)), "nereus_admit")
     return bool(a.value), pb.value
+
+
+def static_status() -> int:
+    """nereus_static_status: device status of the static runs on the current device (reading clears it)."""
+    s = _i()
+    _ck(_lib.nereus_static_status(ctypes.byref(s)), "nereus_static_status")
+    return s.value
 
 
 def strerror(code: int) -> str:

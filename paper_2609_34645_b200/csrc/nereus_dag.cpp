@@ -80,14 +80,34 @@ struct Planner {
             auto it = at.find(sl.gpus);
             if (it != at.end() && !kept.count(it->second)) { kept.insert(it->second); sl.unit = it->second; }
         }
-        const int source = kept.empty() ? *std::min_element(subs.begin(), subs.end()) : *kept.begin();
         std::map<int, int> destroy_of;
+        std::map<int, std::vector<int>> readers;          // unit -> Extends that copy it
         for (int u : subs)
             if (!kept.count(u)) destroy_of[u] = add_prim(NEREUS_OP_DESTROY, m, {u}, {});
+        // Extend copies onto a GPU set disjoint from its source's (Section 5.2(c)): per empty slot, the
+        // lowest-numbered kept sub-unit that shares no GPU with the slot, else the lowest-numbered such sub-unit
+        // at all; a slot that overlaps every sub-unit without coinciding with one cannot be filled by the
+        // paper's primitives
+        auto disjoint = [this](int u, const std::vector<int>& gpus) {
+            for (int a : g.units[u].gpus)
+                if (std::find(gpus.begin(), gpus.end(), a) != gpus.end()) return false;
+            return true;
+        };
         for (Slot& sl : slots) {
             if (sl.unit >= 0) continue;
+            int source = -1;
+            for (int u : kept)
+                if (disjoint(u, sl.gpus)) { source = u; break; }
+            if (source < 0) {
+                std::vector<int> sorted_subs(subs);
+                std::sort(sorted_subs.begin(), sorted_subs.end());
+                for (int u : sorted_subs)
+                    if (disjoint(u, sl.gpus)) { source = u; break; }
+            }
+            if (source < 0) return NEREUS_ERR_UNSUPPORTED;
             sl.unit = add_unit(m, tps, pps, sl.gpus);
             const int e = add_prim(NEREUS_OP_EXTEND, m, {source}, {sl.unit});
+            readers[source].push_back(e);
             auto it = destroy_of.find(source);
             if (it != destroy_of.end()) g.prims[it->second].deps.insert(e);     // the last copy goes after the Extend
         }
@@ -98,7 +118,10 @@ struct Planner {
             for (const Slot& sl : slots)
                 if (sl.target == (int)t) mine.push_back(sl.unit);
             const int tu = add_unit(m, v.tp, v.pp, v.gpus);
-            add_prim(NEREUS_OP_MERGE, m, mine, {tu});
+            const int mg = add_prim(NEREUS_OP_MERGE, m, mine, {tu});
+            // a Merge frees the sub-units it fuses: like a Destroy it waits for the Extends that still copy them
+            for (int u : mine)
+                for (int e : readers[u]) g.prims[mg].deps.insert(e);
         }
         return NEREUS_OK;
     }
@@ -269,8 +292,10 @@ int nereus_dag_plan(nereus_dag_t dag, uint64_t gpu_capacity) {
             if (int rc = P.local_dag((int)m, current_ids[m])) return rc;
         for (const auto& ids : current_ids)
             for (int u : ids) P.occupy(u, true);
-        dag->planned = true;
-        return P.schedule();
+        dag->planned = true;                       // frozen from here on: units and primitives exist
+        const int rc = P.schedule();
+        dag->scheduled = rc == NEREUS_OK;          // only a complete schedule may be lowered
+        return rc;
     } catch (const std::bad_alloc&) { return NEREUS_ERR_NOMEM; }
 }
 

@@ -357,6 +357,143 @@ uint64_t tile_table_raw(const nereus_transition_s& t, uint32_t tile_bytes, RectD
     return total;
 }
 
+
+void expand_tiles(const RectDev* rects, size_t n_rects, TileRec* out) {
+    for (size_t i = 0; i < n_rects; ++i) {
+        const RectDev& q = rects[i];
+        const uint32_t row_blocks = (q.rows + q.rows_per_tile - 1) / q.rows_per_tile;
+        TileRec* o = out + q.first_tile;
+        for (uint32_t rb = 0; rb < row_blocks; ++rb) {
+            const uint32_t r0 = rb * q.rows_per_tile;
+            for (uint32_t cb = 0; cb < q.col_tiles; ++cb) {
+                const uint64_t c0 = (uint64_t)cb * q.tile_w;
+                TileRec e{};
+                e.src_off = q.src_off + (uint64_t)r0 * q.src_pitch + (c0 << q.cast);
+                e.dst_off = q.dst_off + (uint64_t)r0 * q.dst_pitch + c0;
+                e.src_pitch = q.src_pitch; e.dst_pitch = q.dst_pitch;
+                e.rows = std::min(q.rows_per_tile, q.rows - r0);
+                e.width = (uint32_t)std::min<uint64_t>(q.tile_w, q.width - c0);
+                e.src_buf = q.src_buf; e.dst_buf = q.dst_buf;
+                e.replicas = q.replicas; e.replica_stride = q.replica_stride;
+                e.level = q.level; e.cast = q.cast;
+                *o++ = e;
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// validator
+// ---------------------------------------------------------------------------------------------------
+
+namespace {
+
+typedef unsigned __int128 u128;
+
+// Last byte + 1 that a task touches in a buffer, from its first piece.
+inline u128 extent(uint64_t off, uint64_t rows, uint64_t pitch, uint64_t width) {
+    return (u128)off + (u128)(rows - 1) * pitch + width;
+}
+
+// Two destination footprints in one buffer whose bounding intervals overlap: do any of their pieces?
+bool pieces_overlap(const Rect& a, const Rect& b) {
+    if (a.rows == 1 && b.rows == 1) return true;
+    const Rect& lo = a.dst_off <= b.dst_off ? a : b;
+    const Rect& hi = a.dst_off <= b.dst_off ? b : a;
+    if (lo.rows > 1 && hi.rows > 1 && lo.dst_pitch == hi.dst_pitch) {
+        // same period: the later task's pieces sit in the gaps of the earlier one's, or they do not
+        const uint64_t d = (hi.dst_off - lo.dst_off) % lo.dst_pitch;
+        if (d >= lo.width_dst && d + hi.width_dst <= lo.dst_pitch) return false;
+    }
+    uint64_t i = 0, j = 0;                                   // exact: merge the two piece sequences
+    while (i < a.rows && j < b.rows) {
+        const u128 as = (u128)a.dst_off + (u128)i * a.dst_pitch, ae = as + a.width_dst;
+        const u128 bs = (u128)b.dst_off + (u128)j * b.dst_pitch, be = bs + b.width_dst;
+        if (ae <= bs) ++i; else if (be <= as) ++j; else return true;
+    }
+    return false;
+}
+
+}  // namespace
+
+int validate_table(const nereus_transition_s& t, const RectDev* tiled, const uint32_t* first, uint64_t n_tiles,
+                   uint32_t* order) {
+    const size_t ns = t.src_bytes.size(), nd = t.dst_bytes.size(), n = t.rects.size();
+    if (ns + nd > (size_t)kMaxBuffers || t.n_levels < 1 || t.n_levels > kMaxLevels) return NEREUS_ERR_TABLE;
+    if (t.dst_level.size() != nd) return NEREUS_ERR_TABLE;
+    int    prev_level = 0;
+    size_t n_entries = 0;
+    for (size_t i = 0; i < n; ++i) {
+        const Rect& r = t.rects[i];
+        if (r.level < prev_level || r.level >= t.n_levels) return NEREUS_ERR_TABLE;      // execution order
+        prev_level = r.level;
+        if ((r.cast != 0 && r.cast != 1) || r.rows == 0 || r.width_dst == 0 || (r.rows >> 32)) return NEREUS_ERR_TABLE;
+        if (r.replicas < 1 || r.replicas > kMaxReplicas || r.replica_stride < 0 ||
+            (r.replicas > 1 && r.replica_stride < 1)) return NEREUS_ERR_TABLE;
+        if (r.src_buf < 0 || (size_t)r.src_buf >= ns + nd) return NEREUS_ERR_TABLE;
+        if (r.dst_buf < (int64_t)ns ||
+            (size_t)r.dst_buf + (size_t)(r.replicas - 1) * r.replica_stride >= ns + nd) return NEREUS_ERR_TABLE;
+        const uint64_t ws = r.width_dst << r.cast;
+        if ((r.src_off | r.dst_off | r.width_dst) & 15) return NEREUS_ERR_TABLE;
+        if (r.rows > 1) {
+            if ((r.src_pitch | r.dst_pitch) & 15) return NEREUS_ERR_TABLE;
+            if (r.src_pitch < ws || r.dst_pitch < r.width_dst) return NEREUS_ERR_TABLE;   // pieces would overlap
+            if ((r.src_pitch >> 32) || (r.dst_pitch >> 32)) return NEREUS_ERR_TABLE;      // device form holds 32 bits
+        }
+        const uint64_t sbytes = (size_t)r.src_buf < ns ? t.src_bytes[r.src_buf] : t.dst_bytes[r.src_buf - ns];
+        if (extent(r.src_off, r.rows, r.src_pitch, ws) > sbytes) return NEREUS_ERR_TABLE;
+        // a chained task reads what an earlier level wrote, never its own level's output
+        if ((size_t)r.src_buf >= ns && t.dst_level[r.src_buf - ns] >= r.level) return NEREUS_ERR_TABLE;
+        for (int j = 0; j < r.replicas; ++j) {
+            const size_t d = (size_t)r.dst_buf - ns + (size_t)j * r.replica_stride;
+            if (extent(r.dst_off, r.rows, r.dst_pitch, r.width_dst) > t.dst_bytes[d]) return NEREUS_ERR_TABLE;
+            if (t.dst_level[d] != r.level) return NEREUS_ERR_TABLE;
+        }
+        n_entries += (size_t)r.replicas;
+        if (tiled) {
+            const RectDev& q = tiled[i];
+            if (q.src_off != r.src_off || q.dst_off != r.dst_off || q.width != r.width_dst || q.rows != r.rows ||
+                q.src_buf != r.src_buf || q.dst_buf != r.dst_buf || q.level != r.level || q.cast != r.cast ||
+                q.replicas != r.replicas || q.replica_stride != r.replica_stride ||
+                (r.rows > 1 && (q.src_pitch != r.src_pitch || q.dst_pitch != r.dst_pitch)))
+                return NEREUS_ERR_TABLE;
+            if (q.rows_per_tile == 0 || q.tile_w == 0 || q.col_tiles == 0 || (q.tile_w & 15)) return NEREUS_ERR_TABLE;
+            if (q.col_tiles > 1 && q.rows_per_tile != 1) return NEREUS_ERR_TABLE;
+            if ((uint64_t)q.col_tiles * q.tile_w < q.width || (uint64_t)(q.col_tiles - 1) * q.tile_w >= q.width)
+                return NEREUS_ERR_TABLE;
+            const uint64_t row_blocks = ((uint64_t)q.rows + q.rows_per_tile - 1) / q.rows_per_tile;
+            if (q.first_tile != first[i] || (uint64_t)first[i] + row_blocks * q.col_tiles != first[i + 1])
+                return NEREUS_ERR_TABLE;
+        }
+    }
+    if (tiled && first[n] != n_tiles) return NEREUS_ERR_TABLE;
+
+    // destinations pairwise disjoint: one entry per (task, replica), sorted by buffer and first byte; an entry is
+    // compared with the later ones that start inside its bounding interval
+    size_t k = 0;
+    for (size_t i = 0; i < n; ++i)
+        for (int j = 0; j < t.rects[i].replicas; ++j) order[k++] = (uint32_t)i | ((uint32_t)j << 24);
+    auto buf_of = [&t](uint32_t e) {
+        const Rect& r = t.rects[e & 0xFFFFFFu];
+        return (uint32_t)(r.dst_buf + (int)(e >> 24) * r.replica_stride);
+    };
+    std::sort(order, order + n_entries, [&](uint32_t x, uint32_t y) {
+        const uint32_t bx = buf_of(x), by = buf_of(y);
+        if (bx != by) return bx < by;
+        return t.rects[x & 0xFFFFFFu].dst_off < t.rects[y & 0xFFFFFFu].dst_off;
+    });
+    for (size_t a = 0; a < n_entries; ++a) {
+        const Rect& ra = t.rects[order[a] & 0xFFFFFFu];
+        const u128  end = extent(ra.dst_off, ra.rows, ra.dst_pitch, ra.width_dst);
+        for (size_t b = a + 1; b < n_entries && buf_of(order[b]) == buf_of(order[a]); ++b) {
+            const Rect& rb = t.rects[order[b] & 0xFFFFFFu];
+            if ((u128)rb.dst_off >= end) break;
+            if (pieces_overlap(ra, rb)) return NEREUS_ERR_TABLE;
+        }
+    }
+    return NEREUS_OK;
+}
+
 }  // namespace nereus
 
 // ---------------------------------------------------------------------------------------------------
@@ -592,9 +729,32 @@ int nereus_transition_get_rect(nereus_transition_t t, int index, nereus_rect_t* 
     return NEREUS_OK;
 }
 
+int nereus_transition_validate(nereus_transition_t t) {
+    NEREUS_GUARD_BEGIN
+    if (!t) return NEREUS_ERR_ARG;
+    size_t entries = 0;
+    for (const Rect& r : t->rects) entries += (size_t)std::max(1, std::min(r.replicas, kMaxReplicas));
+    if (t->rects.size() >= (1u << 24)) return NEREUS_ERR_UNSUPPORTED;
+    std::vector<uint32_t> order(entries + 1);
+    return validate_table(*t, nullptr, nullptr, 0, order.data());
+    NEREUS_GUARD_END
+}
+
+int nereus_debug_set_rect(nereus_transition_t t, int index, const nereus_rect_t* in) {
+    if (!t || !in || index < 0 || (size_t)index >= t->rects.size()) return NEREUS_ERR_ARG;
+    if (t->dev.rects) return NEREUS_ERR_UNSUPPORTED;          // only before the table has reached a device
+    Rect& r = t->rects[index];
+    r.src_buf = in->src_buf; r.dst_buf = in->dst_buf; r.level = in->level; r.cast = in->cast;
+    r.src_off = in->src_off; r.dst_off = in->dst_off;
+    r.src_pitch = in->src_pitch; r.dst_pitch = in->dst_pitch;
+    r.rows = in->rows; r.width_dst = in->width_bytes_dst;
+    r.replicas = in->replicas; r.replica_stride = in->replica_stride;
+    return NEREUS_OK;
+}
+
 int nereus_dag_lower(nereus_dag_t dag, const nereus_model_desc_t* descs, int n_descs, nereus_transition_t* out) {
     NEREUS_GUARD_BEGIN
-    if (!dag || !descs || !out || !dag->planned || n_descs != (int)dag->stages.size()) return NEREUS_ERR_ARG;
+    if (!dag || !descs || !out || !dag->scheduled || n_descs != (int)dag->stages.size()) return NEREUS_ERR_ARG;
     for (int m = 0; m < n_descs; ++m)
         if (!descs[m]) return NEREUS_ERR_ARG;
     const int n_units = (int)dag->units.size();
@@ -718,7 +878,7 @@ const char* nereus_strerror(int code) {
     case NEREUS_OK:              return "ok";
     case NEREUS_ERR_ARG:         return "invalid argument";
     case NEREUS_ERR_INDIVISIBLE: return "plan does not divide the model, or a piece is not a multiple of 16 bytes";
-    case NEREUS_ERR_UNSUPPORTED: return "unsupported dtype pair, tp > kv_heads, or too many buffers";
+    case NEREUS_ERR_UNSUPPORTED: return "unsupported dtype pair, too many buffers or levels, or a call that is not allowed here";
     case NEREUS_ERR_ALIAS:       return "a destination buffer overlaps a source or another destination";
     case NEREUS_ERR_CUDA:        return "a CUDA call failed";
     case NEREUS_ERR_NOMEM:       return "out of host memory";
@@ -726,6 +886,7 @@ const char* nereus_strerror(int code) {
     case NEREUS_ERR_ALIGN:       return "a shard pointer is not 16-byte aligned";
     case NEREUS_ERR_INFEASIBLE:  return "the transition DAG cannot be scheduled: an acquisition stays blocked";
     case NEREUS_ERR_TOO_LARGE:   return "the transition has more tasks than the fixed scratch of run_static holds";
+    case NEREUS_ERR_TABLE:       return "the task table failed validation: a task leaves its buffers or two tasks collide";
     default:                     return "unknown error";
     }
 }

@@ -100,18 +100,36 @@ struct alignas(16) RectDev {
 };
 static_assert(sizeof(RectDev) == 64, "RectDev must stay 64 bytes");
 
-// Control words on the device.
+// One tile, resolved on the host: tables of up to kDirectMaxTiles tiles carry one record per tile, so that a
+// claimer reaches its addresses with one load instead of a search through the tile prefix.  48 bytes.
+struct alignas(16) TileRec {
+    uint64_t src_off, dst_off;   // of the tile, from the start of its source / destination buffers
+    uint32_t src_pitch, dst_pitch;
+    uint32_t rows, width;        // row pieces in the tile, dst bytes per piece
+    uint16_t src_buf, dst_buf;
+    uint16_t replicas, replica_stride;
+    uint16_t level, cast;
+    uint32_t reserved;
+};
+static_assert(sizeof(TileRec) == 48, "TileRec must stay 48 bytes");
+
+// Control words on the device, one block per device copy of a table.  A run leaves cursor, done and exited at
+// zero for the next one (the last block to finish clears them), so a launch needs no reset in front of it and
+// may be replayed from a captured graph.  status is sticky: the first failure since it was last read.
 struct Ctrl {
-    uint32_t cursor;      // next tile to claim
+    uint32_t cursor;      // tiles claimed dynamically so far
     uint32_t done;        // tiles completed (only maintained for multi-level tables)
+    uint32_t exited;      // blocks of the running launch that have finished
     uint32_t status;      // NEREUS_DEV_*
     uint32_t detail;      // tile index that raised the status
+    uint32_t reserved[3];
 };
+static_assert(sizeof(Ctrl) == 32, "Ctrl is one 32-byte sector");
 
 constexpr int kMaxBuffers = 448;      // pointers carried in the kernel's parameter block
 constexpr int kMaxLevels  = 8;
-constexpr int kCtrlSlots  = 64;
 constexpr int kMaxReplicas = 16;
+constexpr uint32_t kDirectMaxTiles = 1u << 17;   // tables up to this many tiles get per-tile records (6 MiB)
 
 struct Tuning {
     int tile_bytes  = 0;
@@ -124,7 +142,8 @@ struct DeviceTable {                  // one per prepare()
     int       device    = -1;
     RectDev*  rects     = nullptr;
     uint32_t* first     = nullptr;    // n_rects + 1 tile prefix
-    Ctrl*     ctrl      = nullptr;    // kCtrlSlots control blocks, used round robin: one memset per cycle
+    TileRec*  tiles     = nullptr;    // n_tiles records, or null for tables beyond kDirectMaxTiles
+    Ctrl*     ctrl      = nullptr;    // the control block
     uint32_t  runs      = 0;          // runs launched on this device copy
     uint32_t  n_tiles   = 0;
     uint32_t  level_end[kMaxLevels] = {0};   // tiles up to and including each level
@@ -180,7 +199,8 @@ struct nereus_dag_s {
     std::vector<nereus::StageRec> stages;
     std::vector<nereus::UnitRec>  units;
     std::vector<nereus::PrimRec>  prims;
-    bool                          planned = false;
+    bool                          planned = false;     // nereus_dag_plan has run: no more stages or units
+    bool                          scheduled = false;   // ... and every primitive got its place in the schedule
 };
 
 namespace nereus {
@@ -193,6 +213,16 @@ uint64_t tile_table(const nereus_transition_s& t, uint32_t tile_bytes, std::vect
 // Same into caller-provided arrays (rects.size() entries and rects.size() + 1 entries): no allocation.
 uint64_t tile_table_raw(const nereus_transition_s& t, uint32_t tile_bytes, RectDev* out, uint32_t* first,
                         uint32_t level_end[kMaxLevels]);
+
+// One record per tile from a tiled table (out has room for the table's tile count).
+void expand_tiles(const RectDev* rects, size_t n_rects, TileRec* out);
+
+// Host-side check of a table before it reaches the device: every task inside its buffers, the 16-byte rule,
+// pitches that keep row pieces apart, buffer indices and levels in range, a chained task reading only what an
+// earlier level wrote, destinations of one level pairwise disjoint, and (when `tiled` is given) a tiling that
+// covers each task exactly.  `order` is scratch for rects.size() indices.  Allocates nothing.
+int validate_table(const nereus_transition_s& t, const RectDev* tiled, const uint32_t* first, uint64_t n_tiles,
+                   uint32_t* order);
 
 void set_cuda_error(int e);
 

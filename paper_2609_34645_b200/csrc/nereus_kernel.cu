@@ -4,12 +4,18 @@
 // round-to-nearest-even cast.  Pure data movement: the bound is HBM bandwidth, there is no tensor-core work.
 //
 // Execution model
-//   * grid = SMs x ctas_per_sm persistent blocks; every WARP claims tiles on its own: lane 0 takes the next
-//     tile index from a global cursor with one atomicAdd and broadcasts it by shuffle; the claim of the next
-//     tile is issued before the current tile is copied, so its latency hides behind the copy.
-//   * a tile index is resolved to its rect by binary search in the tile-prefix array, then to a row block /
-//     column block of that rect by arithmetic; every lane moves 16-byte vectors, 32 lanes x 16 B = 512 B
-//     contiguous per instruction, kUnroll independent loads in flight per lane before the first store.
+//   * grid = SMs x ctas_per_sm persistent blocks; every WARP claims tiles on its own.  Its first tile is its
+//     own index in the grid (no atomic on the way to the first load); further tiles come from a global cursor:
+//     lane 0 takes the next index with one atomicAdd and broadcasts it by shuffle, and the claim of the next
+//     tile is issued before the current tile is copied, so its latency hides behind the copy.  Chained tables
+//     claim every tile from the cursor: tiles are then handed out in level order to warps that already run,
+//     which is what keeps the level gates free of deadlock whatever else shares the GPU.
+//   * a tile index is resolved by one load of its 48-byte record when the table carries per-tile records
+//     (tables of up to 2^17 tiles), else to its rect by binary search in the tile-prefix array and then to a
+//     row block / column block of that rect by arithmetic; every lane moves 16-byte vectors, 32 lanes x 16 B =
+//     512 B contiguous per instruction, kUnroll independent loads in flight per lane before the first store.
+//   * the last block to finish zeroes the cursor and the counters, so a launch needs no reset in front of
+//     it and can be replayed from a captured graph.
 //   * tables with several dependency levels (chained transitions): a tile of level k waits, with a poll
 //     limit, until every tile of level k-1 has completed; on giving up it records NEREUS_DEV_TIMEOUT and the
 //     warp leaves.  A warp publishes its completed tiles once per level (one fence, one atomic), not per
@@ -25,6 +31,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -46,6 +53,7 @@ void set_cuda_error(int e) { g_last_cuda_error = e; }
 struct WalkParams {
     const RectDev*  rects;
     const uint32_t* first;        // n_rects + 1
+    const TileRec*  tiles;        // n_tiles records, or null
     Ctrl*           ctrl;
     uint32_t        n_rects, n_tiles, n_levels;
     uint32_t        level_end[kMaxLevels];
@@ -58,16 +66,11 @@ constexpr int      kUnrollRect  = 6;            // ... pitched rects (their inde
 constexpr int      kUnrollCast  = 8;            // ... the cast
 constexpr uint32_t kPrefixCache = 2047;         // rects whose tile prefix the vector kernel keeps in shared memory
 constexpr uint32_t kGatePolls   = 1u << 21;     // x ~200 ns sleep: gives up after roughly half a second
+constexpr uint64_t kWaitNanos   = 500ull * 1000 * 1000;   // deadline of an mbarrier wait, on %globaltimer
 
 // ---------------------------------------------------------------------------------------------------
 // device helpers
 // ---------------------------------------------------------------------------------------------------
-
-__device__ __forceinline__ uint32_t claim_tile(Ctrl* ctrl, unsigned lane) {
-    uint32_t g = 0;
-    if (lane == 0) g = atomicAdd(&ctrl->cursor, 1u);
-    return __shfl_sync(0xffffffffu, g, 0);
-}
 
 __device__ __forceinline__ uint32_t claim_tiles(Ctrl* ctrl, unsigned lane, uint32_t n) {
     uint32_t g = 0;
@@ -290,12 +293,47 @@ __device__ __forceinline__ bool resolve_tile(const WalkParams& p, uint32_t g, Re
     return true;
 }
 
+// Tile g of a table that carries per-tile records: one 48-byte load, no search.
+__device__ __forceinline__ bool resolve_direct(const WalkParams& p, uint32_t g, Tile& t) {
+    const uint4* q = reinterpret_cast<const uint4*>(p.tiles + g);
+    const uint4 a = __ldg(q), b = __ldg(q + 1), c = __ldg(q + 2);
+    const uint64_t src_off = ((uint64_t)a.y << 32) | a.x;
+    t.d_off = ((uint64_t)a.w << 32) | a.z;
+    t.sp = b.x; t.dp = b.y; t.nr = b.z; t.w = b.w;
+    const uint32_t src_buf = c.x & 0xFFFFu;
+    t.dst_buf = c.x >> 16;
+    t.reps = c.y & 0xFFFFu; t.rstride = c.y >> 16;
+    t.level = c.z & 0xFFFFu; t.cast = c.z >> 16;
+    if (src_buf >= (uint32_t)kMaxBuffers || t.reps == 0 || t.nr == 0 ||
+        t.dst_buf + (t.reps - 1) * t.rstride >= (uint32_t)kMaxBuffers)
+        return false;
+    t.s = p.bufs[src_buf] + src_off;
+    return true;
+}
+
 __device__ __forceinline__ void raise_status(Ctrl* ctrl, uint32_t status, uint32_t detail) {
     if (atomicCAS(&ctrl->status, (uint32_t)NEREUS_DEV_OK, status) == (uint32_t)NEREUS_DEV_OK) ctrl->detail = detail;
 }
 
+// End of a block's work: the last block of the launch to get here leaves the control words as a fresh launch
+// expects them.  Every claim and every publication of the block happened before its arrival (the barrier
+// orders the block's threads, the fence orders the block against the others), so nothing touches the words
+// after they are cleared.  The status word is not cleared: it is the host's to read.
+__device__ __forceinline__ void finish_block(Ctrl* ctrl) {
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        if (atomicAdd(&ctrl->exited, 1u) == gridDim.x - 1) {
+            __threadfence();
+            ctrl->cursor = 0;
+            ctrl->done = 0;
+            ctrl->exited = 0;
+        }
+    }
+}
+
 // ---------------------------------------------------------------------------------------------------
-// the persistent walker, register-staged vector copy (every table)
+// the persistent walker, register-staged vector copy
 // ---------------------------------------------------------------------------------------------------
 
 __global__ void __launch_bounds__(512, 2) nereus_walk_vec(const __grid_constant__ WalkParams p) {
@@ -305,23 +343,31 @@ __global__ void __launch_bounds__(512, 2) nereus_walk_vec(const __grid_constant_
     uint32_t       open_level = 0;                             // highest level whose gate this warp has passed
     RectRange      rr;
 
-    // small tables: the tile prefix is copied to shared memory once per CTA, so that resolving a tile costs
-    // one trip to memory (the rect record) instead of a chain of dependent ones
+    // tables without per-tile records: the tile prefix is copied to shared memory once per CTA (when it fits),
+    // so that resolving a tile costs one trip to memory (the rect record) instead of a chain of dependent ones
     __shared__ uint32_t s_first[kPrefixCache + 1];
-    const bool cached = p.n_rects <= kPrefixCache;
-    if (cached)
+    const bool direct = p.tiles != nullptr;
+    const bool cached = !direct && p.n_rects <= kPrefixCache;
+    if (cached) {
         for (uint32_t i = threadIdx.x; i <= p.n_rects; i += blockDim.x) s_first[i] = __ldg(p.first + i);
-    __syncthreads();
+        __syncthreads();
+    }
     const uint32_t* const sf = s_first;
     auto first_at = [&p, cached, sf](uint32_t i) { return cached ? sf[i] : __ldg(p.first + i); };
 
-    uint32_t g = claim_tile(ctrl, lane);
+    // single-level tables: the first tile of a warp is its own index, the cursor hands out the tiles beyond
+    // the grid; chained tables take every tile from the cursor (see the head of this file)
+    const uint32_t n_warps = gridDim.x * (blockDim.x >> 5);
+    const uint32_t base    = p.n_levels == 1 ? n_warps : 0u;
+    const bool     more    = p.n_tiles > base;                 // false: nobody ever touches the cursor
+    uint32_t g = p.n_levels == 1 ? blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)
+                                 : claim_tiles(ctrl, lane, 1);
     while (g < p.n_tiles) {
-        const uint32_t next_issued = claim_issue(ctrl, lane, 1);   // in flight while this tile is copied
+        const uint32_t next_issued = more ? claim_issue(ctrl, lane, 1) : 0u;   // in flight while this tile is copied
         Tile t;
-        if (!resolve_tile<false>(p, g, rr, t, first_at)) {
+        if (!(direct ? resolve_direct(p, g, t) : resolve_tile<false>(p, g, rr, t, first_at))) {
             if (lane == 0) raise_status(ctrl, NEREUS_DEV_BOUNDS, g);
-            return;
+            break;
         }
 
         if (t.level != my_level) {
@@ -347,7 +393,7 @@ __global__ void __launch_bounds__(512, 2) nereus_walk_vec(const __grid_constant_
                 if (!ok) raise_status(ctrl, NEREUS_DEV_TIMEOUT, g);
             }
             ok = __shfl_sync(0xffffffffu, ok, 0);
-            if (!ok) return;
+            if (!ok) break;
             __threadfence();
             open_level = t.level;
         }
@@ -363,13 +409,14 @@ __global__ void __launch_bounds__(512, 2) nereus_walk_vec(const __grid_constant_
             copy_rect<kUnrollRect>(t.s, D, t.reps, t.nr, t.w >> 4, t.sp, t.dp, lane);
         }
         if (p.n_levels > 1) ++my_done;
-        g = claim_take(next_issued);
+        g = more ? base + claim_take(next_issued) : p.n_tiles;
     }
     if (my_done) {
         __threadfence();
         __syncwarp();
         if (lane == 0) atomicAdd(&ctrl->done, my_done);
     }
+    finish_block(ctrl);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -403,14 +450,28 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-// Bounded wait for the phase with the given parity; false when it gave up.
+__device__ __forceinline__ uint64_t global_nanos() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait for the phase with the given parity; false when it gave up.  Two limits: a deadline of
+// kWaitNanos (half a second) on the global timer, read every 64 attempts once the first few have failed, and
+// a cap on the attempts as a backstop should the timer not advance (a try_wait suspends the thread for a time
+// the hardware chooses, so the cap alone has no number).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    uint64_t deadline = 0;
     for (uint32_t i = 0; i < kBarrierTries; ++i) {
         uint32_t ok;
         asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
                      "selp.u32 %0, 1, 0, p;\n\t}"
                      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
         if (ok) return true;
+        if ((i & 63u) == 63u) {
+            const uint64_t now = global_nanos();
+            if (deadline == 0) deadline = now + kWaitNanos;
+            else if (now > deadline) return false;
+        }
     }
     return false;
 }
@@ -456,7 +517,10 @@ __device__ __forceinline__ void ring_producer(const WalkParams& p, const Ring& R
     Ctrl* const ctrl = p.ctrl;
     uint32_t    stage = 0, phase = 0, level = 0;
     RectRange   rr;
-    uint32_t    g0 = claim_tiles(ctrl, lane, R.claim);
+    // single-level tables: the first batch is the block's own index, the cursor hands out the batches beyond
+    // the grid; chained tables take every batch from the cursor
+    const uint32_t base = p.n_levels == 1 ? gridDim.x * R.claim : 0u;
+    uint32_t    g0 = p.n_levels == 1 ? blockIdx.x * R.claim : claim_tiles(ctrl, lane, R.claim);
     bool        running = true;
     while (running) {
         const bool     last    = g0 >= p.n_tiles;
@@ -467,7 +531,8 @@ __device__ __forceinline__ void ring_producer(const WalkParams& p, const Ring& R
             bool ok = true;
             if (!end) {
                 // the converting ring (kCast) takes both kinds of tile, the bit-copy ring only its own
-                ok = resolve_tile<true>(p, g, rr, t, [&p](uint32_t i) { return __ldg(p.first + i); }) &&
+                ok = (p.tiles ? resolve_direct(p, g, t)
+                              : resolve_tile<true>(p, g, rr, t, [&p](uint32_t i) { return __ldg(p.first + i); })) &&
                      (kCast || t.cast == 0) &&
                      (((uint64_t)t.nr * t.w) << t.cast) <= R.stage_bytes;
                 if (!ok && lane == 0) raise_status(ctrl, NEREUS_DEV_BOUNDS, g);
@@ -540,7 +605,7 @@ __device__ __forceinline__ void ring_producer(const WalkParams& p, const Ring& R
                 if (++stage == R.n_stages) { stage = 0; phase ^= 1; }
             }
         }
-        g0 = last ? g0 : claim_take(next_issued);
+        g0 = last ? g0 : base + claim_take(next_issued);
     }
 }
 
@@ -701,6 +766,7 @@ nereus_walk_ring(const __grid_constant__ WalkParams p, const uint32_t stage_byte
     if (warp == 0) ring_producer<kCast>(p, R, lane);
     else if (kCast) ring_consumer_cast(p, R, threadIdx.x - 32);
     else ring_consumer_copy(p, R, lane);
+    finish_block(p.ctrl);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -735,36 +801,31 @@ struct Launch {
     size_t   smem = 0;
 };
 
-// The ring takes every table: all bit copy on the bulk-store consumer, anything with a cast in it on the
-// converting consumers (which copy the bit-copy tiles of a mixed table from shared memory as well).
-static bool ring_eligible(const nereus_transition_s& t, bool& cast) {
-    cast = false;
-    for (const Rect& r : t.rects) cast = cast || r.cast;
-    return true;
-}
-
+// Both kernels take every table.  The ring runs an all-bit-copy table on the bulk-store consumer and
+// anything with a cast in it on the converting consumers (which copy the bit-copy tiles of a mixed table from
+// shared memory as well).  Default: the ring for tables that write 64 MiB or more (its per-block start-up
+// costs more than it gains below that), the vector kernel for smaller ones.
 static int resolve_launch(const nereus_transition_s& t, int sms, Launch& L) {
     const int want = t.tuning.variant ? t.tuning.variant : env_int("NEREUS_VARIANT", 0);
     const int asked_tile = t.tuning.tile_bytes ? t.tuning.tile_bytes : env_int("NEREUS_TILE_BYTES", 0);
-    // default: the ring for large single-level bit-copy tables (its per-CTA start-up costs more than it gains
-    // below a few tens of MB), the vector kernel for everything else
-    const bool ring_ok = ring_eligible(t, L.cast);
-    if (want == 2)      L.variant = ring_ok ? 2 : 1;
-    else if (want == 1) L.variant = 1;
-    else                L.variant = (ring_ok && t.bytes_written >= (64ull << 20) &&
-                                     asked_tile <= (L.cast ? 24576 : 49152)) ? 2 : 1;
+    L.cast = false;
+    for (const Rect& r : t.rects) L.cast = L.cast || r.cast;
+    if (want)  L.variant = want;
+    else       L.variant = (t.bytes_written >= (64ull << 20) && asked_tile <= (L.cast ? 24576 : 49152)) ? 2 : 1;
     L.ctas_per_sm = t.tuning.ctas_per_sm ? t.tuning.ctas_per_sm : env_int("NEREUS_CTAS_PER_SM", 2);
     L.threads     = t.tuning.threads     ? t.tuning.threads     : env_int("NEREUS_THREADS", 384);
-    L.tile_bytes  = t.tuning.tile_bytes  ? t.tuning.tile_bytes  : env_int("NEREUS_TILE_BYTES", 0);
+    L.tile_bytes  = asked_tile;
     if (L.variant == 2) { L.ctas_per_sm = t.tuning.ctas_per_sm ? t.tuning.ctas_per_sm : 1; L.threads = 64; }
     if (L.ctas_per_sm < 1 || L.ctas_per_sm > 2 || L.threads < 32 || L.threads > 512 || L.threads % 32)
         return NEREUS_ERR_ARG;
     if (L.tile_bytes == 0) {
         // default: 16 KiB per warp tile (32 KiB per ring stage); smaller tiles for small tables, until at least
-        // every other claimer gets a tile
+        // every other claimer gets a tile; a tile stays a multiple of 512 bytes
         L.tile_bytes = L.variant == 2 ? (L.cast ? 24576 : 32768) : 16384;
         const uint64_t claimers = (uint64_t)sms * L.ctas_per_sm * (L.variant == 2 ? 8 : L.threads / 32);
-        while (L.tile_bytes > 1024 && t.bytes_written / L.tile_bytes < claimers / 2) L.tile_bytes /= 2;
+        while (L.tile_bytes / 2 >= 1024 && (L.tile_bytes / 2) % 512 == 0 &&
+               t.bytes_written / L.tile_bytes < claimers / 2)
+            L.tile_bytes /= 2;
     }
     if (L.tile_bytes < 512 || L.tile_bytes % 512) return NEREUS_ERR_ARG;
     if (L.variant == 2) {
@@ -828,17 +889,34 @@ static int prepare(nereus_transition_s& t) {
     if (n_tiles == 0 && !t.rects.empty()) return NEREUS_ERR_UNSUPPORTED;
     dv.n_tiles = (uint32_t)n_tiles;
 
-    // one allocation: [rects | first | ctrl]
+    // nothing reaches the device that the host has not checked against the declared buffer sizes
+    if (t.rects.size() >= (1u << 24)) return NEREUS_ERR_UNSUPPORTED;
+    size_t entries = 0;
+    for (const Rect& r : t.rects) entries += (size_t)std::max(1, std::min(r.replicas, kMaxReplicas));
+    std::vector<uint32_t> order(entries + 1);
+    if (int rc = validate_table(t, rects.data(), first.data(), n_tiles, order.data())) return rc;
+
+    std::vector<TileRec> tiles;
+    if (n_tiles <= kDirectMaxTiles) {
+        tiles.resize(n_tiles);
+        expand_tiles(rects.data(), rects.size(), tiles.data());
+    }
+
+    // one allocation: [rects | first | tiles | ctrl]
     const size_t rects_b = round_up(rects.size() * sizeof(RectDev), 256);
     const size_t first_b = round_up(first.size() * sizeof(uint32_t), 256);
+    const size_t tiles_b = round_up(tiles.size() * sizeof(TileRec), 256);
+    const size_t ctrl_b  = round_up(sizeof(Ctrl), 256);
     char* base = nullptr;
-    const size_t ctrl_b = round_up(sizeof(Ctrl) * kCtrlSlots, 256);
-    NEREUS_CUDA(cudaMalloc(&base, rects_b + first_b + ctrl_b));
+    NEREUS_CUDA(cudaMalloc(&base, rects_b + first_b + tiles_b + ctrl_b));
     dv.rects = reinterpret_cast<RectDev*>(base);
     dv.first = reinterpret_cast<uint32_t*>(base + rects_b);
-    dv.ctrl  = reinterpret_cast<Ctrl*>(base + rects_b + first_b);
+    dv.tiles = tiles.empty() ? nullptr : reinterpret_cast<TileRec*>(base + rects_b + first_b);
+    dv.ctrl  = reinterpret_cast<Ctrl*>(base + rects_b + first_b + tiles_b);
     cudaError_t e = cudaMemcpy(dv.rects, rects.data(), rects.size() * sizeof(RectDev), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(dv.first, first.data(), first.size() * sizeof(uint32_t), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess && !tiles.empty())
+        e = cudaMemcpy(dv.tiles, tiles.data(), tiles.size() * sizeof(TileRec), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemset(dv.ctrl, 0, ctrl_b);
     if (e != cudaSuccess) { cudaFree(base); set_cuda_error((int)e); (void)cudaGetLastError(); return NEREUS_ERR_CUDA; }
     t.dev = dv;
@@ -886,6 +964,16 @@ static int check_buffers(const nereus_transition_s& t, const void* const* src, v
             if (t.dst_read_level[a] < 0 || t.dst_level[b] <= t.dst_read_level[a]) return NEREUS_ERR_ALIAS;
         }
     }
+    return NEREUS_OK;
+}
+
+// The status word is sticky on the device (first failure wins); reading it hands it to the host and clears it.
+static int read_and_clear_status(Ctrl* ctrl, int* device_status) {
+    Ctrl c;
+    NEREUS_CUDA(cudaMemcpy(&c, ctrl, sizeof(Ctrl), cudaMemcpyDeviceToHost));
+    if (c.status != (uint32_t)NEREUS_DEV_OK)
+        NEREUS_CUDA(cudaMemset(&ctrl->status, 0, 2 * sizeof(uint32_t)));      // status and detail
+    *device_status = (int)c.status;
     return NEREUS_OK;
 }
 
@@ -950,11 +1038,8 @@ int nereus_transition_run(nereus_transition_t t, const void* const* src_ptrs, vo
         if (int rc = resolve_launch(*t, dv.sm_count, L)) return rc;
         L.tile_bytes = dv.tile_bytes;
         WalkParams p;
-        // control words: a fresh (zeroed) block per run; the blocks are zeroed together once per cycle
-        const uint32_t slot = t->dev.runs % kCtrlSlots;
-        if (slot == 0 && t->dev.runs != 0)
-            NEREUS_CUDA(cudaMemsetAsync(dv.ctrl, 0, sizeof(Ctrl) * kCtrlSlots, stream));
-        p.rects = dv.rects; p.first = dv.first; p.ctrl = dv.ctrl + slot;
+        // the control words need no reset: every launch leaves them zeroed for the next one
+        p.rects = dv.rects; p.first = dv.first; p.tiles = dv.tiles; p.ctrl = dv.ctrl;
         p.n_tiles = dv.n_tiles;
         // NEREUS_DEBUG_GATE_BIAS (tests only): raises what a dependency gate waits for, so that it can never
         // open and the bounded wait must give up with NEREUS_DEV_TIMEOUT
@@ -972,11 +1057,8 @@ int nereus_transition_run(nereus_transition_t t, const void* const* src_ptrs, vo
 int nereus_transition_status(nereus_transition_t t, int* device_status) {
     if (!t || !device_status) return NEREUS_ERR_ARG;
     if (!t->dev.rects) { *device_status = NEREUS_DEV_OK; return NEREUS_OK; }
-    Ctrl c;
     if (t->dev.runs == 0) { *device_status = NEREUS_DEV_OK; return NEREUS_OK; }
-    NEREUS_CUDA(cudaMemcpy(&c, t->dev.ctrl + (t->dev.runs - 1) % kCtrlSlots, sizeof(Ctrl), cudaMemcpyDeviceToHost));
-    *device_status = (int)c.status;
-    return NEREUS_OK;
+    return read_and_clear_status(t->dev.ctrl, device_status);
 }
 
 int nereus_transition_launches(nereus_transition_t t, uint64_t* n) {
@@ -1009,7 +1091,8 @@ int nereus_last_cuda_error(void) { return g_last_cuda_error; }
 
 namespace nereus {
 
-constexpr int    kStaticMaxRects    = 4096;
+constexpr int    kStaticMaxRects    = NEREUS_STATIC_MAX_RECTS;
+constexpr int    kStaticMaxEntries  = 4 * kStaticMaxRects;            // (task, replica) pairs the check can sort
 constexpr size_t kStaticRectBytes   = (size_t)kStaticMaxRects * sizeof(RectDev);              // 256 KiB
 constexpr size_t kStaticFirstBytes  = ((size_t)kStaticMaxRects + 1 + 63) / 64 * 64 * sizeof(uint32_t);
 constexpr size_t kStaticScratchBytes = kStaticRectBytes + kStaticFirstBytes + 256;            // ~272 KiB
@@ -1019,6 +1102,14 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBy
 constexpr int kStaticMaxDevices = 64;
 static unsigned char* g_static_ptr[kStaticMaxDevices];   // device address of the array, per device
 static int            g_static_sms[kStaticMaxDevices];
+
+// Host staging of the tiled table: plain file-scope arrays (part of the library's image, so no thread's first
+// call allocates anything), shared by all threads under a lock that is held until the runtime has taken the
+// bytes.
+static std::mutex g_static_lock;
+static RectDev    g_static_rects[kStaticMaxRects];
+static uint32_t   g_static_first[kStaticMaxRects + 1];
+static uint32_t   g_static_order[kStaticMaxEntries + 1];
 
 // Once per device, with that device current: the array's name is only a host-side handle of the symbol;
 // the address a kernel can use comes from cudaGetSymbolAddress.
@@ -1037,47 +1128,69 @@ static int static_scratch(int device, unsigned char** ptr, int* sms) {
     return NEREUS_OK;
 }
 
+static Ctrl* static_ctrl(unsigned char* scratch) {
+    return reinterpret_cast<Ctrl*>(scratch + kStaticRectBytes + kStaticFirstBytes);
+}
+
 }  // namespace nereus
 
 extern "C" int nereus_transition_run_static(nereus_transition_t t, const void* const* src_ptrs,
                                             void* const* dst_ptrs, void* cuda_stream) {
-    try {
-        if (!t || !src_ptrs || !dst_ptrs) return NEREUS_ERR_ARG;
-        if (t->rects.size() > (size_t)kStaticMaxRects) return NEREUS_ERR_TOO_LARGE;
-        if (int rc = check_buffers(*t, src_ptrs, dst_ptrs)) return rc;
-        int device = 0;
-        NEREUS_CUDA(cudaGetDevice(&device));
-        unsigned char* scratch = nullptr;
-        int sms = 0;
-        if (int rc = static_scratch(device, &scratch, &sms)) return rc;
-        cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    if (!t || !src_ptrs || !dst_ptrs) return NEREUS_ERR_ARG;
+    const size_t n_rects = t->rects.size();
+    if (n_rects > (size_t)kStaticMaxRects) return NEREUS_ERR_TOO_LARGE;
+    size_t entries = 0;
+    for (const Rect& r : t->rects) entries += (size_t)std::max(1, std::min(r.replicas, kMaxReplicas));
+    if (entries > (size_t)kStaticMaxEntries) return NEREUS_ERR_TOO_LARGE;
+    if (int rc = check_buffers(*t, src_ptrs, dst_ptrs)) return rc;
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    // the table is uploaded from host arrays that the next call overwrites: a captured copy of them would
+    // replay whatever table came last, so the call is refused while the stream is being captured
+    cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+    NEREUS_CUDA(cudaStreamIsCapturing(stream, &capturing));
+    if (capturing != cudaStreamCaptureStatusNone) return NEREUS_ERR_UNSUPPORTED;
 
-        Launch L;
-        if (int rc = resolve_launch(*t, sms, L)) return rc;
+    std::lock_guard<std::mutex> hold(g_static_lock);
+    int device = 0;
+    NEREUS_CUDA(cudaGetDevice(&device));
+    unsigned char* scratch = nullptr;
+    int sms = 0;
+    if (int rc = static_scratch(device, &scratch, &sms)) return rc;
 
-        WalkParams p;
-        // the tiled table is built in fixed host arrays of the calling thread: no heap allocation either
-        static thread_local RectDev  rects[kStaticMaxRects];
-        static thread_local uint32_t first[kStaticMaxRects + 1];
-        const size_t   n_rects = t->rects.size();
-        const uint64_t n_tiles = tile_table_raw(*t, (uint32_t)L.tile_bytes, rects, first, p.level_end);
-        if (n_tiles == 0 && n_rects != 0) return NEREUS_ERR_UNSUPPORTED;
+    Launch L;
+    if (int rc = resolve_launch(*t, sms, L)) return rc;
 
-        RectDev*  d_rects = reinterpret_cast<RectDev*>(scratch);
-        uint32_t* d_first = reinterpret_cast<uint32_t*>(scratch + kStaticRectBytes);
-        Ctrl*     d_ctrl  = reinterpret_cast<Ctrl*>(scratch + kStaticRectBytes + kStaticFirstBytes);
-        // the array keeps whatever the previous call left: overwrite the table, zero the control words
-        // pageable host memory: the runtime has staged the bytes by the time each call returns, so the arrays may
-        // be reused by the next call
-        NEREUS_CUDA(cudaMemcpyAsync(d_rects, rects, n_rects * sizeof(RectDev), cudaMemcpyHostToDevice, stream));
-        NEREUS_CUDA(cudaMemcpyAsync(d_first, first, (n_rects + 1) * sizeof(uint32_t), cudaMemcpyHostToDevice, stream));
-        NEREUS_CUDA(cudaMemsetAsync(d_ctrl, 0, sizeof(Ctrl), stream));
+    WalkParams p;
+    const uint64_t n_tiles = tile_table_raw(*t, (uint32_t)L.tile_bytes, g_static_rects, g_static_first, p.level_end);
+    if (n_tiles == 0 && n_rects != 0) return NEREUS_ERR_UNSUPPORTED;
+    if (int rc = validate_table(*t, g_static_rects, g_static_first, n_tiles, g_static_order)) return rc;
 
-        p.rects = d_rects; p.first = d_first; p.ctrl = d_ctrl;
-        p.n_tiles = (uint32_t)n_tiles;
-        fill_params(*t, src_ptrs, dst_ptrs, p);
-        if (int rc = launch_walk(L, sms, p, stream)) return rc;
-        if (n_tiles > 0) t->launches += 1;
-        return NEREUS_OK;
-    } catch (const std::bad_alloc&) { return NEREUS_ERR_NOMEM; }
+    RectDev*  d_rects = reinterpret_cast<RectDev*>(scratch);
+    uint32_t* d_first = reinterpret_cast<uint32_t*>(scratch + kStaticRectBytes);
+    Ctrl*     d_ctrl  = static_ctrl(scratch);
+    // The array keeps whatever the previous call left: overwrite the table and zero the cursor and the two
+    // counters (a launch leaves them zeroed, but nothing here relies on how the last one ended).  The status
+    // word stays: it is sticky until nereus_static_status reads it.  The copies come from pageable memory:
+    // the runtime has taken the bytes by the time each call returns, so the lock may then be released.
+    NEREUS_CUDA(cudaMemcpyAsync(d_rects, g_static_rects, n_rects * sizeof(RectDev), cudaMemcpyHostToDevice, stream));
+    NEREUS_CUDA(cudaMemcpyAsync(d_first, g_static_first, (n_rects + 1) * sizeof(uint32_t), cudaMemcpyHostToDevice, stream));
+    NEREUS_CUDA(cudaMemsetAsync(d_ctrl, 0, 3 * sizeof(uint32_t), stream));
+
+    p.rects = d_rects; p.first = d_first; p.tiles = nullptr; p.ctrl = d_ctrl;
+    p.n_tiles = (uint32_t)n_tiles;
+    const uint32_t gate_bias = (uint32_t)env_int("NEREUS_DEBUG_GATE_BIAS", 0);     // tests of the failure path only
+    for (int k = 0; k < kMaxLevels; ++k) p.level_end[k] += gate_bias;
+    fill_params(*t, src_ptrs, dst_ptrs, p);
+    if (int rc = launch_walk(L, sms, p, stream)) return rc;
+    if (n_tiles > 0) t->launches += 1;
+    return NEREUS_OK;
+}
+
+extern "C" int nereus_static_status(int* device_status) {
+    if (!device_status) return NEREUS_ERR_ARG;
+    int device = 0;
+    NEREUS_CUDA(cudaGetDevice(&device));
+    if (device < 0 || device >= kStaticMaxDevices) return NEREUS_ERR_UNSUPPORTED;
+    if (!g_static_ptr[device]) { *device_status = NEREUS_DEV_OK; return NEREUS_OK; }   // no static run here yet
+    return read_and_clear_status(static_ctrl(g_static_ptr[device]), device_status);
 }

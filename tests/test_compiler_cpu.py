@@ -163,6 +163,7 @@ def check_transition(sh, a, b, sdt="bf16", ddt="bf16", vh=False, seed=0, la=0, l
     src = random_src(m, oa, seed, sdt)
     want = O.reshard(m, oa, ob, src, fill=0xA5)
     t = d.compile(B.Plan(a[0], a[1], 0, la), B.Plan(b[0], b[1], B.DTYPES[ddt], lb))
+    assert t.validate() == B.OK                      # what the compiler emits passes the host-side table check
     n_src, n_dst = t.num_buffers()
     assert (n_src, n_dst) == (len(src), len(want))
     for i, s in enumerate(src):
@@ -329,6 +330,7 @@ def test_fuse_independent_and_chained():
 
     # chained round trip: level 0 writes `mid`, level 1 reads it and writes `back`
     ch = B.Transition.fuse([t_ab, t_ba], chained=True)
+    assert ch.validate() == B.OK
     assert ch.num_buffers() == (2, 4)
     assert ch.num_tiles()[1] == 2
     rects = ch.rects()
@@ -345,6 +347,7 @@ def test_fuse_independent_and_chained():
 
     # independent: two model-stages side by side
     ind = B.Transition.fuse([t_ab, t_ba], chained=False)
+    assert ind.validate() == B.OK
     assert ind.num_buffers() == (4, 4)
     src2 = random_src(m, O.Plan(*b), 6, "bf16")
     out = [np.full(ind.buffer_bytes(True, j), 0xA5, np.uint8) for j in range(4)]

@@ -221,7 +221,7 @@ def test_8b_trainer_layout_to_generation_layout_full_size():
 def test_lowered_dag_runs_in_one_launch(variant):
     """The paper's (TP4, PP8) -> (TP8, PP2) example planned as Split / Destroy / Merge, lowered to one table with
     two dependency levels and run in one launch: replicas and target against the oracle."""
-    from oracle import dag as D
+    from oracle import dag_rules as D
     from test_dag_cpu import U, lowered
     sh = I.MICRO
     dag, t, descs = lowered([D.StageChange(D.INFERENCE, [U(4, 8, 0)], [U(8, 2, 0)])], [sh])

@@ -845,16 +845,29 @@ static int resolve_launch(const nereus_transition_s& t, int sms, Launch& L) {
     return NEREUS_OK;
 }
 
+// The ring kernels use more dynamic shared memory than a kernel gets by default: opt in once per device (the
+// launch itself then makes no other runtime call, which keeps it legal inside a stream capture).
+constexpr int kMaxDevices = 64;
+static bool g_ring_ready[kMaxDevices];
+
+static int ring_opt_in(int device) {
+    if (device < 0 || device >= kMaxDevices) return NEREUS_ERR_UNSUPPORTED;
+    if (g_ring_ready[device]) return NEREUS_OK;
+    const int most = 227 * 1024;
+    NEREUS_CUDA(cudaFuncSetAttribute(nereus_walk_ring<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most));
+    NEREUS_CUDA(cudaFuncSetAttribute(nereus_walk_ring<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most));
+    g_ring_ready[device] = true;
+    return NEREUS_OK;
+}
+
 static int launch_walk(const Launch& L, int sms, const WalkParams& p, cudaStream_t stream) {
     if (p.n_tiles == 0) return NEREUS_OK;
     if (L.variant == 2) {
         const unsigned grid = std::max(1u, std::min((unsigned)(sms * L.ctas_per_sm), p.n_tiles));
         if (L.cast) {
-            NEREUS_CUDA(cudaFuncSetAttribute(nereus_walk_ring<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.smem));
             nereus_walk_ring<true><<<grid, 32 + kCastConsumers, L.smem, stream>>>(p, (uint32_t)L.tile_bytes * 2, L.n_stages,
                                                                                   L.piece, L.lag, L.claim);
         } else {
-            NEREUS_CUDA(cudaFuncSetAttribute(nereus_walk_ring<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.smem));
             nereus_walk_ring<false><<<grid, 64, L.smem, stream>>>(p, (uint32_t)L.tile_bytes, L.n_stages, L.piece, L.lag, L.claim);
         }
     } else {
@@ -877,6 +890,7 @@ static int prepare(nereus_transition_s& t) {
     NEREUS_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
     Launch L;
     if (int rc = resolve_launch(t, sms, L)) return rc;
+    if (int rc = ring_opt_in(device)) return rc;
 
     DeviceTable dv;
     dv.device = device;
@@ -1099,7 +1113,7 @@ constexpr size_t kStaticScratchBytes = kStaticRectBytes + kStaticFirstBytes + 25
 
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
-constexpr int kStaticMaxDevices = 64;
+constexpr int kStaticMaxDevices = kMaxDevices;
 static unsigned char* g_static_ptr[kStaticMaxDevices];   // device address of the array, per device
 static int            g_static_sms[kStaticMaxDevices];
 
@@ -1118,6 +1132,7 @@ static int static_scratch(int device, unsigned char** ptr, int* sms) {
     if (!g_static_ptr[device]) {
         unsigned char* p = nullptr;
         NEREUS_CUDA(cudaGetSymbolAddress((void**)&p, g_static_scratch));
+        if (int rc = ring_opt_in(device)) return rc;
         int n = 0;
         NEREUS_CUDA(cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, device));
         g_static_sms[device] = n;

@@ -284,7 +284,7 @@ class Transition:
         v, tb, g, th = _i(), _i(), _i(), _i()
         _ck(_lib.nereus_transition_launch_info(self._h, ctypes.byref(v), ctypes.byref(tb), ctypes.byref(g),
                                                ctypes.byref(th)), "nereus_transition_launch_info")
-        return {"kernel": {1: "nereus_walk_vec", 2: "nereus_walk_ring"}[v.value], "tile_bytes": tb.value,
+        return {"kernel": {1: "nereus_walk_vec", 2: "nereus_walk_ring", 3: "nereus_walk_once"}[v.value], "tile_bytes": tb.value,
                 "grid": g.value, "threads": th.value}
 
     def estimate(self, gbytes_per_s: float, setup_seconds: float = 0.0) -> float:

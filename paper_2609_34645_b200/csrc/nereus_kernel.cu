@@ -106,9 +106,12 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 
 // The three tile bodies below load a batch of vectors once and store it to every destination replica
 // (`reps` is 1 except for replicated transitions); D(j) yields replica j's base pointer for the tile.
+// Each body runs full batches without predicates; what is left goes one vector at a time (the persistent
+// kernel: its tiles are large, tails are rare, registers are scarce) or, with kBatchTail, as ONE predicated
+// batch, so that a small tile's last (or only) loads are in flight together instead of one round trip each.
 
 // Bit copy of a contiguous run of `nvec` 16-byte vectors.
-template <int kUnroll, class Dst>
+template <int kUnroll, bool kBatchTail, class Dst>
 __device__ __forceinline__ void copy_run(const char* __restrict__ s, Dst D, uint32_t reps, uint32_t nvec,
                                          unsigned lane) {
     s += lane * 16;
@@ -128,19 +131,33 @@ __device__ __forceinline__ void copy_run(const char* __restrict__ s, Dst D, uint
         s += 512 * kUnroll;
         off += 512 * kUnroll;
     }
+    if (!kBatchTail) {
 #pragma unroll 1
-    for (uint32_t i = lane; i < left; i += 32) {                  // ragged tail, one vector at a time
-        const uint4 v = ld_stream(s);
+        for (uint32_t i = lane; i < left; i += 32) {              // ragged tail, one vector at a time
+            const uint4 v = ld_stream(s);
 #pragma unroll 1
-        for (uint32_t j = 0; j < reps; ++j) st_stream(D(j) + off, v);
-        s += 512;
-        off += 512;
+            for (uint32_t j = 0; j < reps; ++j) st_stream(D(j) + off, v);
+            s += 512;
+            off += 512;
+        }
+    } else if (left) {                                            // ragged tail: one predicated batch
+        uint4 v[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u)
+            if (lane + 32 * u < left) v[u] = ld_stream(s + u * 512);
+#pragma unroll 1
+        for (uint32_t j = 0; j < reps; ++j) {
+            char* d = D(j) + off;
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u)
+                if (lane + 32 * u < left) st_stream(d + u * 512, v[u]);
+        }
     }
 }
 
 // Bit copy of a pitched tile: `rows` pieces of `vpr` 16-byte vectors each.  Offsets inside a tile fit
 // 32 bits (rows_per_tile x pitch is far below 4 GiB).
-template <int kUnroll, class Dst>
+template <int kUnroll, bool kBatchTail, class Dst>
 __device__ __forceinline__ void copy_rect(const char* __restrict__ s, Dst D, uint32_t reps, uint32_t rows,
                                           uint32_t vpr, uint32_t sp, uint32_t dp, unsigned lane) {
     const uint32_t nvec = rows * vpr;
@@ -163,12 +180,33 @@ __device__ __forceinline__ void copy_rect(const char* __restrict__ s, Dst D, uin
             for (int u = 0; u < kUnroll; ++u) st_stream(d + doff[u], v[u]);
         }
     }
+    if (!kBatchTail) {
 #pragma unroll 1
-    for (; base < nvec; base += 32) {                                  // ragged tail
-        const uint32_t r = base / vpr, c = base - r * vpr;
-        const uint4 v = ld_stream(s + (r * sp + c * 16));
+        for (; base < nvec; base += 32) {                              // ragged tail, one vector at a time
+            const uint32_t r = base / vpr, c = base - r * vpr;
+            const uint4 v = ld_stream(s + (r * sp + c * 16));
 #pragma unroll 1
-        for (uint32_t j = 0; j < reps; ++j) st_stream(D(j) + (r * dp + c * 16), v);
+            for (uint32_t j = 0; j < reps; ++j) st_stream(D(j) + (r * dp + c * 16), v);
+        }
+    } else if (base < nvec) {                                          // ragged tail: one predicated batch
+        uint4    v[kUnroll];
+        uint32_t doff[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const uint32_t idx = base + u * 32;
+            if (idx < nvec) {
+                const uint32_t r = idx / vpr, c = idx - r * vpr;
+                doff[u] = r * dp + c * 16;
+                v[u] = ld_stream(s + (r * sp + c * 16));
+            }
+        }
+#pragma unroll 1
+        for (uint32_t j = 0; j < reps; ++j) {
+            char* d = D(j);
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u)
+                if (base + u * 32 < nvec) st_stream(d + doff[u], v[u]);
+        }
     }
 }
 
@@ -181,7 +219,7 @@ __device__ __forceinline__ uint2 cast_unit(uint4 v) {
     return o;
 }
 
-template <int kUnroll, class Dst>
+template <int kUnroll, bool kBatchTail, class Dst>
 __device__ __forceinline__ void cast_tile(const char* __restrict__ s, Dst D, uint32_t reps, uint32_t rows,
                                           uint32_t upr, uint32_t sp, uint32_t dp, unsigned lane) {
     const uint32_t nunit = rows * upr;
@@ -209,12 +247,33 @@ __device__ __forceinline__ void cast_tile(const char* __restrict__ s, Dst D, uin
             for (int u = 0; u < kUnroll; ++u) st_stream8(d + doff[u], o[u]);
         }
     }
+    if (!kBatchTail) {
 #pragma unroll 1
-    for (; base < nunit; base += 32) {
-        const uint32_t r = base / upr, c = base - r * upr;
-        const uint2 o = cast_unit(ld_stream(s + (r * sp + c * 16)));
+        for (; base < nunit; base += 32) {                             // ragged tail, one unit at a time
+            const uint32_t r = base / upr, c = base - r * upr;
+            const uint2 o = cast_unit(ld_stream(s + (r * sp + c * 16)));
 #pragma unroll 1
-        for (uint32_t j = 0; j < reps; ++j) st_stream8(D(j) + (r * dp + c * 8), o);
+            for (uint32_t j = 0; j < reps; ++j) st_stream8(D(j) + (r * dp + c * 8), o);
+        }
+    } else if (base < nunit) {                                         // ragged tail: one predicated batch
+        uint2    o[kUnroll];
+        uint32_t doff[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const uint32_t idx = base + u * 32;
+            if (idx < nunit) {
+                const uint32_t r = idx / upr, c = idx - r * upr;
+                doff[u] = r * dp + c * 8;
+                o[u] = cast_unit(ld_stream(s + (r * sp + c * 16)));
+            }
+        }
+#pragma unroll 1
+        for (uint32_t j = 0; j < reps; ++j) {
+            char* d = D(j);
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u)
+                if (base + u * 32 < nunit) st_stream8(d + doff[u], o[u]);
+        }
     }
 }
 
@@ -402,11 +461,11 @@ __global__ void __launch_bounds__(512, 2) nereus_walk_vec(const __grid_constant_
         const uint64_t d_off = t.d_off;
         auto D = [&p, dst_buf, rstride, d_off](uint32_t j) { return tile_dst(p, dst_buf, rstride, d_off, j); };
         if (t.cast) {
-            cast_tile<kUnrollCast>(t.s, D, t.reps, t.nr, t.w >> 3, t.sp, t.dp, lane);
+            cast_tile<kUnrollCast, false>(t.s, D, t.reps, t.nr, t.w >> 3, t.sp, t.dp, lane);
         } else if (t.nr == 1) {
-            copy_run<kUnrollRun>(t.s, D, t.reps, t.w >> 4, lane);
+            copy_run<kUnrollRun, false>(t.s, D, t.reps, t.w >> 4, lane);
         } else {
-            copy_rect<kUnrollRect>(t.s, D, t.reps, t.nr, t.w >> 4, t.sp, t.dp, lane);
+            copy_rect<kUnrollRect, false>(t.s, D, t.reps, t.nr, t.w >> 4, t.sp, t.dp, lane);
         }
         if (p.n_levels > 1) ++my_done;
         g = more ? base + claim_take(next_issued) : p.n_tiles;
@@ -417,6 +476,46 @@ __global__ void __launch_bounds__(512, 2) nereus_walk_vec(const __grid_constant_
         if (lane == 0) atomicAdd(&ctrl->done, my_done);
     }
     finish_block(ctrl);
+}
+
+// ---------------------------------------------------------------------------------------------------
+// small tables: one warp per tile, no loop
+// ---------------------------------------------------------------------------------------------------
+//
+// A table of a few thousand tiles is over before a persistent grid has warmed up: what counts is the chain of
+// dependent memory trips in front of the first load and the number of bytes in flight.  Here a warp's tile is
+// its index in the grid and its addresses come with one 48-byte record; there is no cursor, no claim, no
+// shared memory and nothing to reset; the hardware's block scheduler does the balancing.  Single-level tables
+// with per-tile records and at most kOnceMaxBuffers buffers only (the parameter block stays small).
+
+constexpr int kOnceMaxBuffers = 64;
+
+struct OnceParams {
+    const TileRec* tiles;
+    Ctrl*          ctrl;
+    uint32_t       n_tiles;
+    char*          bufs[kOnceMaxBuffers];
+};
+
+__global__ void __launch_bounds__(512, 2) nereus_walk_once(const __grid_constant__ OnceParams p) {
+    const unsigned lane = threadIdx.x & 31;
+    const uint32_t g = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (g >= p.n_tiles) return;
+    const uint4* q = reinterpret_cast<const uint4*>(p.tiles + g);
+    const uint4 a = __ldg(q), b = __ldg(q + 1), c = __ldg(q + 2);
+    const uint32_t src_buf = c.x & 0xFFFFu, dst_buf = c.x >> 16;
+    const uint32_t reps = c.y & 0xFFFFu, rstride = c.y >> 16, cast = c.z >> 16;
+    if (src_buf >= (uint32_t)kOnceMaxBuffers || reps == 0 || b.z == 0 ||
+        dst_buf + (reps - 1) * rstride >= (uint32_t)kOnceMaxBuffers) {
+        if (lane == 0) raise_status(p.ctrl, NEREUS_DEV_BOUNDS, g);
+        return;
+    }
+    const char*    s     = p.bufs[src_buf] + (((uint64_t)a.y << 32) | a.x);
+    const uint64_t d_off = ((uint64_t)a.w << 32) | a.z;
+    auto D = [&p, dst_buf, rstride, d_off](uint32_t j) { return p.bufs[dst_buf + j * rstride] + d_off; };
+    if (cast)          cast_tile<kUnrollCast, true>(s, D, reps, b.z, b.w >> 3, b.x, b.y, lane);
+    else if (b.z == 1) copy_run<kUnrollRun, true>(s, D, reps, b.w >> 4, lane);
+    else               copy_rect<kUnrollRect, true>(s, D, reps, b.z, b.w >> 4, b.x, b.y, lane);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -793,7 +892,7 @@ static int env_int(const char* name, int dflt) {
 
 // Launch shape of one run, from the handle's tuning, the environment and the table.
 struct Launch {
-    int      variant = 1;           // 1 vector copy, 2 bulk-copy ring
+    int      variant = 1;           // 1 vector copy, 2 bulk-copy ring, 3 one warp per tile
     bool     cast = false;          // ring only: the table is all cast
     int      tile_bytes = 0, ctas_per_sm = 0, threads = 0;
     uint32_t n_stages = 0;          // bulk ring
@@ -801,19 +900,26 @@ struct Launch {
     size_t   smem = 0;
 };
 
-// Both kernels take every table.  The ring runs an all-bit-copy table on the bulk-store consumer and
-// anything with a cast in it on the converting consumers (which copy the bit-copy tiles of a mixed table from
-// shared memory as well).  Default: the ring for tables that write 64 MiB or more (its per-block start-up
-// costs more than it gains below that), the vector kernel for smaller ones.
-static int resolve_launch(const nereus_transition_s& t, int sms, Launch& L) {
+// Which kernel walks a table (nereus_transition_tune and NEREUS_VARIANT override):
+//   * single-level tables that write less than 1 GiB through at most kOnceMaxBuffers buffers: one warp per
+//     tile (nereus_walk_once); measured on B200 it is the fastest from a few MB up to about 1 GiB;
+//   * otherwise tables that write 64 MiB or more: the ring (its per-block start-up costs more than it gains
+//     below that); all-bit-copy tables on the bulk-store consumer, anything with a cast in it on the
+//     converting consumers (which copy the bit-copy tiles of a mixed table from shared memory as well);
+//   * what is left (small chained tables, small tables with very many buffers): the persistent vector kernel.
+static int resolve_launch(const nereus_transition_s& t, int sms, Launch& L, bool once_fits = true) {
     const int want = t.tuning.variant ? t.tuning.variant : env_int("NEREUS_VARIANT", 0);
     const int asked_tile = t.tuning.tile_bytes ? t.tuning.tile_bytes : env_int("NEREUS_TILE_BYTES", 0);
     L.cast = false;
     for (const Rect& r : t.rects) L.cast = L.cast || r.cast;
+    const bool once_ok = once_fits && t.n_levels == 1 &&
+                         t.src_bytes.size() + t.dst_bytes.size() <= (size_t)kOnceMaxBuffers;
     if (want)  L.variant = want;
+    else if (once_ok && t.bytes_written < (1ull << 30)) L.variant = 3;
     else       L.variant = (t.bytes_written >= (64ull << 20) && asked_tile <= (L.cast ? 24576 : 49152)) ? 2 : 1;
+    if (L.variant == 3 && !once_ok) L.variant = 1;
     L.ctas_per_sm = t.tuning.ctas_per_sm ? t.tuning.ctas_per_sm : env_int("NEREUS_CTAS_PER_SM", 2);
-    L.threads     = t.tuning.threads     ? t.tuning.threads     : env_int("NEREUS_THREADS", 384);
+    L.threads     = t.tuning.threads     ? t.tuning.threads     : env_int("NEREUS_THREADS", L.variant == 3 ? 256 : 384);
     L.tile_bytes  = asked_tile;
     if (L.variant == 2) { L.ctas_per_sm = t.tuning.ctas_per_sm ? t.tuning.ctas_per_sm : 1; L.threads = 64; }
     if (L.ctas_per_sm < 1 || L.ctas_per_sm > 2 || L.threads < 32 || L.threads > 512 || L.threads % 32)
@@ -823,9 +929,15 @@ static int resolve_launch(const nereus_transition_s& t, int sms, Launch& L) {
         // every other claimer gets a tile; a tile stays a multiple of 512 bytes
         L.tile_bytes = L.variant == 2 ? (L.cast ? 24576 : 32768) : 16384;
         const uint64_t claimers = (uint64_t)sms * L.ctas_per_sm * (L.variant == 2 ? 8 : L.threads / 32);
-        while (L.tile_bytes / 2 >= 1024 && (L.tile_bytes / 2) % 512 == 0 &&
+        while (L.variant != 3 && L.tile_bytes / 2 >= 1024 && (L.tile_bytes / 2) % 512 == 0 &&
                t.bytes_written / L.tile_bytes < claimers / 2)
             L.tile_bytes /= 2;
+        if (L.variant == 3) {
+            // one batch of loads per warp (32 lanes x 8 vectors = 4 KiB), larger only to stay within the
+            // number of tiles that get per-tile records
+            L.tile_bytes = 4096;
+            while (t.bytes_written / L.tile_bytes > kDirectMaxTiles * 3ull / 4) L.tile_bytes *= 2;
+        }
     }
     if (L.tile_bytes < 512 || L.tile_bytes % 512) return NEREUS_ERR_ARG;
     if (L.variant == 2) {
@@ -842,6 +954,22 @@ static int resolve_launch(const nereus_transition_s& t, int sms, Launch& L) {
         if (L.claim < 1 || L.claim > 64) return NEREUS_ERR_ARG;
         if (L.piece < 16 || L.piece % 16 || L.lag < 1 || L.lag > 8 || L.lag + 2 > L.n_stages) return NEREUS_ERR_ARG;
     }
+    return NEREUS_OK;
+}
+
+// Kernel, launch shape and tiling of a table on a device with `sms` SMs, into arrays of rects.size() and
+// rects.size() + 1 entries.  `records`: the caller can carry per-tile records (the allocation-free path
+// cannot); a table that was to run one warp per tile but has more tiles than get records falls back to the
+// kernels that search the tile prefix, with their own tile size.
+static int plan_launch(const nereus_transition_s& t, int sms, bool records, Launch& L, RectDev* rects,
+                       uint32_t* first, uint32_t level_end[kMaxLevels], uint64_t& n_tiles) {
+    if (int rc = resolve_launch(t, sms, L, records)) return rc;
+    n_tiles = tile_table_raw(t, (uint32_t)L.tile_bytes, rects, first, level_end);
+    if (L.variant == 3 && (n_tiles == 0 || n_tiles > kDirectMaxTiles)) {
+        if (int rc = resolve_launch(t, sms, L, false)) return rc;
+        n_tiles = tile_table_raw(t, (uint32_t)L.tile_bytes, rects, first, level_end);
+    }
+    if (n_tiles == 0 && !t.rects.empty()) return NEREUS_ERR_UNSUPPORTED;      // more than 2^32 tiles
     return NEREUS_OK;
 }
 
@@ -870,7 +998,14 @@ static int launch_walk(const Launch& L, int sms, const WalkParams& p, cudaStream
         } else {
             nereus_walk_ring<false><<<grid, 64, L.smem, stream>>>(p, (uint32_t)L.tile_bytes, L.n_stages, L.piece, L.lag, L.claim);
         }
+    } else if (L.variant == 3 && p.tiles) {
+        OnceParams o;
+        o.tiles = p.tiles; o.ctrl = p.ctrl; o.n_tiles = p.n_tiles;
+        for (int k = 0; k < kOnceMaxBuffers; ++k) o.bufs[k] = p.bufs[k];
+        const unsigned warps_per_cta = (unsigned)L.threads / 32;
+        nereus_walk_once<<<(p.n_tiles + warps_per_cta - 1) / warps_per_cta, L.threads, 0, stream>>>(o);
     } else {
+        // (a table asked to run one warp per tile that turned out too large for per-tile records lands here)
         const unsigned warps_per_cta = (unsigned)L.threads / 32;
         unsigned grid = (unsigned)(sms * L.ctas_per_sm);
         grid = std::max(1u, std::min(grid, (p.n_tiles + warps_per_cta - 1) / warps_per_cta));
@@ -888,19 +1023,16 @@ static int prepare(nereus_transition_s& t) {
 
     int sms = 0;
     NEREUS_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
-    Launch L;
-    if (int rc = resolve_launch(t, sms, L)) return rc;
     if (int rc = ring_opt_in(device)) return rc;
-
     DeviceTable dv;
     dv.device = device;
     dv.sm_count = sms;
+    Launch L;
+    std::vector<RectDev>  rects(t.rects.size());
+    std::vector<uint32_t> first(t.rects.size() + 1);
+    uint64_t n_tiles = 0;
+    if (int rc = plan_launch(t, sms, true, L, rects.data(), first.data(), dv.level_end, n_tiles)) return rc;
     dv.tile_bytes = L.tile_bytes; dv.ctas_per_sm = L.ctas_per_sm; dv.threads = L.threads; dv.variant = L.variant;
-
-    std::vector<RectDev>  rects;
-    std::vector<uint32_t> first;
-    const uint64_t n_tiles = tile_table(t, (uint32_t)dv.tile_bytes, rects, first, dv.level_end);
-    if (n_tiles == 0 && !t.rects.empty()) return NEREUS_ERR_UNSUPPORTED;
     dv.n_tiles = (uint32_t)n_tiles;
 
     // nothing reaches the device that the host has not checked against the declared buffer sizes
@@ -996,7 +1128,7 @@ static int read_and_clear_status(Ctrl* ctrl, int* device_status) {
 extern "C" {
 
 int nereus_transition_tune(nereus_transition_t t, int tile_bytes, int ctas_per_sm, int threads, int variant) {
-    if (!t || tile_bytes < 0 || ctas_per_sm < 0 || threads < 0 || variant < 0 || variant > 2) return NEREUS_ERR_ARG;
+    if (!t || tile_bytes < 0 || ctas_per_sm < 0 || threads < 0 || variant < 0 || variant > 3) return NEREUS_ERR_ARG;
     if (tile_bytes && (tile_bytes < 512 || tile_bytes % 512)) return NEREUS_ERR_ARG;
     if (ctas_per_sm > 2 || threads > 512 || threads % 32) return NEREUS_ERR_ARG;
     t->tuning.tile_bytes = tile_bytes; t->tuning.ctas_per_sm = ctas_per_sm;
@@ -1008,28 +1140,38 @@ int nereus_transition_tune(nereus_transition_t t, int tile_bytes, int ctas_per_s
 int nereus_transition_num_tiles(nereus_transition_t t, uint64_t* tiles, int* levels) {
     try {
         if (!t || !tiles || !levels) return NEREUS_ERR_ARG;
-        std::vector<RectDev> rects; std::vector<uint32_t> first; uint32_t le[kMaxLevels];
-        int tb = t->dev.tile_bytes;
-        if (!t->dev.rects) {                      // not prepared: what a 148-SM device would get
-            Launch L;
-            if (int rc = resolve_launch(*t, 148, L)) return rc;
-            tb = L.tile_bytes;
-        }
-        *tiles = tile_table(*t, (uint32_t)tb, rects, first, le);
+        if (t->dev.rects) { *tiles = t->dev.n_tiles; *levels = t->n_levels; return NEREUS_OK; }
+        // not prepared: what a 148-SM device would get
+        std::vector<RectDev> rects(t->rects.size()); std::vector<uint32_t> first(t->rects.size() + 1);
+        uint32_t le[kMaxLevels];
+        Launch L;
+        uint64_t n = 0;
+        if (int rc = plan_launch(*t, 148, true, L, rects.data(), first.data(), le, n)) return rc;
+        *tiles = n;
         *levels = t->n_levels;
         return NEREUS_OK;
     } catch (const std::bad_alloc&) { return NEREUS_ERR_NOMEM; }
 }
 
 int nereus_transition_launch_info(nereus_transition_t t, int* variant, int* tile_bytes, int* grid, int* threads) {
-    if (!t || !variant || !tile_bytes || !grid || !threads) return NEREUS_ERR_ARG;
-    const int sms = t->dev.rects ? t->dev.sm_count : 148;
-    Launch L;
-    if (int rc = resolve_launch(*t, sms, L)) return rc;
-    if (t->dev.rects) L.tile_bytes = t->dev.tile_bytes;
-    *variant = L.variant; *tile_bytes = L.tile_bytes; *grid = sms * L.ctas_per_sm;
-    *threads = L.variant == 2 ? (L.cast ? 32 + (int)kCastConsumers : 64) : L.threads;
-    return NEREUS_OK;
+    try {
+        if (!t || !variant || !tile_bytes || !grid || !threads) return NEREUS_ERR_ARG;
+        const int sms = t->dev.rects ? t->dev.sm_count : 148;
+        Launch L;
+        uint64_t n_tiles = t->dev.n_tiles;
+        if (t->dev.rects) {
+            if (int rc = resolve_launch(*t, sms, L, t->dev.variant == 3)) return rc;
+        } else {
+            std::vector<RectDev> rects(t->rects.size()); std::vector<uint32_t> first(t->rects.size() + 1);
+            uint32_t le[kMaxLevels];
+            if (int rc = plan_launch(*t, sms, true, L, rects.data(), first.data(), le, n_tiles)) return rc;
+        }
+        const int warps = L.threads / 32;
+        *grid = L.variant == 3 ? (int)((n_tiles + warps - 1) / warps) : sms * L.ctas_per_sm;   // one warp per tile
+        *variant = L.variant; *tile_bytes = L.tile_bytes;
+        *threads = L.variant == 2 ? (L.cast ? 32 + (int)kCastConsumers : 64) : L.threads;
+        return NEREUS_OK;
+    } catch (const std::bad_alloc&) { return NEREUS_ERR_NOMEM; }
 }
 
 int nereus_transition_prepare(nereus_transition_t t) {
@@ -1048,9 +1190,9 @@ int nereus_transition_run(nereus_transition_t t, const void* const* src_ptrs, vo
         const DeviceTable& dv = t->dev;
         cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
 
-        Launch L;
-        if (int rc = resolve_launch(*t, dv.sm_count, L)) return rc;
-        L.tile_bytes = dv.tile_bytes;
+        Launch L;                       // the same answer prepare got (it falls back when per-tile records do not fit)
+        if (int rc = resolve_launch(*t, dv.sm_count, L, dv.variant == 3)) return rc;
+        if (L.variant != dv.variant || L.tile_bytes != dv.tile_bytes) return NEREUS_ERR_ARG;
         WalkParams p;
         // the control words need no reset: every launch leaves them zeroed for the next one
         p.rects = dv.rects; p.first = dv.first; p.tiles = dv.tiles; p.ctrl = dv.ctrl;
@@ -1173,11 +1315,9 @@ extern "C" int nereus_transition_run_static(nereus_transition_t t, const void* c
     if (int rc = static_scratch(device, &scratch, &sms)) return rc;
 
     Launch L;
-    if (int rc = resolve_launch(*t, sms, L)) return rc;
-
     WalkParams p;
-    const uint64_t n_tiles = tile_table_raw(*t, (uint32_t)L.tile_bytes, g_static_rects, g_static_first, p.level_end);
-    if (n_tiles == 0 && n_rects != 0) return NEREUS_ERR_UNSUPPORTED;
+    uint64_t n_tiles = 0;      // no room for per-tile records in the fixed array: the kernels that search the prefix
+    if (int rc = plan_launch(*t, sms, false, L, g_static_rects, g_static_first, p.level_end, n_tiles)) return rc;
     if (int rc = validate_table(*t, g_static_rects, g_static_first, n_tiles, g_static_order)) return rc;
 
     RectDev*  d_rects = reinterpret_cast<RectDev*>(scratch);

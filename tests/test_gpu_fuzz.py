@@ -36,7 +36,7 @@ def draw(rng):
     sdt = rng.choice(["bf16", "bf16", "fp32"])
     ddt = "bf16" if sdt == "bf16" else rng.choice(["fp32", "bf16"])
     return dict(sh=sh, a=a, b=b, sdt=sdt, ddt=ddt, la=rng.randrange(4) | pad_a, lb=rng.randrange(4) | pad_b,
-                vh=rng.random() < 0.25, k=rng.choice([1, 1, 1, 2, 3]), variant=rng.choice([1, 2]),
+                vh=rng.random() < 0.25, k=rng.choice([1, 1, 1, 2, 3]), variant=rng.choice([1, 2, 3]),
                 tile=rng.choice([512, 1024, 4096, 16384]))
 
 

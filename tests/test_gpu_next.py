@@ -14,7 +14,7 @@ from paper_2609_34645_b200 import inputs as I
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("variant", [1, 2])
+@pytest.mark.parametrize("variant", [1, 2, 3])
 @pytest.mark.parametrize("a,b,k,sdt,ddt", [((2, 2), (2, 2), 3, "bf16", "bf16"),      # Extend
                                            ((4, 1), (2, 2), 2, "bf16", "bf16"),      # Split into 2 replica units
                                            ((1, 1), (4, 2), 4, "bf16", "bf16"),
@@ -37,7 +37,7 @@ def test_replicated_destinations(a, b, k, sdt, ddt, variant):
         assert dst.guards_intact()
 
 
-@pytest.mark.parametrize("variant", [1, 2])
+@pytest.mark.parametrize("variant", [1, 2, 3])
 def test_state_with_adam_moments(variant):
     sh = I.SMALL
     desc = G.desc_of(sh)
@@ -157,7 +157,7 @@ def test_transition_estimate_predicts_the_measured_time():
     torch.cuda.empty_cache()
 
 
-@pytest.mark.parametrize("variant", [1, 2])
+@pytest.mark.parametrize("variant", [1, 2, 3])
 @pytest.mark.parametrize("la,lb", [(3, 0), (0, 3), (1, 2), (3, 3)])
 def test_layout_variants_on_the_gpu(la, lb, variant):
     """Grouped QKV / row-interleaved gate-up on either side, with and without the cast, both kernels."""
@@ -268,7 +268,7 @@ def test_8b_dag_full_size():
 GQA16 = I.Shape(2, 128, 16, 2, 256, 256)          # 16 q heads, 2 kv heads, head_dim 8
 
 
-@pytest.mark.parametrize("variant", [1, 2])
+@pytest.mark.parametrize("variant", [1, 2, 3])
 @pytest.mark.parametrize("a,b", [((1, 1), (8, 1)), ((8, 2), (2, 1)), ((16, 1), (4, 2)), ((4, 1), (16, 1))])
 def test_kv_head_replication_on_the_gpu(a, b, variant):
     """tp > kv_heads on either side, bit copy and cast, both kernels."""
@@ -306,7 +306,7 @@ def test_8b_tp16_beyond_the_kv_heads_full_size():
     torch.cuda.empty_cache()
 
 
-@pytest.mark.parametrize("variant", [1, 2])
+@pytest.mark.parametrize("variant", [1, 2, 3])
 def test_mixed_cast_and_copy_table(variant):
     """One table with cast tiles (fp32 parameters -> bf16) and bit-copy tiles (fp32 optimizer moments): the
     converting ring serves both kinds."""
@@ -317,7 +317,7 @@ def test_mixed_cast_and_copy_table(variant):
     t = desc.compile_state(pa, pb, 2)
     assert {r.cast for r in t.rects()} == {0, 1}
     t.tune(variant=variant, tile_bytes=4096)
-    assert t.launch_info()["kernel"] == ("nereus_walk_ring" if variant == 2 else "nereus_walk_vec")
+    assert t.launch_info()["kernel"] == {1: "nereus_walk_vec", 2: "nereus_walk_ring", 3: "nereus_walk_once"}[variant]
     src = G.device_sources(desc, pa, "fp32", 1) + G.device_sources(desc, pa, "fp32", 2) + \
         G.device_sources(desc, pa, "fp32", 3)
     dst = G.Guarded([t.buffer_bytes(True, j) for j in range(t.num_buffers()[1])])
@@ -329,7 +329,7 @@ def test_mixed_cast_and_copy_table(variant):
     assert dst.guards_intact()
 
 
-@pytest.mark.parametrize("variant", [1, 2])
+@pytest.mark.parametrize("variant", [1, 2, 3])
 def test_padded_vocabulary_on_the_gpu(variant):
     """Vocabulary padded to a multiple of 128*tp on either side: padding rows stay as they were (sentinel)."""
     sh = I.Shape(2, 64, 4, 4, 128, 1000)

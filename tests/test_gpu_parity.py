@@ -56,6 +56,46 @@ def test_bulk_ring_kernel(tile):
     G.check_against_oracle(I.SMALL, (2, 2), (4, 1), "fp32", "bf16", vh=True, seed=8, tune=tune)
 
 
+@pytest.mark.parametrize("tile", [512, 1536, 4096, 16384])
+def test_one_warp_per_tile_kernel(tile):
+    """nereus_walk_once (one warp per tile, per-tile records, no control words) on the same plan pairs: tiles of
+    less than one batch, of exactly one, of several, ragged tails, 16-byte pieces, casts, value heads."""
+    tune = dict(tile_bytes=tile, variant=3)
+    for a, b in [((1, 1), (4, 2)), ((4, 2), (1, 1)), ((2, 4), (4, 1)), ((4, 4), (2, 2)), ((2, 1), (2, 1))]:
+        t = G.check_against_oracle(I.SMALL, a, b, seed=tile + 2, tune=tune)
+        assert t.launch_info()["kernel"] == "nereus_walk_once"
+    G.check_against_oracle(I.SMALL, (2, 1), (4, 2), vh=True, seed=5, tune=tune)
+    G.check_against_oracle(I.SMALL, (1, 2), (4, 1), "fp32", "fp32", seed=3, tune=tune)
+    for a, b in [((4, 8), (8, 2)), ((8, 1), (1, 8))]:
+        G.check_against_oracle(I.MICRO, a, b, seed=9, tune=tune)
+    for a, b in [((2, 2), (4, 1)), ((1, 1), (2, 2)), ((4, 4), (1, 1)), ((2, 1), (2, 1))]:
+        G.check_against_oracle(I.SMALL, a, b, "fp32", "bf16", seed=2, tune=tune)
+    G.check_against_oracle(I.MICRO, (4, 8), (8, 2), "fp32", "bf16", seed=4, tune=tune)
+    G.check_against_oracle(I.SMALL, (2, 2), (4, 1), "fp32", "bf16", vh=True, seed=8, tune=tune)
+    for threads in (32, 128, 512):
+        G.check_against_oracle(I.SMALL, (2, 2), (4, 1), seed=1, tune=dict(tile_bytes=tile, variant=3, threads=threads))
+
+
+def test_default_kernel_by_table():
+    """What runs when nothing is tuned: one warp per tile for single-level tables below 1 GiB with few buffers,
+    the persistent kernels for chained tables and for tables with more buffers than its parameter block holds."""
+    d = G.desc_of(I.SMALL)
+    assert d.compile(B.Plan(2, 2), B.Plan(4, 1)).launch_info()["kernel"] == "nereus_walk_once"
+    ch = B.Transition.fuse([d.compile(B.Plan(2, 2), B.Plan(4, 1)), d.compile(B.Plan(4, 1), B.Plan(2, 2))], chained=True)
+    assert ch.launch_info()["kernel"] == "nereus_walk_vec"
+    ch.tune(variant=3)                                        # asked for, not possible: falls back
+    assert ch.launch_info()["kernel"] == "nereus_walk_vec"
+    many = G.desc_of(I.MICRO).compile(B.Plan(8, 8), B.Plan(8, 4))          # 96 buffers
+    assert many.launch_info()["kernel"] == "nereus_walk_vec"
+    G.check_against_oracle(I.MICRO, (8, 8), (8, 4), seed=12)
+    big = G.desc_of(I.LLAMA_8B).compile(B.Plan(1, 1), B.Plan(4, 2))
+    assert big.launch_info()["kernel"] == "nereus_walk_ring"
+    # a tile so small that the table has more tiles than get per-tile records: the vector kernel takes over
+    t = G.desc_of(I.Shape(2, 2048, 16, 8, 5632, 8192)).compile(B.Plan(1, 1), B.Plan(4, 1))
+    t.tune(variant=3, tile_bytes=512)
+    assert t.num_tiles()[0] > 1 << 17 and t.launch_info()["kernel"] == "nereus_walk_vec"
+
+
 @pytest.mark.parametrize("threads,ctas", [(512, 2), (256, 1), (32, 1)])
 def test_launch_shapes(threads, ctas):
     G.check_against_oracle(I.SMALL, (2, 2), (4, 1), seed=1, tune=dict(threads=threads, ctas_per_sm=ctas, variant=1))
@@ -82,7 +122,7 @@ def test_fp32_copy_and_value_head():
     G.check_against_oracle(I.SMALL, (2, 2), (4, 1), "fp32", "bf16", vh=True, seed=8)
 
 
-@pytest.mark.parametrize("variant", [1, 2])
+@pytest.mark.parametrize("variant", [1, 2, 3])
 def test_cast_every_fp32_bit_pattern(variant):
     """All 2^32 fp32 bit patterns through the kernel's cast (NaN, Inf, subnormals, ties) against the oracle's
     rule.  The patterns are planted in the embedding of a one-layer model, 2^28 at a time."""

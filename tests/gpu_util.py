@@ -2,6 +2,9 @@
 destination buffers with sentinel fill and guard zones, and the comparison with the CPU oracle."""
 from __future__ import annotations
 
+import os
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 import torch
 
@@ -115,3 +118,76 @@ def check_against_oracle(sh, a, b, sdt="bf16", ddt="bf16", vh=False, seed=0, tun
             raise AssertionError(f"{a}->{b} shard {j}: {bad.size} bytes differ, first at {bad[0]}")
     assert dst.guards_intact()
     return t
+
+
+# ---------------------------------------------------------------- every logical tensor, at any size
+
+def host_workers() -> int:
+    """Threads the full-size comparisons may use: the cores this process may run on, at most 32."""
+    try:
+        n = len(os.sched_getaffinity(0))
+    except AttributeError:
+        n = os.cpu_count() or 1
+    return max(1, min(32, n))
+
+
+def _span_bytes(m, plan, tid, part, es):
+    """Bytes from the first element of a shard's part of logical tensor tid to the end of its last row (the
+    rows of a part are interleaved with other tensors' rows under the grouped and interleaved layouts)."""
+    if not part.held:
+        return 0
+    return (O.part_row(m, plan, tid, part.nr - 1) + 1) * part.nc * es
+
+
+def _compare_one_tensor(m, pa, pb, tid, src, dst_units, ses, des):
+    """One logical tensor through the oracle, from device slices of the sources, against the device result of
+    every destination unit.  The oracle (single-threaded, as it stands) writes the tensor's rows over a host copy
+    of what the device holds in the span of each part: equal afterwards means every element was right."""
+    ns, nd = O.num_shards(m, pa), O.num_shards(m, pb)
+    sparts = []
+    for s in range(ns):
+        p = O.locate(m, pa, s, tid)
+        n = _span_bytes(m, pa, tid, p, ses)
+        sparts.append(src[s][p.offset:p.offset + n].cpu().numpy() if p.held else None)
+    where = [O.locate(m, pb, d, tid) for d in range(nd)]
+    spans = [_span_bytes(m, pb, tid, p, des) for p in where]
+    first = dst_units[0]
+    got = [first[d][p.offset:p.offset + n].cpu().numpy() if p.held else None for d, (p, n) in enumerate(zip(where, spans))]
+    want = [None if g is None else g.copy() for g in got]
+    O.reshard_tensor_parts(m, pa, pb, tid, sparts, want)
+    compared = 0
+    for d, (g, w) in enumerate(zip(got, want)):
+        if g is None:
+            continue
+        if not np.array_equal(g, w):
+            bad = np.flatnonzero(g != w)
+            return f"logical tensor {tid}, destination shard {d}: {bad.size} bytes differ, first at {int(bad[0])}"
+        compared += g.size
+    # further units (replicas) hold what the first one holds, byte for byte
+    for k, dst in enumerate(dst_units[1:], 1):
+        for d, (p, n) in enumerate(zip(where, spans)):
+            if p.held and not torch.equal(dst[d][p.offset:p.offset + n], first[d][p.offset:p.offset + n]):
+                return f"logical tensor {tid}, unit {k}, destination shard {d} differs from unit 0"
+            compared += n if p.held else 0
+    return compared
+
+
+def compare_every_tensor(jobs, workers=None):
+    """jobs: iterable of (model, src plan, dst plan, source buffers, [destination units]) with device buffers
+    (torch uint8) and oracle-side models and plans.  EVERY logical tensor of every job goes through the oracle
+    and is compared element by element with the device result; disjoint tensors run on a pool of host threads
+    (each oracle call is the single-threaded C routine; ctypes and the copies release the interpreter lock).
+    Returns the destination bytes compared; raises AssertionError on the first difference."""
+    tasks = []
+    for m, pa, pb, src, dst_units in jobs:
+        ses, des = O.es(m, pa), O.es(m, pb)
+        for tid in range(O.num_logical(m)):
+            rows, cols = O.logical_shape(m, tid)
+            tasks.append((rows * cols, m, pa, pb, tid, src, dst_units, ses, des))
+    tasks.sort(key=lambda x: -x[0])                         # the embeddings first: they take the longest
+    total = 0
+    with ThreadPoolExecutor(max_workers=workers or host_workers()) as pool:
+        for res in pool.map(lambda a: _compare_one_tensor(*a[1:]), tasks):
+            assert not isinstance(res, str), res
+            total += res
+    return total

@@ -1,18 +1,19 @@
 """Full-size parity of the benchmark workloads, in the launch configuration bench.py times.
 
-The oracle cannot stream 16-130 GB through one core inside a test, so each workload is checked in two ways:
-  * sampled logical tensors (first, middle and last layer, embedding, final norm, head) go through the oracle
-    one by one, from device slices of the sources, and are compared bit for bit with the device result;
-  * a property that holds at any size: for EVERY stored tensor the sum of its elements' bit patterns is the
-    same on the source and the destination side (for the cast: the sum over torch's fp32 -> bf16 conversion of
-    the source, which the CPU pins prove equal to the oracle's rule on non-NaN values), and every replicated
-    copy equals the first.
+Each workload is checked in two ways:
+  * EVERY logical tensor (all 9L+3 of every model-stage) goes through the CPU oracle, from device slices of the
+    sources, and is compared element by element with the device result (gpu_util.compare_every_tensor: the
+    oracle call is the single-threaded routine as it stands; disjoint tensors run on a pool of host threads);
+  * as a second line, a property that holds at any size: for every stored tensor the sum of its elements' bit
+    patterns is the same on the source and the destination side (for the cast: the sum over torch's fp32 ->
+    bf16 conversion of the source), and every replicated copy equals the first.
 """
 import numpy as np
 import pytest
 import torch
 
 import bench
+import gpu_util as G
 from oracle import oracle as O
 from paper_2609_34645_b200 import binding as B
 from paper_2609_34645_b200 import inputs as I
@@ -115,20 +116,29 @@ def _run_workload(name):
     return wl, t, srcs, dsts, descs
 
 
+def oracle_job(st, src, dst_units, src_plan=None, dst_plan=None):
+    """(model, source plan, target plan, sources, destination units) of one model-stage for
+    gpu_util.compare_every_tensor, on the oracle's side of the fence."""
+    sh = st.shape
+    a, b = src_plan or st.src, dst_plan or st.dst
+    m = O.Model(sh.layers, sh.hidden, sh.heads, sh.kv_heads, sh.ffn, sh.vocab, ODT[a[2]], st.value_head)
+    return (m, O.Plan(a[0], a[1], 0, I.layout_of(a)), O.Plan(b[0], b[1], ODT[b[2]], I.layout_of(b)), src, dst_units)
+
+
 def _check_plain_workload(name):
     wl, t, srcs, dsts, descs = _run_workload(name)
     si = di = 0
+    jobs = []
     for st, (desc, pa, pb) in zip(wl.stages, descs):
         ns, nd = desc.num_shards(pa), desc.num_shards(pb)
         src, dst = srcs[si:si + ns], dsts[di:di + nd]
         si += ns
         di += nd
         _check_stage_sums(st, desc, src, dst, pa, pb, st.src[2], st.dst[2])
-        ids = _sample_ids(st.shape.layers) if len(wl.stages) == 1 else \
-            [0, 1, 2, 3, 4, 5, 6, 7, 8, 9, 9 * st.shape.layers + 1, 9 * st.shape.layers + 2]
-        _check_stage_sampled(st, src, dst, st.src, st.dst, ids)
+        jobs.append(oracle_job(st, src, [dst]))
     rd, wr = t.bytes()
-    del srcs, dsts, src, dst
+    assert G.compare_every_tensor(jobs) == wr                 # every destination byte went through the oracle
+    del srcs, dsts, src, dst, jobs
     torch.cuda.empty_cache()
     return rd, wr
 
@@ -203,9 +213,9 @@ def test_32b_round_trip_into_the_sources():
     t.run([b.data_ptr() for b in srcs], [b.data_ptr() for b in dsts], stream.cuda_stream)
     stream.synchronize()
     assert t.status() == B.DEV_OK and t.num_tiles()[1] == 2
-    # forward level against the oracle (the sources hold the same bits again after the way back)
+    # forward level against the oracle, every tensor (the sources hold the same bits again after the way back)
     _check_stage_sums(st, desc, srcs, mid, pa, pb, "bf16", "bf16")
-    _check_stage_sampled(st, srcs, mid, st.src, st.dst, ids + [0])
+    assert G.compare_every_tensor([oracle_job(st, srcs, [mid])]) == parts[0].bytes()[1]
     # the restored sources
     assert [b.view(torch.int16).sum(dtype=torch.int64).item() for b in srcs] == sums
     for (tid, s), (p, want) in kept.items():
@@ -220,6 +230,8 @@ def test_32b_round_trip_into_the_sources():
     assert [b.view(torch.int16).sum(dtype=torch.int64).item() for b in srcs] == sums
     for (tid, s), (p, want) in kept.items():
         assert np.array_equal(srcs[s][p.offset:p.offset + want.size].cpu().numpy(), want), (tid, s)
+    # ... and the way back against the oracle, every tensor: middle layout -> original layout
+    assert G.compare_every_tensor([oracle_job(st, mid, [srcs], st.dst, st.src)]) == parts[1].bytes()[1]
     rd, wr = t.bytes()
     assert abs(rd + wr - 2 * 131.05e9) < 0.3e9
     del srcs, dsts, mid

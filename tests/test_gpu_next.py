@@ -103,9 +103,9 @@ def test_8b_weight_sync_to_two_generation_units_full_size():
     for j in range(n):
         assert torch.equal(dsts[j], dsts[n + j])                      # the two units are identical
     F._check_stage_sums(st, desc, srcs, dsts[:n], pa, pb, "fp32", "bf16")
-    F._check_stage_sampled(st, srcs, dsts[:n], st.src, st.dst, list(range(1, 10)) + [9 * 32 + 1])
     rd, wr = t.bytes()
     assert rd == wr                                                   # 4 B read, 2 x 2 B written per element
+    assert G.compare_every_tensor([F.oracle_job(st, srcs, [dsts[:n], dsts[n:]])]) == wr   # every tensor, both units
     del srcs, dsts
     torch.cuda.empty_cache()
 
@@ -117,7 +117,7 @@ def test_8b_state_with_adam_full_size():
     ns, nd = desc.num_shards(pa), desc.num_shards(pb)
     # parameters
     F._check_stage_sums(st, desc, srcs[:ns], dsts[:nd], pa, pb, "bf16", "bf16")
-    F._check_stage_sampled(st, srcs[:ns], dsts[:nd], st.src, st.dst, list(range(1, 10)) + [9 * 32 + 1])
+    jobs = [F.oracle_job(st, srcs[:ns], [dsts[:nd]])]
     # the two moments: fp32 on both sides, same (tp, pp)
     pa32, pb32 = B.Plan(pa.tp, pa.pp, B.FP32), B.Plan(pb.tp, pb.pp, B.FP32)
     st32 = I.Stage(st.name, st.shape, st.seed, (pa.tp, pa.pp, "fp32"), (pb.tp, pb.pp, "fp32"))
@@ -126,9 +126,10 @@ def test_8b_state_with_adam_full_size():
         s = srcs[ns * (1 + k):ns * (2 + k)]
         d = dsts[nd * (1 + k):nd * (2 + k)]
         F._check_stage_sums(st32, d32, s, d, pa32, pb32, "fp32", "fp32")
-        F._check_stage_sampled(st32, s, d, st32.src, st32.dst, [1, 2, 5, 9, 9 * 32 + 1])
+        jobs.append(F.oracle_job(st32, s, [d]))
     rd, wr = t.bytes()
     assert rd == wr == 5 * (8_030_261_248 * 2 + 65 * 8192 * 3)       # theta bf16 + two fp32 moments = 5x
+    assert G.compare_every_tensor(jobs) == wr                         # every tensor of theta and of both moments
     del srcs, dsts, s, d
     torch.cuda.empty_cache()
 
@@ -179,40 +180,15 @@ def test_layout_variants_on_the_gpu(la, lb, variant):
 
 def test_8b_trainer_layout_to_generation_layout_full_size():
     """fp32 weights in a trainer's layout (grouped QKV, interleaved gate/up, TP2PP2) to blocked bf16 TP4PP1:
-    every fused block of the first and last layer and the sums of all tensors against the oracle."""
+    every tensor against the oracle, and the sums of all stored tensors."""
     name = "8b_grouped_fp32_tp2pp2_to_blocked_bf16_tp4pp1"
     wl, t, srcs, dsts, descs = _run(name)
     st = wl.stages[0]
     desc, pa, pb = descs[0]
     F._check_stage_sums(st, desc, srcs, dsts, pa, pb, "fp32", "bf16")
-    # oracle on whole fused blocks (qkv = stored id 1+6l+1, gate_up = 1+6l+4) of two layers, plus wo / wdown
-    sh = st.shape
-    m = O.Model(sh.layers, sh.hidden, sh.heads, sh.kv_heads, sh.ffn, sh.vocab, O.FP32, False)
-    opa, opb = O.Plan(2, 2, 0, 3), O.Plan(4, 1, O.BF16, 0)
-    for l in (0, 31):
-        for tids, sid in (((1 + 9 * l + 1, 1 + 9 * l + 2, 1 + 9 * l + 3), 1 + 6 * l + 1),
-                          ((1 + 9 * l + 6, 1 + 9 * l + 7), 1 + 6 * l + 4)):
-            # host copies of the fused block of every shard that holds it
-            sblk, dblk, dwant = {}, {}, {}
-            for s in range(4):
-                off, rows, cols, _ = desc.tensor_slice(pa, s, sid)
-                if rows:
-                    sblk[s] = (off, srcs[s][off:off + rows * cols * 4].cpu().numpy())
-            for d in range(4):
-                off, rows, cols, _ = desc.tensor_slice(pb, d, sid)
-                dblk[d] = (off, dsts[d][off:off + rows * cols * 2].cpu().numpy())
-                dwant[d] = np.zeros(rows * cols * 2, np.uint8)
-            for tid in tids:
-                sparts, dparts = [], []
-                for s in range(4):
-                    p = O.locate(m, opa, s, tid)
-                    sparts.append(sblk[s][1][p.offset - sblk[s][0]:] if p.held else None)
-                for d in range(4):
-                    p = O.locate(m, opb, d, tid)
-                    dparts.append(dwant[d][p.offset - dblk[d][0]:])
-                O.reshard_tensor_parts(m, opa, opb, tid, sparts, dparts)
-            for d in range(4):
-                assert np.array_equal(dblk[d][1], dwant[d]), (l, sid, d)
+    # every tensor through the oracle; under the grouped and interleaved layouts a part's rows are interleaved
+    # with other tensors' rows, which the comparison handles by the span of each part
+    G.compare_every_tensor([F.oracle_job(st, srcs, [dsts])])
     del srcs, dsts
     torch.cuda.empty_cache()
 
@@ -259,8 +235,10 @@ def test_8b_dag_full_size():
     desc = extra[1][0]
     F._check_stage_sums(st, desc, srcs, dsts[32:], B.Plan(4, 8), B.Plan(8, 2), "bf16", "bf16")
     F._check_stage_sums(st, desc, srcs, dsts[:8], B.Plan(4, 8), B.Plan(4, 2), "bf16", "bf16")
-    F._check_stage_sampled(st, srcs, dsts[32:], (4, 8, "bf16"), (8, 2, "bf16"),
-                           list(range(1, 10)) + [0, 9 * 32 + 1, 9 * 32 + 2, 9 * 31 + 5, 9 * 31 + 9])
+    # every tensor through the oracle: the first replica against (TP4,PP8)->(TP4,PP2) (the other three equal it,
+    # checked above), the target against the direct (TP4,PP8)->(TP8,PP2)
+    G.compare_every_tensor([F.oracle_job(st, srcs, [dsts[:8]], (4, 8, "bf16"), (4, 2, "bf16")),
+                            F.oracle_job(st, srcs, [dsts[32:]], (4, 8, "bf16"), (8, 2, "bf16"))])
     del srcs, dsts
     torch.cuda.empty_cache()
 
@@ -291,7 +269,7 @@ def test_8b_tp16_beyond_the_kv_heads_full_size():
     wl, t, srcs, dsts, descs = _run("8b_tp4pp1_to_tp16pp1")
     st = wl.stages[0]
     desc, pa, pb = descs[0]
-    F._check_stage_sampled(st, srcs, dsts, st.src, st.dst, list(range(1, 10)) + [0, 9 * 32 + 1, 9 * 32 + 2, 9 * 17 + 3])
+    G.compare_every_tensor([F.oracle_job(st, srcs, [dsts])])          # every tensor through the oracle
     # kv heads: ranks 2g and 2g+1 hold the same K and V rows of every layer
     for tid in (1 + 6 * 0 + 1, 1 + 6 * 31 + 1):
         off, rows, cols, _ = desc.tensor_slice(pb, 0, tid)

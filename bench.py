@@ -4,7 +4,8 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
 
 A step is one pass of the whole hot path (table walk: claim, copy / cast, finish) over one workload, by
-default the 8B Split TP1PP1 -> TP4PP2 the metric is quoted on.  Inputs are seeded synthetic N(0, 0.02)
+default the 8B Split TP1PP1 -> TP4PP2 the metric is quoted on; at N = 1 the default run then measures the other
+configurations one after the other in the same process and appends them as `workloads` to the one JSON line.  Inputs are seeded synthetic N(0, 0.02)
 weights, resident in HBM before the timed region; the working set (>= 32 GB) is far larger than L2, so no
 flush is needed between iterations.  With N > 1 (torchrun) every rank runs an independent replica of the
 workload on its own GPU (the path has no exchange step: replicas only), and the value is the sum over
@@ -48,7 +49,12 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--e2e-steps", type=int, default=2)
-    ap.add_argument("--cpu-layers", type=int, default=16, help="layers in the CPU-oracle sample (about 1 s each)")
+    ap.add_argument("--cpu-layers", type=int, default=12,
+                    help="layers in the CPU-oracle sample, next to embedding and head (about 1 s each on one core)")
+    ap.add_argument("--others", default="all", choices=["all", "configs", "none"],
+                    help="workloads measured after the headline in the same run (N = 1 only): the other BASELINE "
+                         "configs, or those and the k-unit / optimizer-state / layout / DAG workloads, or none")
+    ap.add_argument("--other-steps", type=int, default=10)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--tile-bytes", type=int, default=0)
@@ -129,12 +135,44 @@ class ClockSampler:
 
 # ------------------------------------------------------------------------------------------------ workload
 
-def build_workload(name, device, tune):
-    """Compiles the workload's transition(s) and allocates seeded sources and sentinel destinations."""
+class DoesNotFit(RuntimeError):
+    pass
+
+
+def workload_device_bytes(name) -> int:
+    """Device memory the workload's shard buffers take (host work only: layouts and compiled tables)."""
     from paper_2609_34645_b200 import binding as B
     from paper_2609_34645_b200 import inputs as I
 
     wl = I.WORKLOADS[name]
+    if wl.dag:
+        dag, descs = _plan_dag(wl)
+        t = dag.lower(descs)
+        ns, nd = t.num_buffers()
+        return sum(t.buffer_bytes(False, i) for i in range(ns)) + sum(t.buffer_bytes(True, j) for j in range(nd))
+    tot = 0
+    for st in wl.stages:
+        sh = st.shape
+        d = B.ModelDesc(sh.layers, sh.hidden, sh.heads, sh.kv_heads, sh.ffn, sh.vocab, B.DTYPES[st.src[2]], st.value_head)
+        for plan, k in ((st.src, 1), (st.dst, st.replicas)):
+            tot += k * sum(d.shard_sizes(B.Plan(plan[0], plan[1], B.DTYPES[plan[2]], I.layout_of(plan))))
+            tot += st.n_opt * sum(d.shard_sizes(B.Plan(plan[0], plan[1], B.FP32, I.layout_of(plan))))
+    return tot                                  # a round trip lands in the sources: nothing more
+
+
+def build_workload(name, device, tune, check_fit=False):
+    """Compiles the workload's transition(s) and allocates seeded sources and sentinel destinations.
+    check_fit: raise DoesNotFit instead of allocating when cudaMemGetInfo says the buffers do not fit."""
+    import torch
+    from paper_2609_34645_b200 import binding as B
+    from paper_2609_34645_b200 import inputs as I
+
+    wl = I.WORKLOADS[name]
+    if check_fit:
+        torch.cuda.empty_cache()
+        need, (free, _) = workload_device_bytes(name), torch.cuda.mem_get_info(device)
+        if need * 1.01 + (1 << 30) > free:
+            raise DoesNotFit(f"needs {need / 1e9:.1f} GB of device memory, {free / 1e9:.1f} GB free")
     parts, descs, srcs, dsts, keep = [], [], [], [], []
     if wl.dag:
         return build_dag_workload(wl, device, tune)
@@ -191,10 +229,8 @@ def build_workload(name, device, tune):
     return wl, t, srcs, dsts, (parts, keep, descs)
 
 
-def build_dag_workload(wl, device, tune):
-    """A plan change planned as a DAG of EMU primitives and lowered to one task table."""
+def _plan_dag(wl):
     from paper_2609_34645_b200 import binding as B
-    from paper_2609_34645_b200 import inputs as I
 
     dag, descs = B.Dag(), []
     for st, (kind, current, target) in zip(wl.stages, wl.dag):
@@ -208,6 +244,15 @@ def build_dag_workload(wl, device, tune):
             for tp, pp, first in coll:
                 dag.add_unit(m, is_target, tp, pp, list(range(first, first + tp * pp)))
     dag.plan(0)
+    return dag, descs
+
+
+def build_dag_workload(wl, device, tune):
+    """A plan change planned as a DAG of EMU primitives and lowered to one task table."""
+    from paper_2609_34645_b200 import binding as B
+    from paper_2609_34645_b200 import inputs as I
+
+    dag, descs = _plan_dag(wl)
     t = dag.lower(descs)
     units, prims = dag.units(), dag.prims()
     created = {u for p in prims for u in p["dst"]}
@@ -237,11 +282,14 @@ def build_dag_workload(wl, device, tune):
 
 # ------------------------------------------------------------------------------------------------ CPU oracle leg
 
-def oracle_sample(workload_name, layers, device_srcs=None):
-    """Times the oracle, as it stands, on the tensors of the first `layers` layers of the workload's first
-    stage (gather -> cast -> slice per logical tensor).  Returns (GB/s on algorithmic bytes, seconds, desc)."""
+def oracle_sample(workload_name, layers, device_srcs=None, with_ends=False, workers=1):
+    """Times the oracle, as it stands, on the logical tensors of the first `layers` layers of the workload's
+    first stage (gather -> cast -> slice per logical tensor), with_ends also on the embedding, the final norm
+    and the head.  workers = 1: one tensor after the other on one core, the oracle as defined.  workers > 1: the
+    same single-threaded routine over disjoint tensors on a pool of host threads (ctypes releases the
+    interpreter lock), wall-clock over the whole pool.  Returns (GB/s on algorithmic bytes, seconds, what)."""
     import numpy as np
-    import torch
+    from concurrent.futures import ThreadPoolExecutor
     from oracle import oracle as O
     from paper_2609_34645_b200 import inputs as I
 
@@ -253,8 +301,11 @@ def oracle_sample(workload_name, layers, device_srcs=None):
     pb = O.Plan(st.dst[0], st.dst[1], odt[st.dst[2]], I.layout_of(st.dst))
     layers = max(1, min(layers, sh.layers))
     ses, des = I.element_size(st.src[2]), I.element_size(st.dst[2])
-    total_s, total_bytes = 0.0, 0
-    for tid in range(1, 1 + 9 * layers):
+    ids = list(range(1, 1 + 9 * layers))
+    if with_ends:
+        ids = [0] + ids + [9 * sh.layers + 1, 9 * sh.layers + 2]
+    jobs, total_bytes = [], 0
+    for tid in ids:
         src_parts, dst_parts = [], []
         for s in range(O.num_shards(m, pa)):
             p = O.locate(m, pa, s, tid)
@@ -277,12 +328,38 @@ def oracle_sample(workload_name, layers, device_srcs=None):
             dst_parts.append(np.empty(p.nr * p.nc * des, np.uint8) if p.held else None)
             if p.held:
                 total_bytes += p.nr * p.nc * (ses + des)
-        t0 = time.perf_counter()
-        O.reshard_tensor_parts(m, pa, pb, tid, src_parts, dst_parts)
-        total_s += time.perf_counter() - t0
-    what = f"oracle on the {9 * layers} logical tensors of layers 0..{layers - 1} of stage '{st.name}' " \
-           f"({total_bytes / 1e9:.2f} GB read+written of the workload)"
+        jobs.append((tid, src_parts, dst_parts))
+    t0 = time.perf_counter()
+    if workers <= 1:
+        for tid, sp, dp in jobs:
+            O.reshard_tensor_parts(m, pa, pb, tid, sp, dp)
+    else:
+        jobs.sort(key=lambda j: -sum(x.size for x in j[2] if x is not None))
+        with ThreadPoolExecutor(max_workers=workers) as pool:
+            list(pool.map(lambda j: O.reshard_tensor_parts(m, pa, pb, j[0], j[1], j[2]), jobs))
+    total_s = time.perf_counter() - t0
+    ends = "embedding, final norm, head and " if with_ends else ""
+    what = f"oracle on {len(ids)} logical tensors ({ends}layers 0..{layers - 1}) of stage '{st.name}': " \
+           f"{total_bytes / 1e9:.2f} GB read+written of the workload's {_algorithmic_gb(workload_name):.2f} GB"
     return total_bytes / total_s / 1e9, total_s, what
+
+
+def _algorithmic_gb(workload_name):
+    from paper_2609_34645_b200 import binding as B
+    from paper_2609_34645_b200 import inputs as I
+    st = I.WORKLOADS[workload_name].stages[0]
+    sh = st.shape
+    d = B.ModelDesc(sh.layers, sh.hidden, sh.heads, sh.kv_heads, sh.ffn, sh.vocab, B.DTYPES[st.src[2]], st.value_head)
+    t = d.compile(B.Plan(st.src[0], st.src[1], B.DTYPES[st.src[2]], I.layout_of(st.src)),
+                  B.Plan(st.dst[0], st.dst[1], B.DTYPES[st.dst[2]], I.layout_of(st.dst)))
+    return sum(t.bytes()) / 1e9
+
+
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
 
 
 def run_reference(args):
@@ -421,15 +498,101 @@ def run_ours(args):
         try:
             from oracle import oracle as O
             O.build()
-            v, s, what = oracle_sample(args.workload, args.cpu_layers, srcs)
+            v, s, what = oracle_sample(args.workload, args.cpu_layers, srcs, with_ends=True)
             line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": what,
                                     "seconds": s}
+            cores = host_cores()
+            v, s, what = oracle_sample(args.workload, args.cpu_layers, srcs, with_ends=True, workers=cores)
+            line["cpu_baseline_all_cores"] = {
+                "value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "seconds": s,
+                "sample": what + f"; the same single-threaded routine over disjoint tensors on {cores} host threads"}
         except Exception as e:      # the baseline is a report, never a dependency of the GPU number
             line["cpu_baseline"] = {"value": None, "unit": UNIT, "cores": 1, "kind": "oracle",
                                     "sample": f"failed: {e!r}"}
+    if world == 1 and args.others != "none" and args.workload == DEFAULT_WORKLOAD:
+        del srcs, dsts, sp, dp, t, keep, wl
+        line["workloads"] = measure_others(args, device, gpu_id, peak, peak_kind)
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+OTHER_CONFIGS = ["tiny_tp2pp1_to_tp1pp1", "8b_tp4pp2_to_tp1pp1", "8b_fp32_tp2pp2_to_bf16_tp4pp1", "ppo5_8b",
+                 "32b_tp2pp4_to_tp8pp1_and_back"]
+OTHER_NEXT = ["8b_extend_tp4pp2_x2", "8b_fp32_tp2pp2_to_bf16_tp4pp1_x2", "8b_state_adam_tp2pp2_to_tp4pp1",
+              "8b_grouped_fp32_tp2pp2_to_blocked_bf16_tp4pp1", "8b_tp4pp1_to_tp16pp1", "8b_dag_tp4pp8_to_tp8pp2"]
+L2_BYTES = 126 << 20
+
+
+def measure_others(args, device, gpu_id, peak, peak_kind):
+    """The other configurations, one after the other in this process, each on freshly allocated buffers: kernel
+    time per launch by CUDA events on the launching stream, clocks sampled during each timed region.  Workloads
+    smaller than L2 get L2 flushed between iterations (256 MiB written, then 256 MiB read, so that no dirty
+    lines are left to be written back during the timed launch); a workload that does not fit is skipped with
+    the reason."""
+    import gc
+    import torch
+    from paper_2609_34645_b200 import binding as B
+
+    out = []
+    tune = dict(tile_bytes=0, ctas_per_sm=0, threads=0, variant=0)
+    stream = torch.cuda.current_stream()
+    for name in OTHER_CONFIGS + (OTHER_NEXT if args.others == "all" else []):
+        gc.collect()
+        torch.cuda.empty_cache()
+        t0 = time.perf_counter()
+        try:
+            wl, t, srcs, dsts, keep = build_workload(name, device, tune, check_fit=True)
+        except DoesNotFit as e:
+            out.append({"workload": name, "skipped": str(e)})
+            continue
+        rd, wr = t.bytes()
+        sp = B.Transition.pointer_array([b.data_ptr() for b in srcs])
+        dp = B.Transition.pointer_array([b.data_ptr() for b in dsts])
+        small = rd + wr < 4 * L2_BYTES
+        steps = 2000 if small else max(3, args.other_steps)        # long enough for the clock sampler to see it
+        flush = (torch.empty(256 << 20, dtype=torch.uint8, device=device),
+                 torch.ones(256 << 20, dtype=torch.uint8, device=device)) if small else None
+        for _ in range(3):
+            t.run(sp, dp, stream.cuda_stream)
+        torch.cuda.synchronize()
+        build_s = time.perf_counter() - t0
+        sampler = ClockSampler(gpu_id)
+        sampler.start()
+        timed = min(steps, 200)                                     # event pairs kept for the per-launch time
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(timed)]
+        torch.cuda.synchronize()
+        launches0 = t.launches()
+        for k in range(steps):
+            if flush:
+                flush[0].fill_(k & 127)
+                flush[1].sum()
+            if k < timed:
+                ev[k][0].record(stream)
+            t.run(sp, dp, stream.cuda_stream)
+            if k < timed:
+                ev[k][1].record(stream)
+        torch.cuda.synchronize()
+        clocks = sampler.stop()
+        per = [a.elapsed_time(b) for a, b in ev]
+        kernel_ms = statistics.mean(per)
+        n_trans = t.num_tiles()[1] if wl.dag else len(wl.stages) * (2 if wl.round_trip else 1)
+        achieved = (rd + wr) / 1e9 / (kernel_ms / 1e3)
+        ok = t.status() == B.DEV_OK
+        out.append({
+            "workload": name, "ms_per_step": kernel_ms, "ms_min": min(per), "value": achieved, "unit": UNIT,
+            "ms_per_transition": kernel_ms / n_trans, "transitions_per_step": n_trans,
+            "frac_of_nominal_8TBps": achieved / NOMINAL_HBM_GBS,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "frac": achieved / peak,
+                         "peak_kind": f"of {peak_kind}"},
+            "kernel": t.launch_info()["kernel"], "launch": t.launch_info(), "tiles": t.num_tiles()[0],
+            "levels": t.num_tiles()[1], "bytes_read": rd, "bytes_written": wr, "steps": steps,
+            "gpu_launches": t.launches() - launches0, "device_status_ok": ok,
+            "l2": "flushed between iterations: 256 MiB written, then 256 MiB read" if small
+                  else "inputs larger than L2, no flush",
+            "clocks": clocks, "build_s": round(build_s, 1)})
+        del srcs, dsts, sp, dp, t, keep, wl, flush
+    return out
 
 
 def host_memory_budget() -> int:

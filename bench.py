@@ -55,6 +55,8 @@ def parse_args():
                     help="workloads measured after the headline in the same run (N = 1 only): the other BASELINE "
                          "configs, or those and the k-unit / optimizer-state / layout / DAG workloads, or none")
     ap.add_argument("--other-steps", type=int, default=10)
+    ap.add_argument("--small-steps", type=int, default=2000,
+                    help="timed iterations of a workload smaller than L2 (long enough for the clock sampler)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--tile-bytes", type=int, default=0)
@@ -550,9 +552,9 @@ def measure_others(args, device, gpu_id, peak, peak_kind):
         sp = B.Transition.pointer_array([b.data_ptr() for b in srcs])
         dp = B.Transition.pointer_array([b.data_ptr() for b in dsts])
         small = rd + wr < 4 * L2_BYTES
-        steps = 2000 if small else max(3, args.other_steps)        # long enough for the clock sampler to see it
+        steps = max(3, args.small_steps if small else args.other_steps)
         flush = (torch.empty(256 << 20, dtype=torch.uint8, device=device),
-                 torch.ones(256 << 20, dtype=torch.uint8, device=device)) if small else None
+                 torch.ones(32 << 20, dtype=torch.int64, device=device)) if small else None
         for _ in range(3):
             t.run(sp, dp, stream.cuda_stream)
         torch.cuda.synchronize()

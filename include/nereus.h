@@ -200,18 +200,26 @@ int nereus_transition_validate(nereus_transition_t t);
  * validator can be shown a corrupted table.  Errors: ARG, UNSUPPORTED (the table is already on a device). */
 int nereus_debug_set_rect(nereus_transition_t t, int index, const nereus_rect_t* task);
 
-/* Launch tuning; 0 keeps the default of a field.  tile_bytes: target bytes per claimed tile (multiple of
- * 512).  ctas_per_sm, threads: persistent grid = SMs * ctas_per_sm blocks of `threads` threads.
- * variant: 0 default (the ring for tables of 64 MiB and more, the vector kernel below), 1 register-staged
- * vector copy, 2 bulk-copy shared-memory ring.  tile_bytes 0 = 16 KiB for the vector kernel, 32 KiB per
- * ring stage (24 KiB when the table contains a cast: the stage then holds the fp32 source), halved for small
- * tables until at least every other claimer gets a tile.  A ring stage must fit four times into the shared
- * memory of an SM, else ARG at prepare.
+/* Launch tuning; 0 keeps the default of a field.  tile_bytes: target bytes per tile (multiple of 512).
+ * ctas_per_sm, threads: the persistent kernels' grid = SMs * ctas_per_sm blocks of `threads` threads; kernel 3
+ * takes `threads` only (its grid follows the tile count).
+ * variant: which kernel walks the table.
+ *   0  default: kernel 3 for single-level tables that write less than 1 GiB through at most 64 buffers;
+ *      otherwise kernel 2 for tables that write 64 MiB or more and kernel 1 below that
+ *   1  persistent register-staged vector copy: a warp per tile, tiles claimed from a cursor (16 KiB tiles,
+ *      smaller for small tables until every other warp finds work)
+ *   2  persistent bulk-copy ring through shared memory (32 KiB per stage; 24 KiB when the table contains a
+ *      cast: the stage then holds the fp32 source).  A stage must fit four times into the shared memory of
+ *      an SM, else ARG at prepare
+ *   3  one warp per tile without a loop, addresses from per-tile records (4 KiB tiles, down to 1 KiB for
+ *      tables too small to give every resident warp a tile, larger as needed to stay within 2^17 tiles);
+ *      asked for on a chained table, on more than 64 buffers or on more than 2^17 tiles it falls back to 1
  * Drops the device copy of the table (the next prepare/run uploads it again).  Errors: ARG. */
 int nereus_transition_tune(nereus_transition_t t, int tile_bytes, int ctas_per_sm, int threads, int variant);
 
 /* The launch shape the next run on the current device will use (after nereus_transition_prepare; before it,
- * what a 148-SM device would get): kernel variant (1 vector copy, 2 bulk ring), tile bytes, grid, block. */
+ * what a 148-SM device would get): the kernel that runs (1, 2 or 3 as above, after any fall-back), tile
+ * bytes, grid, block. */
 int nereus_transition_launch_info(nereus_transition_t t, int* variant, int* tile_bytes, int* grid, int* threads);
 
 /* ---- execution (the local layout change of Section 6.2) ---------------------------------------------- */

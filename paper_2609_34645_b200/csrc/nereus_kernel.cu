@@ -1,9 +1,10 @@
-// Device side of the EMU reshard for sm_100a: one persistent kernel walks the task table of a compiled
-// transition (the local layout change of Section 6.2 of the Nereus paper) and moves every rect-copy task's
-// bytes from the source shards to the destination shards, with an optional fused fp32 -> bf16
-// round-to-nearest-even cast.  Pure data movement: the bound is HBM bandwidth, there is no tensor-core work.
+// Device side of the EMU reshard for sm_100a: ONE kernel launch walks the task table of a compiled transition
+// (the local layout change of Section 6.2 of the Nereus paper) and moves every rect-copy task's bytes from the
+// source shards to the destination shards, with an optional fused fp32 -> bf16 round-to-nearest-even cast.
+// Pure data movement: the bound is HBM bandwidth, there is no tensor-core work.  Three kernels share the table
+// format and the tile bodies; the host picks one per table (resolve_launch).
 //
-// Execution model
+// nereus_walk_vec, persistent, register-staged
 //   * grid = SMs x ctas_per_sm persistent blocks; every WARP claims tiles on its own.  Its first tile is its
 //     own index in the grid (no atomic on the way to the first load); further tiles come from a global cursor:
 //     lane 0 takes the next index with one atomicAdd and broadcasts it by shuffle, and the claim of the next
@@ -14,17 +15,19 @@
 //     (tables of up to 2^17 tiles), else to its rect by binary search in the tile-prefix array and then to a
 //     row block / column block of that rect by arithmetic; every lane moves 16-byte vectors, 32 lanes x 16 B =
 //     512 B contiguous per instruction, kUnroll independent loads in flight per lane before the first store.
-//   * the last block to finish zeroes the cursor and the counters, so a launch needs no reset in front of
-//     it and can be replayed from a captured graph.
 //   * tables with several dependency levels (chained transitions): a tile of level k waits, with a poll
 //     limit, until every tile of level k-1 has completed; on giving up it records NEREUS_DEV_TIMEOUT and the
 //     warp leaves.  A warp publishes its completed tiles once per level (one fence, one atomic), not per
 //     tile.  Loads bypass L1 (ld.global.cg) so a level reads what another SM wrote before it.
-//   * second kernel, nereus_walk_ring, for large tables: one CTA per SM, a producer warp
-//     that claims tiles and issues cp.async.bulk global -> shared copies into a ring of stages, and a
-//     consumer warp that issues cp.async.bulk shared -> global stores (cast tables: fifteen consumer warps that
-//     convert from shared memory and store with plain 16-byte stores); mbarriers track both directions and
-//     every wait has an iteration limit.
+// nereus_walk_ring, persistent, for large tables: one CTA per SM, a producer warp that claims tiles and issues
+//     cp.async.bulk global -> shared copies into a ring of stages, and a consumer warp that issues
+//     cp.async.bulk shared -> global stores (tables with a cast: fifteen consumer warps that convert from
+//     shared memory and store with plain 16-byte stores); mbarriers track both directions and every wait has
+//     a deadline on the global timer and an iteration limit.
+// nereus_walk_once, not persistent, for small and medium single-level tables: one warp per tile, the tile's
+//     addresses from its record, no cursor, no shared memory.
+// In both persistent kernels the last block to finish zeroes the cursor and the counters, so a launch needs no
+// reset in front of it and can be replayed from a captured graph.
 #include <cuda_runtime.h>
 
 #include <algorithm>
@@ -933,9 +936,11 @@ static int resolve_launch(const nereus_transition_s& t, int sms, Launch& L, bool
                t.bytes_written / L.tile_bytes < claimers / 2)
             L.tile_bytes /= 2;
         if (L.variant == 3) {
-            // one batch of loads per warp (32 lanes x 8 vectors = 4 KiB), larger only to stay within the
+            // one batch of loads per warp (32 lanes x 8 vectors = 4 KiB); smaller while the table would not
+            // give every resident warp (32 per SM at 64 registers) a tile, larger only to stay within the
             // number of tiles that get per-tile records
             L.tile_bytes = 4096;
+            while (L.tile_bytes > 1024 && t.bytes_written / L.tile_bytes < (uint64_t)sms * 32) L.tile_bytes /= 2;
             while (t.bytes_written / L.tile_bytes > kDirectMaxTiles * 3ull / 4) L.tile_bytes *= 2;
         }
     }

@@ -90,8 +90,10 @@ WORKLOADS = {
         Stage("32b", DENSE_32B, 8, (2, 4, "bf16"), (8, 1, "bf16")),), round_trip=True),
 }
 
-# profiling stand-in: the 8B shape cut to 4 layers (3.85 GB each side: larger than L2, small enough for a
-# multi-pass profiler capture); same tensor classes and piece sizes as the full Split
+# Profiling stand-ins, kept for the commands quoted under profiles/ (not BASELINE configurations, never a
+# bench line): the 8B shape cut to 4 layers (3.85 GB each side: larger than L2, small enough for a multi-pass
+# profiler capture; same tensor classes and piece sizes as the full Split), and a 244 MiB table of the size
+# class that runs one warp per tile
 LLAMA_8B_4L = Shape(4, 4096, 32, 8, 14336, 128256)
 WORKLOADS["8b4l_tp1pp1_to_tp4pp2"] = Workload("8b4l_tp1pp1_to_tp4pp2", (
     Stage("8b4l", LLAMA_8B_4L, 1, (1, 1, "bf16"), (4, 2, "bf16")),))
@@ -99,6 +101,9 @@ WORKLOADS["8b4l_tp4pp2_to_tp1pp1"] = Workload("8b4l_tp4pp2_to_tp1pp1", (
     Stage("8b4l", LLAMA_8B_4L, 1, (4, 2, "bf16"), (1, 1, "bf16")),))
 WORKLOADS["8b4l_fp32_tp2pp2_to_bf16_tp4pp1"] = Workload("8b4l_fp32_tp2pp2_to_bf16_tp4pp1", (
     Stage("8b4l_master", LLAMA_8B_4L, 2, (2, 2, "fp32"), (4, 1, "bf16")),))
+MID_244MIB = Shape(2, 2048, 16, 8, 5632, 8192)
+WORKLOADS["mid244_tp1pp1_to_tp4pp1"] = Workload("mid244_tp1pp1_to_tp4pp1", (
+    Stage("mid244", MID_244MIB, 1, (1, 1, "bf16"), (4, 1, "bf16")),))
 
 # the next rows: k destination units (Extend / replica units) and the EMU's optimizer state
 WORKLOADS["8b_extend_tp4pp2_x2"] = Workload("8b_extend_tp4pp2_x2", (

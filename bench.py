@@ -593,6 +593,9 @@ def measure_others(args, device, gpu_id, peak, peak_kind):
             "l2": "flushed between iterations: 256 MiB written, then 256 MiB read" if small
                   else "inputs larger than L2, no flush",
             "clocks": clocks, "build_s": round(build_s, 1)})
+        alone = time_stages_alone(wl, keep, srcs, dsts, stream)
+        if alone:
+            out[-1]["ms_per_stage_alone"] = alone        # every model-stage's transition launched on its own
         del srcs, dsts, sp, dp, t, keep, wl, flush
     return out
 

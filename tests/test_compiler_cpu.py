@@ -427,6 +427,38 @@ def test_state_with_optimizer_tensors():
     assert rd == wr == theta * (1 + 2 * 2)            # fp32 moments are twice the bf16 parameters, each
 
 
+def test_launch_shapes_without_a_device():
+    """launch_info before prepare answers for a 148-SM device: the default kernel by table, and forced kernels on
+    tables they were not made for (a tiny cast table through the ring: the halved default tile must stay a
+    multiple of 512 bytes)."""
+    d32 = desc_of(I.Shape(1, 64, 4, 2, 64, 64), B.FP32)
+    t = d32.compile(B.Plan(2, 1), B.Plan(1, 1, B.BF16))
+    assert t.launch_info()["kernel"] == "nereus_walk_once" and t.launch_info()["tile_bytes"] == 1024
+    t.tune(variant=2)
+    li = t.launch_info()
+    assert li["kernel"] == "nereus_walk_ring" and li["tile_bytes"] % 512 == 0 and li["tile_bytes"] >= 1024
+    assert li["threads"] == 512 and li["grid"] == 148             # the converting ring: 1 + 15 warps, one CTA per SM
+    t.tune(variant=1)
+    assert t.launch_info()["kernel"] == "nereus_walk_vec" and t.launch_info()["tile_bytes"] % 512 == 0
+    big = desc_of(I.LLAMA_8B).compile(B.Plan(1, 1), B.Plan(4, 2))
+    li = big.launch_info()
+    assert (li["kernel"], li["tile_bytes"], li["grid"], li["threads"]) == ("nereus_walk_ring", 32768, 148, 64)
+    assert big.num_tiles() == (506756, 1)
+    mid = desc_of(I.Shape(2, 2048, 16, 8, 5632, 8192)).compile(B.Plan(1, 1), B.Plan(4, 1))
+    li = mid.launch_info()
+    assert li["kernel"] == "nereus_walk_once" and li["tile_bytes"] == 4096
+    assert li["grid"] == -(-mid.num_tiles()[0] // 8) and li["threads"] == 256
+    mid.tune(variant=3, tile_bytes=512)                           # more tiles than get per-tile records
+    assert mid.launch_info()["kernel"] == "nereus_walk_vec"
+    ch = B.Transition.fuse([desc_of(I.TINY).compile(B.Plan(2, 1), B.Plan(1, 1)),
+                            desc_of(I.TINY).compile(B.Plan(1, 1), B.Plan(2, 1))], chained=True)
+    assert ch.launch_info()["kernel"] == "nereus_walk_vec"
+    for bad in (dict(variant=4), dict(tile_bytes=700), dict(threads=100), dict(ctas_per_sm=3)):
+        with pytest.raises(B.NereusError) as e:
+            ch.tune(**bad)
+        assert e.value.code == B.ERR_ARG
+
+
 def test_buffer_limit_of_one_launch():
     """One launch addresses at most 448 buffers (its parameter block): a fused table at the limit compiles, one
     beyond it is refused; so is a single transition with more shards than that."""

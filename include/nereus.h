@@ -188,6 +188,11 @@ int nereus_transition_num_rects(nereus_transition_t t, int* n);
 int nereus_transition_get_rect(nereus_transition_t t, int index, nereus_rect_t* out);
 /* Tiles one run claims, and dependency levels. */
 int nereus_transition_num_tiles(nereus_transition_t t, uint64_t* tiles, int* levels);
+/* Tiles [first, first + count) of the tiling one run walks, in claim order, each as the task it amounts to
+ * (`rows` pieces of `width_bytes_dst` bytes at its own offsets): what a claimer of tile g moves.  These are
+ * the per-tile records that tables of up to 2^17 tiles carry to the device.  `out` (host) holds `count`
+ * entries.  For inspection and tests.  Errors: ARG (range), TOO_LARGE (more than 2^24 tiles), NOMEM. */
+int nereus_transition_get_tiles(nereus_transition_t t, uint64_t first, uint64_t count, nereus_rect_t* out);
 /* Checks the task table on the host, as nereus_transition_prepare and nereus_transition_run_static do before
  * anything reaches a device (Section 6.2, "Safe concurrent execution": a buffer is only read or written inside
  * its declared extent and nothing writes where another task of the same step writes): every task lies inside

@@ -107,6 +107,7 @@ _SIGS = {
     "nereus_transition_num_rects": [_vp, _P(_i)],
     "nereus_transition_get_rect": [_vp, _i, _P(Rect)],
     "nereus_transition_num_tiles": [_vp, _P(ctypes.c_uint64), _P(_i)],
+    "nereus_transition_get_tiles": [_vp, ctypes.c_uint64, ctypes.c_uint64, _P(Rect)],
     "nereus_transition_tune": [_vp, _i, _i, _i, _i],
     "nereus_transition_prepare": [_vp],
     "nereus_transition_launch_info": [_vp, _P(_i), _P(_i), _P(_i), _P(_i)],
@@ -276,6 +277,14 @@ class Transition:
         t, l = ctypes.c_uint64(), _i()
         _ck(_lib.nereus_transition_num_tiles(self._h, ctypes.byref(t), ctypes.byref(l)), "nereus_transition_num_tiles")
         return t.value, l.value
+
+    def tiles(self, first=0, count=None) -> list:
+        """The tiling one run walks, each tile as the task it amounts to (nereus_transition_get_tiles)."""
+        if count is None:
+            count = self.num_tiles()[0] - first
+        arr = (Rect * max(1, count))()
+        _ck(_lib.nereus_transition_get_tiles(self._h, first, count, arr), "nereus_transition_get_tiles")
+        return list(arr[:count])
 
     def tune(self, tile_bytes=0, ctas_per_sm=0, threads=0, variant=0):
         _ck(_lib.nereus_transition_tune(self._h, tile_bytes, ctas_per_sm, threads, variant), "nereus_transition_tune")

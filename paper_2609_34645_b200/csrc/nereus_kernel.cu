@@ -1158,6 +1158,37 @@ int nereus_transition_num_tiles(nereus_transition_t t, uint64_t* tiles, int* lev
     } catch (const std::bad_alloc&) { return NEREUS_ERR_NOMEM; }
 }
 
+int nereus_transition_get_tiles(nereus_transition_t t, uint64_t first, uint64_t count, nereus_rect_t* out) {
+    try {
+        if (!t || !out) return NEREUS_ERR_ARG;
+        // the tiling of the prepared table, else what a 148-SM device would get
+        std::vector<RectDev> rects(t->rects.size()); std::vector<uint32_t> prefix(t->rects.size() + 1);
+        uint32_t le[kMaxLevels];
+        Launch L;
+        uint64_t n = 0;
+        if (t->dev.rects) {
+            if (int rc = resolve_launch(*t, t->dev.sm_count, L, t->dev.variant == 3)) return rc;
+            n = tile_table_raw(*t, (uint32_t)t->dev.tile_bytes, rects.data(), prefix.data(), le);
+        } else if (int rc = plan_launch(*t, 148, true, L, rects.data(), prefix.data(), le, n)) {
+            return rc;
+        }
+        if (first > n || count > n - first) return NEREUS_ERR_ARG;
+        if (n > (1u << 24)) return NEREUS_ERR_TOO_LARGE;              // an inspection call, not for 2^32 tiles
+        std::vector<TileRec> tiles(n);
+        expand_tiles(rects.data(), rects.size(), tiles.data());
+        for (uint64_t k = 0; k < count; ++k) {
+            const TileRec& e = tiles[first + k];
+            nereus_rect_t& o = out[k];
+            o.src_buf = e.src_buf; o.dst_buf = e.dst_buf; o.level = e.level; o.cast = e.cast;
+            o.src_off = e.src_off; o.dst_off = e.dst_off;
+            o.src_pitch = e.src_pitch; o.dst_pitch = e.dst_pitch;
+            o.rows = e.rows; o.width_bytes_dst = e.width; o.width_bytes_src = (uint64_t)e.width << e.cast;
+            o.replicas = e.replicas; o.replica_stride = e.replica_stride;
+        }
+        return NEREUS_OK;
+    } catch (const std::bad_alloc&) { return NEREUS_ERR_NOMEM; }
+}
+
 int nereus_transition_launch_info(nereus_transition_t t, int* variant, int* tile_bytes, int* grid, int* threads) {
     try {
         if (!t || !variant || !tile_bytes || !grid || !threads) return NEREUS_ERR_ARG;

@@ -317,6 +317,54 @@ def test_tiles_cover_tasks():
         t.tune(tile_bytes=1000)
 
 
+@pytest.mark.parametrize("kind", ["split", "merge_cast", "layouts_replicated", "chained"])
+@pytest.mark.parametrize("tune", [dict(), dict(tile_bytes=512), dict(tile_bytes=1536, variant=1),
+                                  dict(tile_bytes=4096, variant=2), dict(tile_bytes=65536, variant=3)])
+def test_tiles_executed_one_by_one_equal_the_oracle(kind, tune):
+    """What the kernels walk: every tile of the tiling, executed on host bytes as the small task it amounts to,
+    in claim order.  The result must equal the oracle's, every payload byte written exactly once, and the tiles
+    must be the tasks cut up (same buffers, level, cast; levels in order)."""
+    sh = I.SMALL
+    if kind == "split":
+        d, m = desc_of(sh), omodel_of(sh)
+        oa, ob, k = O.Plan(1, 1), O.Plan(4, 2), 1
+        t = d.compile(B.Plan(1, 1), B.Plan(4, 2))
+    elif kind == "merge_cast":
+        d, m = desc_of(sh, B.FP32), omodel_of(sh, O.FP32)
+        oa, ob, k = O.Plan(4, 2), O.Plan(2, 1, O.BF16), 1
+        t = d.compile(B.Plan(4, 2), B.Plan(2, 1, B.BF16))
+    elif kind == "layouts_replicated":
+        d, m = desc_of(sh), omodel_of(sh)
+        oa, ob, k = O.Plan(2, 2, 0, 3), O.Plan(4, 1, 0, 0), 2
+        t = d.compile_replicated(B.Plan(2, 2, 0, 3), B.Plan(4, 1, 0, 0), 2)
+    else:
+        d, m = desc_of(sh), omodel_of(sh)
+        oa, ob, k = O.Plan(2, 2), O.Plan(4, 1), 1
+        t = B.Transition.fuse([d.compile(B.Plan(2, 2), B.Plan(4, 1)), d.compile(B.Plan(4, 1), B.Plan(2, 2))], chained=True)
+    t.tune(**tune)
+    src = random_src(m, oa, 17, "fp32" if kind == "merge_cast" else "bf16")
+    n_src, n_dst = t.num_buffers()
+    got = [np.full(t.buffer_bytes(True, j), 0xA5, np.uint8) for j in range(n_dst)]
+    counts = [np.zeros(g.size, np.uint8) for g in got]
+    tiles = t.tiles()
+    assert len(tiles) == t.num_tiles()[0]
+    assert [x.level for x in tiles] == sorted(x.level for x in tiles)
+    assert sum(x.rows * x.width_bytes_dst * x.replicas for x in tiles) == t.bytes()[1]
+    tile_bytes = t.launch_info()["tile_bytes"]
+    assert all(x.rows * x.width_bytes_dst <= max(tile_bytes, x.width_bytes_dst) for x in tiles)
+    assert t.tiles(3, 2)[0].dst_off == tiles[3].dst_off and len(t.tiles(len(tiles), 0)) == 0
+    interpret(tiles, src, got, counts)
+    want = O.reshard_replicated(m, oa, ob, k, src, fill=0xA5)
+    for g, w in zip(got, want):
+        assert np.array_equal(g, w)
+    if kind == "chained":
+        for mk, g, s_ in zip(payload_mask(m, oa), got[4:], src):
+            assert np.array_equal(g[mk], s_[mk])
+    m_dst = omodel_of(sh, O.BF16) if kind == "merge_cast" else m
+    for j, mask in enumerate(payload_mask(m_dst, O.Plan(ob.tp, ob.pp)) * k):
+        assert np.array_equal(counts[j] == 1, mask), "every payload byte written exactly once, padding never"
+
+
 # ---------------------------------------------------------------- fuse
 
 def test_fuse_independent_and_chained():

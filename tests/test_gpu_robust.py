@@ -11,7 +11,7 @@ from paper_2609_34645_b200 import inputs as I
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("variant,chained", [(1, False), (2, False), (1, True), (2, True)])
+@pytest.mark.parametrize("variant,chained", [(1, False), (2, False), (3, False), (1, True), (2, True)])
 def test_captured_run_replays_with_new_sources(variant, chained):
     """One run captured with cudaStreamBeginCapture and replayed three times, the sources refilled before each
     replay: every replay must move the new contents (the kernel leaves its control words zeroed for the next

@@ -101,6 +101,13 @@ WORKLOADS["8b4l_tp4pp2_to_tp1pp1"] = Workload("8b4l_tp4pp2_to_tp1pp1", (
     Stage("8b4l", LLAMA_8B_4L, 1, (4, 2, "bf16"), (1, 1, "bf16")),))
 WORKLOADS["8b4l_fp32_tp2pp2_to_bf16_tp4pp1"] = Workload("8b4l_fp32_tp2pp2_to_bf16_tp4pp1", (
     Stage("8b4l_master", LLAMA_8B_4L, 2, (2, 2, "fp32"), (4, 1, "bf16")),))
+# ... and the 8B layer shape with 2 layers and a 32K vocabulary (1.41 GB per side in bf16): what multi-pass
+# captures run on, a few GB on the device in all; the per-layer tensor classes and piece sizes are the 8B model's
+LLAMA_8B_2L_V32K = Shape(2, 4096, 32, 8, 14336, 32768)
+WORKLOADS["8b2l_tp1pp1_to_tp4pp2"] = Workload("8b2l_tp1pp1_to_tp4pp2", (
+    Stage("8b2l", LLAMA_8B_2L_V32K, 1, (1, 1, "bf16"), (4, 2, "bf16")),))
+WORKLOADS["8b2l_fp32_tp2pp2_to_bf16_tp4pp1"] = Workload("8b2l_fp32_tp2pp2_to_bf16_tp4pp1", (
+    Stage("8b2l_master", LLAMA_8B_2L_V32K, 2, (2, 2, "fp32"), (4, 1, "bf16")),))
 MID_244MIB = Shape(2, 2048, 16, 8, 5632, 8192)
 WORKLOADS["mid244_tp1pp1_to_tp4pp1"] = Workload("mid244_tp1pp1_to_tp4pp1", (
     Stage("mid244", MID_244MIB, 1, (1, 1, "bf16"), (4, 1, "bf16")),))

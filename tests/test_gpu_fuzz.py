@@ -71,3 +71,42 @@ def test_random_transitions(chunk):
         assert dst.guards_intact(), c
         ran += 1
     assert ran >= 6
+
+
+@pytest.mark.parametrize("chunk", range(3))
+def test_random_chains(chunk):
+    """Chains of two to four transitions fused into one table (one launch, dependency levels), through
+    nereus_transition_run or through the allocation-free entry point: every intermediate layout and the last one
+    against the oracle applied step by step."""
+    import torch
+    ran = 0
+    for k in range(25):
+        rng = random.Random(9000 + 100 * chunk + k)
+        sh = rng.choice([I.SMALL, I.MICRO, I.TINY])
+        chain = [rng.choice(valid_plans(sh)) for _ in range(rng.choice([2, 3, 3, 4]))]
+        d = G.desc_of(sh)
+        try:
+            parts = [d.compile(B.Plan(*a), B.Plan(*b)) for a, b in zip(chain, chain[1:])]
+        except B.NereusError as e:
+            assert e.code == B.ERR_INDIVISIBLE, chain
+            continue
+        t = B.Transition.fuse(parts, chained=True) if len(parts) > 1 else parts[0]
+        t.tune(variant=rng.choice([0, 1, 2]), tile_bytes=rng.choice([0, 512, 1024, 4096, 16384]))
+        src = G.device_sources_by_oracle(sh, O.Plan(*chain[0]), "bf16", k)
+        dst = G.Guarded([t.buffer_bytes(True, j) for j in range(t.num_buffers()[1])])
+        stream = torch.cuda.current_stream()
+        if rng.random() < 0.4 and len(t.rects()) <= B.STATIC_MAX_RECTS:
+            t.run_static([s.data_ptr() for s in src], dst.ptrs(), stream.cuda_stream)
+            stream.synchronize()
+            assert B.static_status() == B.DEV_OK
+        else:
+            G.run_transition(t, src, dst.bufs)
+        host, at, m = [s.cpu().numpy() for s in src], 0, G.omodel_of(sh)
+        for a, b in zip(chain, chain[1:]):
+            want = O.reshard(m, O.Plan(*a), O.Plan(*b), host, fill=G.SENTINEL)
+            for g, w in zip(dst.bufs[at:at + len(want)], want):
+                assert np.array_equal(g.cpu().numpy(), w), (chain, a, b)
+            at, host = at + len(want), want
+        assert dst.guards_intact(), chain
+        ran += 1
+    assert ran >= 10

@@ -249,9 +249,11 @@ int nereus_transition_prepare(nereus_transition_t t);
  * on the device. */
 int nereus_transition_run(nereus_transition_t t, const void* const* src_ptrs, void* const* dst_ptrs,
                           void* cuda_stream);
-/* Environment variables read by run(): NEREUS_TILE_BYTES, NEREUS_CTAS_PER_SM, NEREUS_THREADS, NEREUS_VARIANT
- * (defaults of the tuning fields), NEREUS_RING_PIECE, NEREUS_RING_LAG, NEREUS_RING_CLAIM (ring internals), and, for tests of the
- * failure path only, NEREUS_DEBUG_GATE_BIAS: a count added to what every dependency gate waits for, so that
+/* Environment variables read by prepare() and by every run(): NEREUS_TILE_BYTES, NEREUS_CTAS_PER_SM,
+ * NEREUS_THREADS, NEREUS_VARIANT (defaults of the tuning fields; a run whose kernel or tile size no longer is
+ * what the table was prepared with returns ARG: call nereus_transition_tune to re-prepare), NEREUS_RING_PIECE,
+ * NEREUS_RING_LAG, NEREUS_RING_CLAIM (ring internals), and, for tests of the failure path only,
+ * NEREUS_DEBUG_GATE_BIAS: a count added to what every dependency gate waits for, so that
  * the gate cannot open; the waits then run into their poll limit (about half a second), the run ends with
  * device status NEREUS_DEV_TIMEOUT and the destinations of the gated levels stay unwritten. */
 

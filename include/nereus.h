@@ -73,6 +73,7 @@ extern "C" {
 #define NEREUS_ERR_TOO_LARGE     -9   /* more tasks than the fixed scratch of nereus_transition_run_static */
 /* -10 is NEREUS_ERR_INFEASIBLE, declared with the transition DAG below */
 #define NEREUS_ERR_TABLE         -11  /* the task table failed the host-side check that precedes every upload */
+#define NEREUS_ERR_TOO_SMALL     -12  /* a buffer handed to nereus_transition_run_sized is shorter than required */
 
 /* device status word (nereus_transition_status) */
 #define NEREUS_DEV_OK             0
@@ -249,6 +250,12 @@ int nereus_transition_prepare(nereus_transition_t t);
  * on the device. */
 int nereus_transition_run(nereus_transition_t t, const void* const* src_ptrs, void* const* dst_ptrs,
                           void* cuda_stream);
+/* The same, with the lengths in bytes of the caller's buffers (host arrays, one entry per pointer): a buffer
+ * shorter than nereus_transition_buffer_bytes is refused with NEREUS_ERR_TOO_SMALL before anything is enqueued.
+ * Together with the check of the table against those required lengths (nereus_transition_validate, run by
+ * prepare) this bounds every access of the kernel by what the caller really holds.  Errors: as run, TOO_SMALL. */
+int nereus_transition_run_sized(nereus_transition_t t, const void* const* src_ptrs, const size_t* src_sizes,
+                                void* const* dst_ptrs, const size_t* dst_sizes, void* cuda_stream);
 /* Environment variables read by prepare() and by every run(): NEREUS_TILE_BYTES, NEREUS_CTAS_PER_SM,
  * NEREUS_THREADS, NEREUS_VARIANT (defaults of the tuning fields; a run whose kernel or tile size no longer is
  * what the table was prepared with returns ARG: call nereus_transition_tune to re-prepare), NEREUS_RING_PIECE,

@@ -25,6 +25,7 @@ ERR_CUDA, ERR_NOMEM, ERR_MISMATCH, ERR_ALIGN = -5, -6, -7, -8
 ERR_TOO_LARGE = -9
 ERR_INFEASIBLE = -10
 ERR_TABLE = -11
+ERR_TOO_SMALL = -12
 GENERATION, INFERENCE, TRAINING = 0, 1, 2
 OP_SPLIT, OP_DESTROY, OP_EXTEND, OP_MERGE = 0, 1, 2, 3
 STATIC_MAX_RECTS = 4096
@@ -112,6 +113,7 @@ _SIGS = {
     "nereus_transition_prepare": [_vp],
     "nereus_transition_launch_info": [_vp, _P(_i), _P(_i), _P(_i), _P(_i)],
     "nereus_transition_run": [_vp, _P(_vp), _P(_vp), _vp],
+    "nereus_transition_run_sized": [_vp, _P(_vp), _P(_sz), _P(_vp), _P(_sz), _vp],
     "nereus_transition_status": [_vp, _P(_i)],
     "nereus_transition_launches": [_vp, _P(ctypes.c_uint64)],
     "nereus_last_cuda_error": [],
@@ -326,6 +328,12 @@ class Transition:
         if not isinstance(dst_ptrs, ctypes.Array):
             dst_ptrs = self.pointer_array(dst_ptrs)
         return _lib.nereus_transition_run(self._h, src_ptrs, dst_ptrs, _vp(stream))
+
+    def run_sized_raw(self, src_ptrs, src_sizes, dst_ptrs, dst_sizes, stream=0) -> int:
+        """nereus_transition_run_sized: run() with the lengths of the caller's buffers; returns the error code."""
+        sp, dp = self.pointer_array(src_ptrs), self.pointer_array(dst_ptrs)
+        ss, ds = (_sz * len(src_sizes))(*src_sizes), (_sz * len(dst_sizes))(*dst_sizes)
+        return _lib.nereus_transition_run_sized(self._h, sp, ss, dp, ds, _vp(stream))
 
     def run_static(self, src_ptrs, dst_ptrs, stream=0):
         """nereus_transition_run_static: the same transition without any device allocation, for callers

@@ -887,6 +887,7 @@ const char* nereus_strerror(int code) {
     case NEREUS_ERR_INFEASIBLE:  return "the transition DAG cannot be scheduled: an acquisition stays blocked";
     case NEREUS_ERR_TOO_LARGE:   return "the transition has more tasks than the fixed scratch of run_static holds";
     case NEREUS_ERR_TABLE:       return "the task table failed validation: a task leaves its buffers or two tasks collide";
+    case NEREUS_ERR_TOO_SMALL:   return "a shard buffer is shorter than the transition requires";
     default:                     return "unknown error";
     }
 }

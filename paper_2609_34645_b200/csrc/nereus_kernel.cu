@@ -1246,6 +1246,17 @@ int nereus_transition_run(nereus_transition_t t, const void* const* src_ptrs, vo
     } catch (const std::bad_alloc&) { return NEREUS_ERR_NOMEM; }
 }
 
+int nereus_transition_run_sized(nereus_transition_t t, const void* const* src_ptrs, const size_t* src_sizes,
+                                void* const* dst_ptrs, const size_t* dst_sizes, void* cuda_stream) {
+    if (!t || !src_ptrs || !dst_ptrs || !src_sizes || !dst_sizes) return NEREUS_ERR_ARG;
+    // the table was checked against the sizes it declares; here the caller's buffers are checked against those
+    for (size_t i = 0; i < t->src_bytes.size(); ++i)
+        if (src_sizes[i] < t->src_bytes[i]) return NEREUS_ERR_TOO_SMALL;
+    for (size_t j = 0; j < t->dst_bytes.size(); ++j)
+        if (dst_sizes[j] < t->dst_bytes[j]) return NEREUS_ERR_TOO_SMALL;
+    return nereus_transition_run(t, src_ptrs, dst_ptrs, cuda_stream);
+}
+
 int nereus_transition_status(nereus_transition_t t, int* device_status) {
     if (!t || !device_status) return NEREUS_ERR_ARG;
     if (!t->dev.rects) { *device_status = NEREUS_DEV_OK; return NEREUS_OK; }

@@ -421,6 +421,12 @@ def test_run_rejects_bad_pointers_before_any_cuda_call():
     assert t.run_raw([src[0] + 8, src[1]], [base + (2 << 30)]) == B.ERR_ALIGN
     assert t.run_raw(src, [src[1] + sizes[1] - 256]) == B.ERR_ALIAS        # dst overlaps a source's tail
     assert t.run_raw(src, [src[0] - 16]) == B.ERR_ALIAS
+    # declared lengths: a buffer shorter than required is refused, before any CUDA call as well
+    dst, need = [base + (2 << 30)], [t.buffer_bytes(True, 0)]
+    assert t.run_sized_raw(src, [sizes[0], sizes[1] - 1], dst, need) == B.ERR_TOO_SMALL
+    assert t.run_sized_raw(src, sizes, dst, [need[0] - 256]) == B.ERR_TOO_SMALL
+    assert t.run_sized_raw([0, src[1]], sizes, dst, need) == B.ERR_ARG            # then run()'s own checks
+    assert "shorter" in B.strerror(B.ERR_TOO_SMALL)
 
 
 # ---------------------------------------------------------------- replicas (Extend) and optimizer state

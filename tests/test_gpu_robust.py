@@ -74,6 +74,24 @@ def test_corrupted_table_is_refused_before_the_upload():
     assert e.value.code == B.ERR_UNSUPPORTED
 
 
+def test_run_with_declared_lengths():
+    d = G.desc_of(I.SMALL)
+    t = d.compile(B.Plan(2, 2), B.Plan(4, 1))
+    src = G.device_sources(d, B.Plan(2, 2), "bf16", 4)
+    dst = G.Guarded([t.buffer_bytes(True, j) for j in range(4)])
+    sp, ss = [s.data_ptr() for s in src], [s.numel() for s in src]
+    assert t.run_sized_raw(sp, ss, dst.ptrs(), [n - 16 for n in dst.sizes]) == B.ERR_TOO_SMALL
+    torch.cuda.synchronize()
+    assert t.launches() == 0 and all(bool((r == G.SENTINEL).all()) for r in dst.raw)
+    assert t.run_sized_raw(sp, ss, dst.ptrs(), dst.sizes) == B.OK
+    torch.cuda.synchronize()
+    assert t.status() == B.DEV_OK
+    want = G.oracle_expected(I.SMALL, (2, 2), (4, 1), "bf16", "bf16", False, [s.cpu().numpy() for s in src])
+    for g, w in zip(dst.bufs, want):
+        assert np.array_equal(g.cpu().numpy(), w)
+    assert dst.guards_intact()
+
+
 def test_many_runs_back_to_back_need_no_reset():
     """200 launches of one handle without a synchronise in between: each finds the control words zeroed by the
     one before it."""

@@ -1339,7 +1339,7 @@ static Ctrl* static_ctrl(unsigned char* scratch) {
 }  // namespace nereus
 
 extern "C" int nereus_transition_run_static(nereus_transition_t t, const void* const* src_ptrs,
-                                            void* const* dst_ptrs, void* cuda_stream) {
+                                            void* const* dst_ptrs, void* cuda_stream) try {
     if (!t || !src_ptrs || !dst_ptrs) return NEREUS_ERR_ARG;
     const size_t n_rects = t->rects.size();
     if (n_rects > (size_t)kStaticMaxRects) return NEREUS_ERR_TOO_LARGE;
@@ -1386,6 +1386,8 @@ extern "C" int nereus_transition_run_static(nereus_transition_t t, const void* c
     if (int rc = launch_walk(L, sms, p, stream)) return rc;
     if (n_tiles > 0) t->launches += 1;
     return NEREUS_OK;
+} catch (...) {
+    return NEREUS_ERR_UNSUPPORTED;      // the lock could not be taken; nothing here allocates, so nothing else throws
 }
 
 extern "C" int nereus_static_status(int* device_status) {

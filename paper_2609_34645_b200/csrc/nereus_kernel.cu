@@ -98,10 +98,28 @@ __device__ __forceinline__ uint4 ld_stream(const char* p) { return __ldcg(reinte
 __device__ __forceinline__ void  st_stream(char* p, uint4 v) { __stcs(reinterpret_cast<uint4*>(p), v); }
 __device__ __forceinline__ void  st_stream8(char* p, uint2 v) { __stcs(reinterpret_cast<uint2*>(p), v); }
 
-// two fp32 -> packed bf16x2, round to nearest even; NaN (any payload, either sign) -> 0x7FC0
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+// two fp32 -> packed bf16x2, round to nearest even (the instruction's own rounding: ties to even, overflow to
+// +-Inf, subnormals rounded, signed zero kept).  For a NaN the instruction leaves the pattern 0x7FFF in that half,
+// which no other input produces (finite values end at 0x7F80 = Inf); the rule of this library is 0x7FC0 for
+// every NaN, so such halves are rewritten.  The test is on the packed result: (half & 0x7FFF) + 1 reaches
+// 0x8000 exactly for 0x7FFF / 0xFFFF, and the carry cannot leave its half.
+__device__ __forceinline__ uint32_t cvt_bf16x2(float lo, float hi) {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ uint32_t nan_halves(uint32_t r) { return ((r & 0x7FFF7FFFu) + 0x00010001u) & 0x80008000u; }
+__device__ __forceinline__ uint32_t fix_nan_halves(uint32_t r) {
+    const uint32_t n = nan_halves(r);
+    if (n & 0x00008000u) r = (r & 0xFFFF0000u) | 0x00007FC0u;
+    if (n & 0x80000000u) r = (r & 0x0000FFFFu) | 0x7FC00000u;
+    return r;
+}
+// The same rule without a branch, for the register-staged kernels (a data-dependent branch between their loads
+// and stores costs them up to 5%; the ring's converting warps, which are bound by instruction issue, gain 2%
+// from testing eight results at once instead).
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    uint32_t r = cvt_bf16x2(lo, hi);
     if (lo != lo) r = (r & 0xFFFF0000u) | 0x00007FC0u;
     if (hi != hi) r = (r & 0x0000FFFFu) | 0x7FC00000u;
     return r;
@@ -818,10 +836,14 @@ __device__ __forceinline__ void ring_consumer_cast(const WalkParams& p, const Ri
                 const uint4 a = *reinterpret_cast<const uint4*>(src + r * ws + c * 32);
                 const uint4 b = *reinterpret_cast<const uint4*>(src + r * ws + c * 32 + 16);
                 uint4 o;
-                o.x = pack_bf16x2(__uint_as_float(a.x), __uint_as_float(a.y));
-                o.y = pack_bf16x2(__uint_as_float(a.z), __uint_as_float(a.w));
-                o.z = pack_bf16x2(__uint_as_float(b.x), __uint_as_float(b.y));
-                o.w = pack_bf16x2(__uint_as_float(b.z), __uint_as_float(b.w));
+                o.x = cvt_bf16x2(__uint_as_float(a.x), __uint_as_float(a.y));
+                o.y = cvt_bf16x2(__uint_as_float(a.z), __uint_as_float(a.w));
+                o.z = cvt_bf16x2(__uint_as_float(b.x), __uint_as_float(b.y));
+                o.w = cvt_bf16x2(__uint_as_float(b.z), __uint_as_float(b.w));
+                if (nan_halves(o.x) | nan_halves(o.y) | nan_halves(o.z) | nan_halves(o.w)) {   // rare: a NaN among the eight
+                    o.x = fix_nan_halves(o.x); o.y = fix_nan_halves(o.y);
+                    o.z = fix_nan_halves(o.z); o.w = fix_nan_halves(o.w);
+                }
                 const uint32_t doff = r * m.dp + c * 16;
                 for (uint32_t j = 0; j < m.reps; ++j)
                     st_stream(tile_dst(p, m.dst_buf, m.rstride, m.d_off, j) + doff, o);

@@ -552,6 +552,8 @@ struct StageMeta {
     uint32_t nr, w, dp;
     uint32_t kind;          // kStageData, kStageEnd or kStageFlush
     uint16_t dst_buf, reps, rstride, cast;
+    uint32_t magic;         // converting ring: ceil(2^32 / (w / 16)), so that a row index is one multiply
+    uint32_t reserved;
 };
 constexpr uint32_t kStageData = 0, kStageEnd = 1, kStageFlush = 2;
 
@@ -711,6 +713,9 @@ __device__ __forceinline__ void ring_producer(const WalkParams& p, const Ring& R
                     m.d_off = t.d_off; m.nr = t.nr; m.w = t.w; m.dp = t.dp;
                     m.dst_buf = (uint16_t)t.dst_buf; m.reps = (uint16_t)t.reps; m.rstride = (uint16_t)t.rstride;
                     m.cast = (uint16_t)t.cast;
+                    // 16-byte units per row piece; a stage holds fewer than 2^16 of them, so umulhi(idx, magic)
+                    // is idx / units exactly (units = 1: the quotient is idx itself, flagged by magic = 0)
+                    m.magic = (kCast && t.nr > 1 && (t.w >> 4) > 1) ? 0xFFFFFFFFu / (t.w >> 4) + 1u : 0u;
                     m.kind = kStageData;
                     mbar_arrive_expect_tx(bar, t.nr * ws);
                 }
@@ -814,39 +819,41 @@ __device__ __forceinline__ void ring_consumer_cast(const WalkParams& p, const Ri
             __syncwarp();
             if (lane == 0 && unpublished) atomicAdd(&ctrl->done, unpublished);
             unpublished = 0;
-        } else if (!m.cast) {
-            // a bit-copy tile of a mixed table: 16 bytes per lane straight from the stage
-            const unsigned char* src = R.data + (size_t)stage * R.stage_bytes;
-            const uint32_t vpr = m.w >> 4, nvec = m.nr * vpr;
-#pragma unroll 2
-            for (uint32_t idx = ct; idx < nvec; idx += kCastConsumers) {
-                const uint32_t r = idx / vpr, c = idx - r * vpr;
-                const uint4 v = *reinterpret_cast<const uint4*>(src + r * m.w + c * 16);
-                const uint32_t doff = r * m.dp + c * 16;
-                for (uint32_t j = 0; j < m.reps; ++j)
-                    st_stream(tile_dst(p, m.dst_buf, m.rstride, m.d_off, j) + doff, v);
-            }
-            ++unpublished;
         } else {
+            // The stage holds the tile's row pieces back to back, so unit idx sits at idx * (bytes per unit) and
+            // only its destination needs the row: idx * 16 + row * (pitch - width).  Rows come from one multiply
+            // with the reciprocal the producer left in the record (a 32-bit division per unit would be a third
+            // of this loop's instructions).
             const unsigned char* src = R.data + (size_t)stage * R.stage_bytes;
-            const uint32_t upr = m.w >> 4, nunit = m.nr * upr, ws = m.w << 1;
+            const uint32_t nunit = (m.nr * m.w) >> 4, gap = m.dp - m.w;
+            auto row_of = [&m](uint32_t idx) { return m.nr == 1 ? 0u : (m.magic ? __umulhi(idx, m.magic) : idx); };
+            if (!m.cast) {
+                // a bit-copy tile of a mixed table: 16 bytes per lane straight from the stage
 #pragma unroll 2
-            for (uint32_t idx = ct; idx < nunit; idx += kCastConsumers) {
-                const uint32_t r = idx / upr, c = idx - r * upr;
-                const uint4 a = *reinterpret_cast<const uint4*>(src + r * ws + c * 32);
-                const uint4 b = *reinterpret_cast<const uint4*>(src + r * ws + c * 32 + 16);
-                uint4 o;
-                o.x = cvt_bf16x2(__uint_as_float(a.x), __uint_as_float(a.y));
-                o.y = cvt_bf16x2(__uint_as_float(a.z), __uint_as_float(a.w));
-                o.z = cvt_bf16x2(__uint_as_float(b.x), __uint_as_float(b.y));
-                o.w = cvt_bf16x2(__uint_as_float(b.z), __uint_as_float(b.w));
-                if (nan_halves(o.x) | nan_halves(o.y) | nan_halves(o.z) | nan_halves(o.w)) {   // rare: a NaN among the eight
-                    o.x = fix_nan_halves(o.x); o.y = fix_nan_halves(o.y);
-                    o.z = fix_nan_halves(o.z); o.w = fix_nan_halves(o.w);
+                for (uint32_t idx = ct; idx < nunit; idx += kCastConsumers) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(src + idx * 16);
+                    const uint32_t doff = idx * 16 + row_of(idx) * gap;
+                    for (uint32_t j = 0; j < m.reps; ++j)
+                        st_stream(tile_dst(p, m.dst_buf, m.rstride, m.d_off, j) + doff, v);
                 }
-                const uint32_t doff = r * m.dp + c * 16;
-                for (uint32_t j = 0; j < m.reps; ++j)
-                    st_stream(tile_dst(p, m.dst_buf, m.rstride, m.d_off, j) + doff, o);
+            } else {
+#pragma unroll 2
+                for (uint32_t idx = ct; idx < nunit; idx += kCastConsumers) {
+                    const uint4 a = *reinterpret_cast<const uint4*>(src + idx * 32);
+                    const uint4 b = *reinterpret_cast<const uint4*>(src + idx * 32 + 16);
+                    uint4 o;
+                    o.x = cvt_bf16x2(__uint_as_float(a.x), __uint_as_float(a.y));
+                    o.y = cvt_bf16x2(__uint_as_float(a.z), __uint_as_float(a.w));
+                    o.z = cvt_bf16x2(__uint_as_float(b.x), __uint_as_float(b.y));
+                    o.w = cvt_bf16x2(__uint_as_float(b.z), __uint_as_float(b.w));
+                    if (nan_halves(o.x) | nan_halves(o.y) | nan_halves(o.z) | nan_halves(o.w)) {   // rare: a NaN among the eight
+                        o.x = fix_nan_halves(o.x); o.y = fix_nan_halves(o.y);
+                        o.z = fix_nan_halves(o.z); o.w = fix_nan_halves(o.w);
+                    }
+                    const uint32_t doff = idx * 16 + row_of(idx) * gap;
+                    for (uint32_t j = 0; j < m.reps; ++j)
+                        st_stream(tile_dst(p, m.dst_buf, m.rstride, m.d_off, j) + doff, o);
+                }
             }
             ++unpublished;
         }

@@ -389,8 +389,10 @@ int nereus_dag_lower(nereus_dag_t dag, const nereus_model_desc_t* descs, int n_d
  * cudaMemcpyAsync and a 12-byte memset ahead of the kernel).
  *   - A transition with more tasks (nereus_transition_num_rects), or with more than 4 * NEREUS_STATIC_MAX_RECTS
  *     (task, replica) pairs, is refused with NEREUS_ERR_TOO_LARGE.
- *   - The first call on a device looks the array's device address up (cudaGetSymbolAddress) and reads the
- *     SM count.  While `cuda_stream` is being captured the call is refused with NEREUS_ERR_UNSUPPORTED: the
+ *   - The first call on a device does the set-up for that device: it looks the array's device address up
+ *     (cudaGetSymbolAddress), reads the SM count and opts the kernels into their shared memory.  Make that
+ *     first call before any stream capture begins.  While `cuda_stream` is being captured every call is
+ *     refused with NEREUS_ERR_UNSUPPORTED: the
  *     table is uploaded from host arrays that the next call overwrites, so a captured upload would replay
  *     whichever table came last.
  *   - The uploads read pageable host memory: the runtime takes the bytes before each copy call returns, and

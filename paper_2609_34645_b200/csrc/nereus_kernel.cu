@@ -938,7 +938,8 @@ struct Launch {
 //   * otherwise tables that write 64 MiB or more: the ring (its per-block start-up costs more than it gains
 //     below that); all-bit-copy tables on the bulk-store consumer, anything with a cast in it on the
 //     converting consumers (which copy the bit-copy tiles of a mixed table from shared memory as well);
-//   * what is left (small chained tables, small tables with very many buffers): the persistent vector kernel.
+//   * what is left (small chained tables, small tables with very many buffers, large bit-copy tables with 4% or
+//     more of their bytes in row pieces below 1 KiB): the persistent vector kernel.
 static int resolve_launch(const nereus_transition_s& t, int sms, Launch& L, bool once_fits = true) {
     const int want = t.tuning.variant ? t.tuning.variant : env_int("NEREUS_VARIANT", 0);
     const int asked_tile = t.tuning.tile_bytes ? t.tuning.tile_bytes : env_int("NEREUS_TILE_BYTES", 0);
@@ -950,6 +951,15 @@ static int resolve_launch(const nereus_transition_s& t, int sms, Launch& L, bool
     else if (once_ok && t.bytes_written < (1ull << 30)) L.variant = 3;
     else       L.variant = (t.bytes_written >= (64ull << 20) && asked_tile <= (L.cast ? 24576 : 49152)) ? 2 : 1;
     if (L.variant == 3 && !once_ok) L.variant = 1;
+    if (!want && L.variant == 2 && !L.cast && t.n_levels == 1) {
+        // Row pieces below 1 KiB travel as one bulk copy each, and at 512 bytes those cost the ring 4 - 5% of a
+        // whole 8B table in which they are 8% of the bytes (TP 16: 6.54 TB/s against 6.84 at 1 KiB pieces), while
+        // the vector kernel moves them at its usual rate (6.72): it takes such tables.
+        uint64_t small = 0;
+        for (const Rect& r : t.rects)
+            if (r.rows > 1 && r.width_dst < 1024) small += r.rows * r.width_dst * (uint64_t)r.replicas;
+        if (small * 25 >= t.bytes_written) L.variant = 1;
+    }
     L.ctas_per_sm = t.tuning.ctas_per_sm ? t.tuning.ctas_per_sm : env_int("NEREUS_CTAS_PER_SM", 2);
     L.threads     = t.tuning.threads     ? t.tuning.threads     : env_int("NEREUS_THREADS", L.variant == 3 ? 256 : 384);
     L.tile_bytes  = asked_tile;

@@ -498,6 +498,10 @@ def test_launch_shapes_without_a_device():
     li = big.launch_info()
     assert (li["kernel"], li["tile_bytes"], li["grid"], li["threads"]) == ("nereus_walk_ring", 32768, 148, 64)
     assert big.num_tiles() == (506756, 1)
+    # 512-byte row pieces (wo at TP16) in 8% of the bytes: the large table goes to the vector kernel
+    tp16 = desc_of(I.LLAMA_8B).compile(B.Plan(4, 1), B.Plan(16, 1))
+    assert tp16.launch_info()["kernel"] == "nereus_walk_vec" and tp16.launch_info()["tile_bytes"] == 16384
+    assert desc_of(I.LLAMA_8B).compile(B.Plan(4, 1), B.Plan(8, 1)).launch_info()["kernel"] == "nereus_walk_ring"
     mid = desc_of(I.Shape(2, 2048, 16, 8, 5632, 8192)).compile(B.Plan(1, 1), B.Plan(4, 1))
     li = mid.launch_info()
     assert li["kernel"] == "nereus_walk_once" and li["tile_bytes"] == 4096

@@ -211,7 +211,9 @@ int nereus_debug_set_rect(nereus_transition_t t, int index, const nereus_rect_t*
  * takes `threads` only (its grid follows the tile count).
  * variant: which kernel walks the table.
  *   0  default: kernel 3 for single-level tables that write less than 1 GiB through at most 64 buffers;
- *      otherwise kernel 2 for tables that write 64 MiB or more and kernel 1 below that
+ *      otherwise kernel 2 for tables that write 64 MiB or more and kernel 1 below that; kernel 1 also for large
+ *      bit-copy tables with 4% or more of their bytes in row pieces shorter than 1 KiB (each such piece is one
+ *      bulk copy in kernel 2, which costs it more than the register path)
  *   1  persistent register-staged vector copy: a warp per tile, tiles claimed from a cursor (16 KiB tiles,
  *      smaller for small tables until every other warp finds work)
  *   2  persistent bulk-copy ring through shared memory (32 KiB per stage; 24 KiB when the table contains a
@@ -236,7 +238,7 @@ int nereus_transition_launch_info(nereus_transition_t t, int* variant, int* tile
  * tile, which saves the kernel the search for a tile's task.  Errors: ARG, UNSUPPORTED, NEREUS_ERR_TABLE, CUDA. */
 int nereus_transition_prepare(nereus_transition_t t);
 /* Enqueues the whole transition on `cuda_stream` (a cudaStream_t; NULL = the default stream) as one
- * persistent kernel and returns without synchronising.
+ * kernel launch and returns without synchronising.
  *   src_ptrs (host array of device pointers): source shard i = p*tp + r; read-only during the run.
  *   dst_ptrs (host array of device pointers): destination shards; every byte of every stored tensor is
  *            written exactly once, padding is untouched.

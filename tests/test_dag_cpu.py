@@ -62,6 +62,75 @@ def figure_changes():
     return [reward, actor, critic]
 
 
+# ---------------------------------------------------------------- the paper's examples, from the golden file
+
+def _parse_unit(text):
+    layout, where = text.split("@")
+    tp, pp = (int(x) for x in layout.split("x"))
+    if "+" in where or "-" in where:
+        gpus = []
+        for part in where.split("+"):
+            lo, _, hi = part.partition("-")
+            gpus += list(range(int(lo), int(hi or lo) + 1))
+    else:
+        gpus = list(range(int(where), int(where) + tp * pp))
+    assert len(gpus) == tp * pp, text
+    return D.Unit(tp, pp, tuple(gpus))
+
+
+def golden_examples():
+    import os
+    kinds = {"generation": D.GENERATION, "inference": D.INFERENCE, "training": D.TRAINING}
+    out, cur = [], None
+    with open(os.path.join(os.path.dirname(__file__), "golden", "dag_examples.txt")) as f:
+        for line in f:
+            w = line.split("#")[0].split()
+            if not w:
+                continue
+            if w[0] == "example":
+                cur = {"name": w[1], "stages": [], "tsub": {}, "ops": {}, "waits": []}
+            elif w[0] == "stage":
+                t = w.index("target")
+                cur["stages"].append(D.StageChange(kinds[w[1]], [_parse_unit(u) for u in w[3:t]],
+                                                   [_parse_unit(u) for u in w[t + 1:]], S))
+            elif w[0] == "tsub":
+                cur["tsub"][int(w[1])] = tuple(int(x) for x in w[2].split("x"))
+            elif w[0] == "ops":
+                cur["ops"][int(w[1])] = w[2:]
+            elif w[0] == "waits":
+                (m, op), (n, rel) = (x.split(":") for x in w[1:3])
+                cur["waits"].append((int(m), op, int(n), rel))
+            elif w[0] == "end":
+                out.append(cur)
+    return out
+
+
+@pytest.mark.parametrize("ex", golden_examples(), ids=lambda e: e["name"])
+def test_examples_the_paper_gives(ex):
+    """tests/golden/dag_examples.txt: each example with unlimited memory (the decomposition), and, where the
+    paper names a wait, once more with every GPU full (the resource-dependency edges)."""
+    changes = ex["stages"]
+    units, prims = planned(changes)
+    for m, want in ex["tsub"].items():
+        assert D.t_sub(changes[m].current[0], changes[m].target[0]) == want
+        subs = [units[u][1:3] for p in prims if p["stage"] == m and p["op"] == D.SPLIT for u in p["dst"]]
+        assert all(x == want for x in subs)
+    for m, want in ex["ops"].items():
+        assert ops(prims, m) == want, (ex["name"], m)
+    assert not any(p["resource_deps"] for p in prims)
+    if ex["waits"]:
+        # full GPUs: room for the largest shard that has to sit anywhere plus one split's worth of new shards
+        cap = max(ch.state_bytes // (u.tp * u.pp) for ch in changes for u in ch.current + ch.target)
+        cap += max([ch.state_bytes // (D.t_sub(ch.current[0], ch.target[0])[0] * D.t_sub(ch.current[0], ch.target[0])[1])
+                    for ch in changes if (ch.current[0].tp, ch.current[0].pp) != D.t_sub(ch.current[0], ch.target[0])] or [0]) // 2
+        units, prims = planned(changes, cap)
+        for m, op, n, rel in ex["waits"]:
+            waiting = [p for p in prims if p["stage"] == m and D.OP_NAMES[p["op"]] == op]
+            assert waiting and all(
+                any(prims[r]["stage"] == n and D.OP_NAMES[prims[r]["op"]] == rel for r in p["resource_deps"])
+                for p in waiting), (ex["name"], m, op)
+
+
 def test_reward_inference_example_of_the_dag_figure():
     """(TP4, PP8) is split into four (TP4, PP2) units, two are destroyed, the remaining two are merged into
     (TP8, PP2); actor and critic Extend onto GPUs 49-64 wait for the reward Destroys that release them."""

@@ -40,36 +40,6 @@ def _workload_bytes(name):
     return tot
 
 
-def _sample_ids(L):
-    layers = sorted({0, L // 2, L - 1})
-    ids = [0, 9 * L + 1, 9 * L + 2]
-    for l in layers:
-        ids += list(range(1 + 9 * l, 10 + 9 * l))
-    return ids
-
-
-def _check_stage_sampled(st, src, dst, src_plan, dst_plan, ids=None):
-    """Oracle parity of sampled logical tensors: src/dst are the stage's device buffers."""
-    sh = st.shape
-    m = O.Model(sh.layers, sh.hidden, sh.heads, sh.kv_heads, sh.ffn, sh.vocab, ODT[src_plan[2]], st.value_head)
-    pa, pb = O.Plan(src_plan[0], src_plan[1]), O.Plan(dst_plan[0], dst_plan[1], ODT[dst_plan[2]])
-    ses, des = I.element_size(src_plan[2]), I.element_size(dst_plan[2])
-    for tid in ids or _sample_ids(sh.layers):
-        sparts, dparts, where = [], [], []
-        for s in range(O.num_shards(m, pa)):
-            p = O.locate(m, pa, s, tid)
-            sparts.append(src[s][p.offset:p.offset + p.nr * p.nc * ses].cpu().numpy() if p.held else None)
-        for d in range(O.num_shards(m, pb)):
-            p = O.locate(m, pb, d, tid)
-            dparts.append(np.empty(p.nr * p.nc * des, np.uint8) if p.held else None)
-            where.append(p)
-        O.reshard_tensor_parts(m, pa, pb, tid, sparts, dparts)
-        for d, (p, want) in enumerate(zip(where, dparts)):
-            if p.held:
-                got = dst[d][p.offset:p.offset + want.size].cpu().numpy()
-                assert np.array_equal(got, want), f"stage {st.name} logical tensor {tid} dst shard {d}"
-
-
 def _check_stage_sums(st, desc, src, dst, pa, pb, sdt, ddt):
     """Every stored tensor: element sums agree between the two sides; replicas agree with the first copy."""
     ses, des = I.element_size(sdt), I.element_size(ddt)

@@ -520,7 +520,10 @@ def run_ours(args):
                                     "sample": f"failed: {e!r}"}
     if world == 1 and args.others != "none" and args.workload == DEFAULT_WORKLOAD:
         del srcs, dsts, sp, dp, t, keep, wl
-        line["workloads"] = measure_others(args, device, gpu_id, peak, peak_kind)
+        try:                        # the headline above never depends on what follows
+            line["workloads"] = measure_others(args, device, gpu_id, peak, peak_kind)
+        except Exception as e:
+            line["workloads"] = [{"error": repr(e)}]
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -554,6 +557,11 @@ def measure_others(args, device, gpu_id, peak, peak_kind):
             wl, t, srcs, dsts, keep = build_workload(name, device, tune, check_fit=True)
         except DoesNotFit as e:
             out.append({"workload": name, "skipped": str(e)})
+            continue
+        except Exception as e:      # e.g. an allocation that fails although the pre-flight passed
+            out.append({"workload": name, "skipped": f"could not be set up: {e!r}"})
+            gc.collect()
+            torch.cuda.empty_cache()
             continue
         rd, wr = t.bytes()
         sp = B.Transition.pointer_array([b.data_ptr() for b in srcs])

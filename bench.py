@@ -697,10 +697,14 @@ def run_e2e(args, t, srcs, dsts, sp, dp, stream, algo_bytes, world, device):
     free, _ = torch.cuda.mem_get_info(device)
     aliased = {b.data_ptr() for b in srcs} & {b.data_ptr() for b in dsts}
     if not aliased and need * 1.02 + (2 << 30) < free:
-        srcs2 = [torch.empty_like(b) for b in srcs]
-        dsts2 = [torch.empty_like(b) for b in dsts]
-        sets.append((srcs2, dsts2, B.Transition.pointer_array([b.data_ptr() for b in srcs2]),
-                     B.Transition.pointer_array([b.data_ptr() for b in dsts2])))
+        try:
+            srcs2 = [torch.empty_like(b) for b in srcs]
+            dsts2 = [torch.empty_like(b) for b in dsts]
+            sets.append((srcs2, dsts2, B.Transition.pointer_array([b.data_ptr() for b in srcs2]),
+                         B.Transition.pointer_array([b.data_ptr() for b in dsts2])))
+        except Exception:           # no room after all: one set, one step after the other
+            srcs2 = dsts2 = None
+            torch.cuda.empty_cache()
     n = len(sets)
     s_in, s_out = (torch.cuda.Stream(device), torch.cuda.Stream(device)) if n == 2 else (stream, stream)
     ev_in = [torch.cuda.Event() for _ in range(n)]

@@ -503,6 +503,11 @@ def run_ours(args):
     per_stage = time_stages_alone(wl, keep, srcs, dsts, stream)
     if per_stage:
         line["config"]["ms_per_stage_alone"] = per_stage
+    if world == 1:
+        try:
+            line["config"]["balance"] = block_balance(t, sp, dp, stream)
+        except Exception as e:      # a diagnostic, never a dependency of the number
+            line["config"]["balance"] = {"error": repr(e)}
     if not args.no_cpu_baseline and world == 1:
         try:
             from oracle import oracle as O
@@ -611,8 +616,34 @@ def measure_others(args, device, gpu_id, peak, peak_kind):
         alone = time_stages_alone(wl, keep, srcs, dsts, stream)
         if alone:
             out[-1]["ms_per_stage_alone"] = alone        # every model-stage's transition launched on its own
+        try:
+            out[-1]["balance"] = block_balance(t, sp, dp, stream)
+        except Exception as e:
+            out[-1]["balance"] = {"error": repr(e)}
         del srcs, dsts, sp, dp, t, keep, wl, flush
     return out
+
+
+def block_balance(t, sp, dp, stream):
+    """One traced run (outside every timed region): how evenly the blocks of the launch were loaded and how far
+    apart they finished, from the GPU's global timer."""
+    import torch
+
+    t.trace(True)
+    t.prepare()
+    for _ in range(2):
+        t.run(sp, dp, stream.cuda_stream)
+    torch.cuda.synchronize()
+    rec = [r for r in t.trace_read() if r[3]]
+    t.trace(False)
+    t.prepare()
+    if not rec:
+        return None
+    begin, ends = min(r[1] for r in rec), [r[2] for r in rec]
+    return {"blocks": len(rec), "tiles_min": min(r[3] for r in rec), "tiles_max": max(r[3] for r in rec),
+            "start_spread_us": (max(r[1] for r in rec) - begin) / 1e3,
+            "first_block_done_us": (min(ends) - begin) / 1e3, "last_block_done_us": (max(ends) - begin) / 1e3,
+            "finish_spread_us": (max(ends) - min(ends)) / 1e3}
 
 
 def host_memory_budget() -> int:

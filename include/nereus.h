@@ -273,6 +273,18 @@ int nereus_transition_status(nereus_transition_t t, int* device_status);
 /* Kernels this handle has launched since it was created (one per run). */
 int nereus_transition_launches(nereus_transition_t t, uint64_t* n);
 
+/* Per-block trace of a run, for looking at load balance (who got how many tiles, how far apart the blocks
+ * finish): the tool this library offers where the paper's framework instrumentation provides kernel times
+ * (Section 4.1, monitor phase).  nereus_transition_trace(t, 1) switches it on (and drops the device copy of the
+ * table, like nereus_transition_tune); every run then zeroes the trace (one small memset in front of the
+ * kernel, so a traced run is not what one times) and every block records the GPU's global timer when it starts
+ * and when it finishes and the number of tiles it moved.  nereus_transition_trace_read copies the records of
+ * the last run to `out` (host, `cap` entries; *n gets the number of blocks) after the caller has synchronised.
+ * Errors: ARG (also: tracing is off, cap too small), CUDA. */
+typedef struct { uint64_t begin_ns, end_ns; uint32_t tiles, block; } nereus_block_trace_t;
+int nereus_transition_trace(nereus_transition_t t, int enable);
+int nereus_transition_trace_read(nereus_transition_t t, nereus_block_trace_t* out, int cap, int* n);
+
 /* ---- cost side: the transition estimate and the admission gate (Sections 4.3 and 6) ------------------- */
 
 /* L_tran of a compiled transition: in the paper the critical-path cost is a function of the bytes moved, the

@@ -80,6 +80,12 @@ class Horizon(ctypes.Structure):
         return self.h_steps
 
 
+class BlockTrace(ctypes.Structure):
+    """nereus_block_trace_t: one block of a traced run."""
+    _fields_ = [("begin_ns", ctypes.c_uint64), ("end_ns", ctypes.c_uint64), ("tiles", ctypes.c_uint32),
+                ("block", ctypes.c_uint32)]
+
+
 class PrimInfo(ctypes.Structure):
     """nereus_prim_t."""
     _fields_ = [(n, ctypes.c_int32) for n in ("op", "stage", "n_src", "n_dst", "n_deps", "n_resource_deps",
@@ -116,6 +122,8 @@ _SIGS = {
     "nereus_transition_run_sized": [_vp, _P(_vp), _P(_sz), _P(_vp), _P(_sz), _vp],
     "nereus_transition_status": [_vp, _P(_i)],
     "nereus_transition_launches": [_vp, _P(ctypes.c_uint64)],
+    "nereus_transition_trace": [_vp, _i],
+    "nereus_transition_trace_read": [_vp, _P(BlockTrace), _i, _P(_i)],
     "nereus_last_cuda_error": [],
     "nereus_dag_create": [_P(_vp)],
     "nereus_dag_destroy": [_vp],
@@ -358,6 +366,17 @@ class Transition:
         s = _i()
         _ck(_lib.nereus_transition_status(self._h, ctypes.byref(s)), "nereus_transition_status")
         return s.value
+
+    def trace(self, enable=True) -> None:
+        """Switches the per-block trace on or off (drops the device copy of the table)."""
+        _ck(_lib.nereus_transition_trace(self._h, int(enable)), "nereus_transition_trace")
+
+    def trace_read(self) -> list:
+        """[(block, begin_ns, end_ns, tiles)] of the last run; the caller has synchronised."""
+        cap = max(1, self.launch_info()["grid"])
+        arr, n = (BlockTrace * cap)(), _i()
+        _ck(_lib.nereus_transition_trace_read(self._h, arr, cap, ctypes.byref(n)), "nereus_transition_trace_read")
+        return [(r.block, r.begin_ns, r.end_ns, r.tiles) for r in arr[:n.value]]
 
     def launches(self) -> int:
         n = ctypes.c_uint64()

@@ -126,6 +126,14 @@ struct Ctrl {
 };
 static_assert(sizeof(Ctrl) == 32, "Ctrl is one 32-byte sector");
 
+// Optional per-block trace of one run (nereus_transition_trace): when the block started, when it finished, how
+// many tiles it moved.  Same layout as nereus_block_trace_t.
+struct BlockTrace {
+    uint64_t begin_ns, end_ns;   // the GPU's global timer
+    uint32_t tiles, block;
+};
+static_assert(sizeof(BlockTrace) == sizeof(nereus_block_trace_t), "BlockTrace is the public record");
+
 constexpr int kMaxBuffers = 448;      // pointers carried in the kernel's parameter block
 constexpr int kMaxLevels  = 8;
 constexpr int kMaxReplicas = 16;
@@ -143,6 +151,8 @@ struct DeviceTable {                  // one per prepare()
     RectDev*  rects     = nullptr;
     uint32_t* first     = nullptr;    // n_rects + 1 tile prefix
     TileRec*  tiles     = nullptr;    // n_tiles records, or null for tables beyond kDirectMaxTiles
+    BlockTrace* trace   = nullptr;    // one record per block of the launch, or null when tracing is off
+    uint32_t  trace_blocks = 0;
     Ctrl*     ctrl      = nullptr;    // the control block
     uint32_t  runs      = 0;          // runs launched on this device copy
     uint32_t  n_tiles   = 0;
@@ -163,6 +173,7 @@ struct nereus_transition_s {
     int                       n_levels = 1;
     uint64_t                  bytes_read = 0, bytes_written = 0;
     nereus::Tuning            tuning;
+    bool                      trace = false;  // nereus_transition_trace
     nereus::DeviceTable       dev;
     uint64_t                  launches = 0;
 };

@@ -58,6 +58,7 @@ struct WalkParams {
     const uint32_t* first;        // n_rects + 1
     const TileRec*  tiles;        // n_tiles records, or null
     Ctrl*           ctrl;
+    BlockTrace*     trace;        // one record per block, or null
     uint32_t        n_rects, n_tiles, n_levels;
     uint32_t        level_end[kMaxLevels];
     char*           bufs[kMaxBuffers];
@@ -391,6 +392,24 @@ __device__ __forceinline__ bool resolve_direct(const WalkParams& p, uint32_t g, 
     return true;
 }
 
+__device__ __forceinline__ uint64_t global_nanos() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Tracing (off unless nereus_transition_trace switched it on): a block's first thread notes when the block
+// starts and ends, every warp adds the tiles it moved.
+__device__ __forceinline__ void trace_begin(BlockTrace* trace) {
+    if (trace && threadIdx.x == 0) { trace[blockIdx.x].begin_ns = global_nanos(); trace[blockIdx.x].block = blockIdx.x; }
+}
+__device__ __forceinline__ void trace_tiles(BlockTrace* trace, uint32_t n, unsigned lane) {
+    if (trace && lane == 0 && n) atomicAdd(&trace[blockIdx.x].tiles, n);
+}
+__device__ __forceinline__ void trace_end(BlockTrace* trace) {           // after the block's closing barrier
+    if (trace && threadIdx.x == 0) trace[blockIdx.x].end_ns = global_nanos();
+}
+
 __device__ __forceinline__ void raise_status(Ctrl* ctrl, uint32_t status, uint32_t detail) {
     if (atomicCAS(&ctrl->status, (uint32_t)NEREUS_DEV_OK, status) == (uint32_t)NEREUS_DEV_OK) ctrl->detail = detail;
 }
@@ -421,7 +440,9 @@ __global__ void __launch_bounds__(512, 2) nereus_walk_vec(const __grid_constant_
     Ctrl* const    ctrl = p.ctrl;
     uint32_t       my_done = 0, my_level = 0;                  // tiles completed and not yet published
     uint32_t       open_level = 0;                             // highest level whose gate this warp has passed
+    uint32_t       moved = 0;                                  // tiles this warp moved (for the trace)
     RectRange      rr;
+    trace_begin(p.trace);
 
     // tables without per-tile records: the tile prefix is copied to shared memory once per CTA (when it fits),
     // so that resolving a tile costs one trip to memory (the rect record) instead of a chain of dependent ones
@@ -489,6 +510,7 @@ __global__ void __launch_bounds__(512, 2) nereus_walk_vec(const __grid_constant_
             copy_rect<kUnrollRect, false>(t.s, D, t.reps, t.nr, t.w >> 4, t.sp, t.dp, lane);
         }
         if (p.n_levels > 1) ++my_done;
+        ++moved;
         g = more ? base + claim_take(next_issued) : p.n_tiles;
     }
     if (my_done) {
@@ -496,7 +518,9 @@ __global__ void __launch_bounds__(512, 2) nereus_walk_vec(const __grid_constant_
         __syncwarp();
         if (lane == 0) atomicAdd(&ctrl->done, my_done);
     }
+    trace_tiles(p.trace, moved, lane);
     finish_block(ctrl);
+    trace_end(p.trace);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -514,6 +538,7 @@ constexpr int kOnceMaxBuffers = 64;
 struct OnceParams {
     const TileRec* tiles;
     Ctrl*          ctrl;
+    BlockTrace*    trace;         // one record per block, or null
     uint32_t       n_tiles;
     char*          bufs[kOnceMaxBuffers];
 };
@@ -522,6 +547,11 @@ __global__ void __launch_bounds__(512, 2) nereus_walk_once(const __grid_constant
     const unsigned lane = threadIdx.x & 31;
     const uint32_t g = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (g >= p.n_tiles) return;
+    if (p.trace && lane == 0) {                      // no barrier in this kernel: first warp in, last warp out
+        BlockTrace* tr = p.trace + blockIdx.x;
+        if (atomicCAS(reinterpret_cast<unsigned long long*>(&tr->begin_ns), 0ull, (unsigned long long)global_nanos()) == 0ull)
+            tr->block = blockIdx.x;
+    }
     const uint4* q = reinterpret_cast<const uint4*>(p.tiles + g);
     const uint4 a = __ldg(q), b = __ldg(q + 1), c = __ldg(q + 2);
     const uint32_t src_buf = c.x & 0xFFFFu, dst_buf = c.x >> 16;
@@ -537,6 +567,13 @@ __global__ void __launch_bounds__(512, 2) nereus_walk_once(const __grid_constant
     if (cast)          cast_tile<kUnrollCast, true>(s, D, reps, b.z, b.w >> 3, b.x, b.y, lane);
     else if (b.z == 1) copy_run<kUnrollRun, true>(s, D, reps, b.w >> 4, lane);
     else               copy_rect<kUnrollRect, true>(s, D, reps, b.z, b.w >> 4, b.x, b.y, lane);
+    if (p.trace) {
+        __syncwarp();
+        if (lane == 0) {
+            atomicAdd(&p.trace[blockIdx.x].tiles, 1u);
+            atomicMax(reinterpret_cast<unsigned long long*>(&p.trace[blockIdx.x].end_ns), (unsigned long long)global_nanos());
+        }
+    }
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -571,11 +608,6 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 }
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ uint64_t global_nanos() {
-    uint64_t t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
 }
 // Bounded wait for the phase with the given parity; false when it gave up.  Two limits: a deadline of
 // kWaitNanos (half a second) on the global timer, read every 64 attempts once the first few have failed, and
@@ -637,7 +669,7 @@ __device__ __forceinline__ void wait_store_reads(uint32_t pending) {
 template <bool kCast>
 __device__ __forceinline__ void ring_producer(const WalkParams& p, const Ring& R, unsigned lane) {
     Ctrl* const ctrl = p.ctrl;
-    uint32_t    stage = 0, phase = 0, level = 0;
+    uint32_t    stage = 0, phase = 0, level = 0, moved = 0;
     RectRange   rr;
     // single-level tables: the first batch is the block's own index, the cursor hands out the batches beyond
     // the grid; chained tables take every batch from the cursor
@@ -727,11 +759,13 @@ __device__ __forceinline__ void ring_producer(const WalkParams& p, const Ring& R
                     for (uint32_t r = lane; r < t.nr; r += 32)
                         bulk_load(base + r * ws, t.s + (size_t)r * t.sp, ws, bar);
                 }
+                ++moved;
                 if (++stage == R.n_stages) { stage = 0; phase ^= 1; }
             }
         }
         g0 = last ? g0 : base + claim_take(next_issued);
     }
+    trace_tiles(p.trace, moved, lane);
 }
 
 // Consumer warp of the bit-copy ring: stores full stages with bulk copies, hands them back `lag` stages later.
@@ -884,6 +918,7 @@ nereus_walk_ring(const __grid_constant__ WalkParams p, const uint32_t stage_byte
     R.lag = lag;
     R.claim = claim;
     const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    trace_begin(p.trace);
 
     if (threadIdx.x == 0) {
         for (uint32_t i = 0; i < n_stages; ++i) {
@@ -898,6 +933,7 @@ nereus_walk_ring(const __grid_constant__ WalkParams p, const uint32_t stage_byte
     else if (kCast) ring_consumer_cast(p, R, threadIdx.x - 32);
     else ring_consumer_copy(p, R, lane);
     finish_block(p.ctrl);
+    trace_end(p.trace);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -910,6 +946,7 @@ static void drop_device_table(nereus_transition_s& t) {
         if (cudaGetDevice(&cur) == cudaSuccess) {
             if (cur != t.dev.device) cudaSetDevice(t.dev.device);
             if (t.dev.rects) cudaFree(t.dev.rects);
+            if (t.dev.trace) cudaFree(t.dev.trace);
             if (cur != t.dev.device) cudaSetDevice(cur);
         }
         (void)cudaGetLastError();
@@ -1044,7 +1081,7 @@ static int launch_walk(const Launch& L, int sms, const WalkParams& p, cudaStream
         }
     } else if (L.variant == 3 && p.tiles) {
         OnceParams o;
-        o.tiles = p.tiles; o.ctrl = p.ctrl; o.n_tiles = p.n_tiles;
+        o.tiles = p.tiles; o.ctrl = p.ctrl; o.trace = p.trace; o.n_tiles = p.n_tiles;
         for (int k = 0; k < kOnceMaxBuffers; ++k) o.bufs[k] = p.bufs[k];
         const unsigned warps_per_cta = (unsigned)L.threads / 32;
         nereus_walk_once<<<(p.n_tiles + warps_per_cta - 1) / warps_per_cta, L.threads, 0, stream>>>(o);
@@ -1109,6 +1146,20 @@ static int prepare(nereus_transition_s& t) {
         e = cudaMemcpy(dv.tiles, tiles.data(), tiles.size() * sizeof(TileRec), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemset(dv.ctrl, 0, ctrl_b);
     if (e != cudaSuccess) { cudaFree(base); set_cuda_error((int)e); (void)cudaGetLastError(); return NEREUS_ERR_CUDA; }
+    if (t.trace) {
+        // one record per block of the launch this table will get
+        const uint32_t warps = (uint32_t)L.threads / 32;
+        dv.trace_blocks = L.variant == 3 ? (dv.n_tiles + warps - 1) / warps : (uint32_t)(sms * L.ctas_per_sm);
+        dv.trace_blocks = std::max(1u, dv.trace_blocks);
+        e = cudaMalloc(&dv.trace, (size_t)dv.trace_blocks * sizeof(BlockTrace));
+        if (e == cudaSuccess) e = cudaMemset(dv.trace, 0, (size_t)dv.trace_blocks * sizeof(BlockTrace));
+        if (e != cudaSuccess) {
+            cudaFree(base);
+            if (dv.trace) cudaFree(dv.trace);
+            set_cuda_error((int)e); (void)cudaGetLastError();
+            return NEREUS_ERR_CUDA;
+        }
+    }
     t.dev = dv;
     return NEREUS_OK;
 }
@@ -1270,8 +1321,10 @@ int nereus_transition_run(nereus_transition_t t, const void* const* src_ptrs, vo
         if (L.variant != dv.variant || L.tile_bytes != dv.tile_bytes) return NEREUS_ERR_ARG;
         WalkParams p;
         // the control words need no reset: every launch leaves them zeroed for the next one
-        p.rects = dv.rects; p.first = dv.first; p.tiles = dv.tiles; p.ctrl = dv.ctrl;
+        p.rects = dv.rects; p.first = dv.first; p.tiles = dv.tiles; p.ctrl = dv.ctrl; p.trace = dv.trace;
         p.n_tiles = dv.n_tiles;
+        if (dv.trace)               // tracing: every run starts from an empty trace
+            NEREUS_CUDA(cudaMemsetAsync(dv.trace, 0, (size_t)dv.trace_blocks * sizeof(BlockTrace), stream));
         // NEREUS_DEBUG_GATE_BIAS (tests only): raises what a dependency gate waits for, so that it can never
         // open and the bounded wait must give up with NEREUS_DEV_TIMEOUT
         const uint32_t gate_bias = (uint32_t)env_int("NEREUS_DEBUG_GATE_BIAS", 0);
@@ -1301,6 +1354,21 @@ int nereus_transition_status(nereus_transition_t t, int* device_status) {
     if (!t->dev.rects) { *device_status = NEREUS_DEV_OK; return NEREUS_OK; }
     if (t->dev.runs == 0) { *device_status = NEREUS_DEV_OK; return NEREUS_OK; }
     return read_and_clear_status(t->dev.ctrl, device_status);
+}
+
+int nereus_transition_trace(nereus_transition_t t, int enable) {
+    if (!t) return NEREUS_ERR_ARG;
+    t->trace = enable != 0;
+    drop_device_table(*t);
+    return NEREUS_OK;
+}
+
+int nereus_transition_trace_read(nereus_transition_t t, nereus_block_trace_t* out, int cap, int* n) {
+    if (!t || !out || !n || cap < 0) return NEREUS_ERR_ARG;
+    if (!t->dev.trace || (uint32_t)cap < t->dev.trace_blocks) return NEREUS_ERR_ARG;
+    NEREUS_CUDA(cudaMemcpy(out, t->dev.trace, (size_t)t->dev.trace_blocks * sizeof(BlockTrace), cudaMemcpyDeviceToHost));
+    *n = (int)t->dev.trace_blocks;
+    return NEREUS_OK;
 }
 
 int nereus_transition_launches(nereus_transition_t t, uint64_t* n) {
@@ -1417,7 +1485,7 @@ extern "C" int nereus_transition_run_static(nereus_transition_t t, const void* c
     NEREUS_CUDA(cudaMemcpyAsync(d_first, g_static_first, (n_rects + 1) * sizeof(uint32_t), cudaMemcpyHostToDevice, stream));
     NEREUS_CUDA(cudaMemsetAsync(d_ctrl, 0, 3 * sizeof(uint32_t), stream));
 
-    p.rects = d_rects; p.first = d_first; p.tiles = nullptr; p.ctrl = d_ctrl;
+    p.rects = d_rects; p.first = d_first; p.tiles = nullptr; p.ctrl = d_ctrl; p.trace = nullptr;
     p.n_tiles = (uint32_t)n_tiles;
     const uint32_t gate_bias = (uint32_t)env_int("NEREUS_DEBUG_GATE_BIAS", 0);     // tests of the failure path only
     for (int k = 0; k < kMaxLevels; ++k) p.level_end[k] += gate_bias;

@@ -92,6 +92,40 @@ def test_run_with_declared_lengths():
     assert dst.guards_intact()
 
 
+@pytest.mark.parametrize("variant,chained", [(1, False), (2, False), (3, False), (1, True), (2, True)])
+def test_per_block_trace(variant, chained):
+    """Tracing on: every tile is accounted to exactly one block, blocks start before they end, the result is
+    still the oracle's; tracing off again: nothing to read."""
+    sh, a, b = I.SMALL, (1, 1), (4, 2)
+    d = G.desc_of(sh)
+    t = d.compile(B.Plan(*a), B.Plan(*b))
+    if chained:
+        t = B.Transition.fuse([t, d.compile(B.Plan(*b), B.Plan(*a))], chained=True)
+    t.tune(variant=variant, tile_bytes=2048)
+    t.trace(True)
+    src = G.device_sources(d, B.Plan(*a), "bf16", 21)
+    dst = G.Guarded([t.buffer_bytes(True, j) for j in range(t.num_buffers()[1])])
+    for _ in range(2):                                                   # the second run starts from an empty trace
+        G.run_transition(t, src, dst.bufs)
+    rec = t.trace_read()
+    grid = t.launch_info()["grid"]
+    assert 0 < len(rec) <= grid
+    assert sum(r[3] for r in rec) == t.num_tiles()[0]
+    busy = [r for r in rec if r[3]]
+    assert all(r[2] >= r[1] > 0 for r in busy) and [r[0] for r in busy] == sorted({r[0] for r in busy})
+    spread_us = (max(r[2] for r in busy) - min(r[1] for r in busy)) / 1e3
+    assert 0 < spread_us < 1e5
+    want = G.oracle_expected(sh, a, b, "bf16", "bf16", False, [s.cpu().numpy() for s in src])
+    for g, w in zip(dst.bufs[:8], want):
+        assert np.array_equal(g.cpu().numpy(), w)
+    assert dst.guards_intact()
+    t.trace(False)
+    G.run_transition(t, src, dst.bufs)
+    with pytest.raises(B.NereusError) as e:
+        t.trace_read()
+    assert e.value.code == B.ERR_ARG
+
+
 def test_many_runs_back_to_back_need_no_reset():
     """200 launches of one handle without a synchronise in between: each finds the control words zeroed by the
     one before it."""

@@ -427,6 +427,12 @@ def test_run_rejects_bad_pointers_before_any_cuda_call():
     assert t.run_sized_raw(src, sizes, dst, [need[0] - 256]) == B.ERR_TOO_SMALL
     assert t.run_sized_raw([0, src[1]], sizes, dst, need) == B.ERR_ARG            # then run()'s own checks
     assert "shorter" in B.strerror(B.ERR_TOO_SMALL)
+    # the per-block trace: nothing to read before a traced run has been prepared
+    t.trace(True)
+    with pytest.raises(B.NereusError) as e:
+        t.trace_read()
+    assert e.value.code == B.ERR_ARG
+    t.trace(False)
 
 
 # ---------------------------------------------------------------- replicas (Extend) and optimizer state
